@@ -1,0 +1,95 @@
+// Internal declarations shared by the translation units of libgdws.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "gdws.h"
+
+namespace gdws {
+
+constexpr int kChunk = 64;          // intermediate channels per tensor-core K chunk (one 128-byte swizzle row of bf16)
+constexpr int kTileRows = 128;      // output pixels per tensor-core tile (UMMA M)
+constexpr int kMaxK = 7;
+constexpr int kMaxSmem = 227 * 1024;
+
+// Bits of the device status word.
+enum : int {
+    kStatusWaitStage = 1,   // wait for a free shared-memory stage ran out
+    kStatusWaitOperand = 2, // wait for an operand (bulk copy / producer warps) ran out
+    kStatusWaitMma = 4,     // wait for the tensor-core commit ran out
+};
+
+struct Tile {
+    int TN = 0, PH = 0, PW = 0;      // images x rows x columns of output pixels per 128-row tile
+    int tiles_n = 0, tiles_h = 0, tiles_w = 0;
+    int IH = 0, IW = 0, IWp = 0;     // input patch rows / columns / row pitch (elements) per image
+    int plane = 0;                   // elements between consecutive channels in the staged input
+    int CB = 0;                      // channels per staged block
+    int nsb = 0;                     // pointwise-weight stages
+    size_t smem = 0;                 // dynamic shared memory of the fused kernel
+    int64_t tiles() const { return (int64_t)tiles_n * tiles_h * tiles_w; }
+};
+
+}  // namespace gdws
+
+struct gdws_plan_s {
+    int C = 0, D = 0, k = 0, stride = 0, pad = 0;
+    int G = 0, Gpad = 0, Dpad = 0, nchunks = 0;
+    std::vector<int32_t> g, off, chan;
+
+    int opt_path = GDWS_PATH_AUTO;
+    int opt_relu = 0;
+    int opt_tile = 0;
+    int opt_a_layout = 0;
+    int opt_dw_math = 0;
+
+    // device side (allocated by ensure_device)
+    int device = -1;
+    int32_t *d_off = nullptr;      // [C+1]
+    int32_t *d_chan = nullptr;     // [Gpad], -1 for padding
+    float *d_dw = nullptr;         // [Gpad][k*k] fp32 depthwise filters, zero rows for padding
+    uint32_t *d_dw2 = nullptr;     // [Gpad][k*k] the same filters as bf16 pairs (w,w)
+    uint16_t *d_pw_img = nullptr;  // [nchunks][Dpad*64] bf16, 128-byte-swizzled K-major operand images
+    float *d_bias = nullptr;       // [Dpad]
+    int *d_status = nullptr;       // device status word
+    bool packed = false;
+
+    void *ws = nullptr;
+    size_t ws_bytes = 0;
+
+    void *stage_x = nullptr, *stage_y = nullptr;  // gdws_forward_host staging
+    size_t stage_x_bytes = 0, stage_y_bytes = 0;
+
+    int64_t launches = 0;
+};
+
+namespace gdws {
+
+void set_error(const char *fmt, ...);
+gdws_status_t fail(gdws_status_t st, const char *fmt, ...);
+gdws_status_t cuda_fail(cudaError_t e, const char *what);
+gdws_status_t ensure_device(gdws_plan_s *p);   // allocate device tables on the current device
+gdws_status_t check_arch();
+bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *t);
+
+inline size_t dtype_size(gdws_dtype_t d) { return d == GDWS_F32 ? 4 : 2; }
+
+// f32.cu
+gdws_status_t f32_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, const float *dw_w, float *z, cudaStream_t s);
+gdws_status_t f32_pointwise(gdws_plan_s *p, const float *z, const float *pw_w, const float *bias,
+                            gdws_tensor_t *y, cudaStream_t s);
+gdws_status_t f32_fused(gdws_plan_s *p, const gdws_tensor_t *x, const float *dw_w, const float *pw_w,
+                        const float *bias, gdws_tensor_t *y, cudaStream_t s);
+
+// bf16.cu
+gdws_status_t bf16_pack(gdws_plan_s *p, const void *dw_w, const void *pw_w, const float *bias,
+                        gdws_dtype_t dtype, cudaStream_t s);
+gdws_status_t bf16_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cudaStream_t s);
+gdws_status_t bf16_pointwise(gdws_plan_s *p, const void *z, gdws_tensor_t *y, cudaStream_t s);
+gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t s);
+
+}  // namespace gdws

@@ -1,0 +1,331 @@
+// Host side of libgdws: plan construction, options, queries, tile choice, errors.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "gdws_internal.h"
+
+namespace gdws {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+gdws_status_t fail(gdws_status_t st, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+gdws_status_t cuda_fail(cudaError_t e, const char *what)
+{
+    snprintf(g_err, sizeof(g_err), "%s: %s", what, cudaGetErrorString(e));
+    return GDWS_ERR_CUDA;
+}
+
+gdws_status_t check_arch()
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+    if (major != 10)
+        return fail(GDWS_ERR_ARCH, "device %d has compute capability %d.x; this library needs 10.x (sm_100a)", dev, major);
+    return GDWS_OK;
+}
+
+static void free_device(gdws_plan_s *p)
+{
+    if (p->device < 0) return;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    cudaSetDevice(p->device);
+    cudaDeviceSynchronize();
+    cudaFree(p->d_off);
+    cudaFree(p->d_chan);
+    cudaFree(p->d_dw);
+    cudaFree(p->d_dw2);
+    cudaFree(p->d_pw_img);
+    cudaFree(p->d_bias);
+    cudaFree(p->d_status);
+    cudaFree(p->stage_x);
+    cudaFree(p->stage_y);
+    cudaSetDevice(cur);
+    p->device = -1;
+}
+
+gdws_status_t ensure_device(gdws_plan_s *p)
+{
+    if (p->device >= 0) return GDWS_OK;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    const size_t k2 = (size_t)p->k * p->k;
+    const size_t img = (size_t)p->nchunks * p->Dpad * kChunk * sizeof(uint16_t);
+#define GDWS_TRY_ALLOC(ptr, bytes)                                                   \
+    do {                                                                             \
+        e = cudaMalloc((void **)&(ptr), (bytes));                                    \
+        if (e != cudaSuccess) {                                                      \
+            p->device = dev;                                                         \
+            free_device(p);                                                          \
+            cudaGetLastError();                                                      \
+            return fail(GDWS_ERR_ALLOC, "cudaMalloc(%zu) failed: %s", (size_t)(bytes), cudaGetErrorString(e)); \
+        }                                                                            \
+    } while (0)
+    GDWS_TRY_ALLOC(p->d_off, sizeof(int32_t) * (p->C + 1));
+    GDWS_TRY_ALLOC(p->d_chan, sizeof(int32_t) * p->Gpad);
+    GDWS_TRY_ALLOC(p->d_dw, sizeof(float) * p->Gpad * k2);
+    GDWS_TRY_ALLOC(p->d_dw2, sizeof(uint32_t) * p->Gpad * k2);
+    GDWS_TRY_ALLOC(p->d_pw_img, img);
+    GDWS_TRY_ALLOC(p->d_bias, sizeof(float) * p->Dpad);
+    GDWS_TRY_ALLOC(p->d_status, sizeof(int));
+#undef GDWS_TRY_ALLOC
+    p->device = dev;
+    e = cudaMemcpy(p->d_off, p->off.data(), sizeof(int32_t) * (p->C + 1), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(p->d_chan, p->chan.data(), sizeof(int32_t) * p->Gpad, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_bias, 0, sizeof(float) * p->Dpad);
+    if (e != cudaSuccess) {
+        free_device(p);
+        return cuda_fail(e, "plan table upload");
+    }
+    return GDWS_OK;
+}
+
+static int round_up(int a, int b) { return (a + b - 1) / b * b; }
+
+// Shared-memory need of the fused bf16 kernel for a candidate tile.
+static size_t fused_smem(const gdws_plan_s *p, const Tile &t)
+{
+    size_t a = 2 * (size_t)kTileRows * kChunk * 2;                 // two intermediate-tile stages
+    size_t b = (size_t)t.nsb * p->Dpad * kChunk * 2;               // pointwise-weight stages
+    size_t x = 2 * (size_t)t.CB * t.plane * 2;                     // two staged input blocks
+    return a + b + x + 1024 /*alignment slack*/ + 256 /*barriers*/;
+}
+
+bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
+{
+    const int Ho = gdws_out_dim(h, p->k, p->stride, p->pad);
+    const int Wo = gdws_out_dim(w, p->k, p->stride, p->pad);
+    if (n < 1 || Ho < 1 || Wo < 1) return false;
+    double best = 1e300;
+    bool found = false;
+    const int forced = p->opt_tile;
+    static const int pws[4] = {32, 16, 8, 4};
+    for (int pi = 0; pi < 4; ++pi) {
+        const int PW = pws[pi];
+        for (int PH = 1; PH * PW <= kTileRows; ++PH) {
+            if (PW == 4 && (PH & 1)) continue;   // 4-wide patches pair two rows into one 8-pixel group
+            const int maxTN = kTileRows / (PH * PW);
+            for (int TN = 1; TN <= maxTN; ++TN) {
+                if (TN > 1 && (PH * PW) % 8) continue;
+                if (forced) {
+                    if (TN != ((forced >> 16) & 0xff) || PH != ((forced >> 8) & 0xff) || PW != (forced & 0xff)) continue;
+                }
+                Tile t;
+                t.TN = TN; t.PH = PH; t.PW = PW;
+                t.tiles_w = (Wo + PW - 1) / PW;
+                t.tiles_h = (Ho + PH - 1) / PH;
+                t.tiles_n = (n + TN - 1) / TN;
+                t.IH = (PH - 1) * p->stride + p->k;
+                t.IW = (PW - 1) * p->stride + p->k;
+                t.IWp = round_up(t.IW, 8);
+                int plane = TN * t.IH * t.IWp;        // elements; make the byte stride = 16 (mod 128)
+                while ((plane * 2) % 128 != 16) plane += 8;
+                t.plane = plane;
+                bool fits = false;
+                for (int CB = 16; CB >= 8 && !fits; CB -= 8) {
+                    // register prefetch of the next block: at most 12 16-byte loads per thread
+                    const int64_t loads = (int64_t)TN * t.IH * t.IWp * (CB / 8);
+                    if (loads > 12 * 256) continue;
+                    for (int nsb = 4; nsb >= 2 && !fits; --nsb) {
+                        t.CB = CB; t.nsb = nsb;
+                        t.smem = fused_smem(p, t);
+                        if (t.smem <= (size_t)kMaxSmem) fits = true;
+                    }
+                }
+                if (!fits) continue;
+                const double tiles = (double)t.tiles();
+                const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IWp) - 1e-3 * PW;
+                if (cost < best) { best = cost; *out = t; found = true; }
+            }
+        }
+    }
+    return found;
+}
+
+}  // namespace gdws
+
+using namespace gdws;
+
+extern "C" {
+
+int gdws_out_dim(int in, int k, int stride, int pad)
+{
+    if (k < 1 || stride < 1) return 0;
+    const int span = in + 2 * pad - k;
+    return span < 0 ? 0 : span / stride + 1;
+}
+
+gdws_status_t gdws_plan(int C, int D, int k, int stride, int pad, const int32_t *g, gdws_plan_t **out)
+{
+    if (!out) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: out is NULL");
+    *out = nullptr;
+    if (!g) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: g is NULL");
+    if (C < 1 || D < 1) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: C=%d, D=%d must be >= 1", C, D);
+    if (C > (1 << 20) || D > (1 << 20)) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: C or D too large");
+    if (k < 1 || k > kMaxK) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: k=%d outside 1..%d", k, kMaxK);
+    if (stride < 1 || stride > 4) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: stride=%d outside 1..4", stride);
+    if (pad < 0 || pad > k) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: pad=%d outside 0..k", pad);
+    int64_t G = 0;
+    for (int c = 0; c < C; ++c) {
+        if (g[c] < 0) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: g[%d]=%d is negative", c, g[c]);
+        if (g[c] > (1 << 16)) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: g[%d]=%d too large", c, g[c]);
+        G += g[c];
+    }
+    if (G < 1) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: sum of g is 0");
+    if (G > (1 << 24)) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan: sum of g too large");
+    gdws_plan_s *p = new (std::nothrow) gdws_plan_s;
+    if (!p) return fail(GDWS_ERR_ALLOC, "gdws_plan: out of host memory");
+    p->C = C; p->D = D; p->k = k; p->stride = stride; p->pad = pad;
+    p->G = (int)G;
+    p->Gpad = round_up((int)G, kChunk);
+    p->Dpad = round_up(D, 16);
+    p->nchunks = p->Gpad / kChunk;
+    try {
+        p->g.assign(g, g + C);
+        p->off.resize(C + 1);
+        p->chan.assign(p->Gpad, -1);
+    } catch (...) {
+        delete p;
+        return fail(GDWS_ERR_ALLOC, "gdws_plan: out of host memory");
+    }
+    int32_t acc = 0;
+    for (int c = 0; c < C; ++c) {          // Property 2: rows of channel c start at off_c
+        p->off[c] = acc;
+        for (int j = 0; j < g[c]; ++j) p->chan[acc + j] = c;
+        acc += g[c];
+    }
+    p->off[C] = acc;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
+        gdws_status_t st = ensure_device(p);
+        if (st != GDWS_OK) { delete p; return st; }
+    } else {
+        cudaGetLastError();
+    }
+    *out = p;
+    return GDWS_OK;
+}
+
+gdws_status_t gdws_plan_set_option(gdws_plan_t *p, int key, int value)
+{
+    if (!p) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan_set_option: plan is NULL");
+    switch (key) {
+    case GDWS_OPT_PATH:
+        if (value < GDWS_PATH_AUTO || value > GDWS_PATH_UNFUSED) return fail(GDWS_ERR_INVALID_ARG, "bad path %d", value);
+        p->opt_path = value; return GDWS_OK;
+    case GDWS_OPT_RELU:
+        if (value != 0 && value != 1) return fail(GDWS_ERR_INVALID_ARG, "relu must be 0 or 1");
+        p->opt_relu = value; return GDWS_OK;
+    case GDWS_OPT_TILE: {
+        if (value != 0) {
+            const int TN = (value >> 16) & 0xff, PH = (value >> 8) & 0xff, PW = value & 0xff;
+            if (!(PW == 4 || PW == 8 || PW == 16 || PW == 32) || TN < 1 || PH < 1 || TN * PH * PW > kTileRows ||
+                (PW == 4 && (PH & 1)) || (TN > 1 && (PH * PW) % 8))
+                return fail(GDWS_ERR_INVALID_ARG, "bad tile TN=%d PH=%d PW=%d", TN, PH, PW);
+        }
+        p->opt_tile = value; return GDWS_OK;
+    }
+    case GDWS_OPT_A_LAYOUT:
+        if (value != 0 && value != 1) return fail(GDWS_ERR_INVALID_ARG, "a_layout must be 0 or 1");
+        p->opt_a_layout = value; return GDWS_OK;
+    case GDWS_OPT_DW_MATH:
+        if (value != 0 && value != 1) return fail(GDWS_ERR_INVALID_ARG, "dw_math must be 0 or 1");
+        p->opt_dw_math = value; return GDWS_OK;
+    default:
+        return fail(GDWS_ERR_INVALID_ARG, "unknown option %d", key);
+    }
+}
+
+gdws_status_t gdws_plan_info(const gdws_plan_t *p, int *G, int *G_pad, int64_t *macs_per_pixel, int64_t *params)
+{
+    if (!p) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan_info: plan is NULL");
+    if (G) *G = p->G;
+    if (G_pad) *G_pad = p->Gpad;
+    const int64_t v = (int64_t)p->G * ((int64_t)p->k * p->k + p->D);   // Eq. 3 per output pixel
+    if (macs_per_pixel) *macs_per_pixel = v;
+    if (params) *params = v;
+    return GDWS_OK;
+}
+
+gdws_status_t gdws_plan_tables(const gdws_plan_t *p, int32_t *off, int32_t *chan)
+{
+    if (!p) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan_tables: plan is NULL");
+    if (off) memcpy(off, p->off.data(), sizeof(int32_t) * (p->C + 1));
+    if (chan) memcpy(chan, p->chan.data(), sizeof(int32_t) * p->Gpad);
+    return GDWS_OK;
+}
+
+gdws_status_t gdws_plan_tile(const gdws_plan_t *p, int n, int h, int w, int *TN, int *PH, int *PW, int64_t *tiles)
+{
+    if (!p) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan_tile: plan is NULL");
+    Tile t;
+    if (!choose_tile(p, n, h, w, &t))
+        return fail(GDWS_ERR_UNSUPPORTED, "no fused tile fits n=%d h=%d w=%d", n, h, w);
+    if (TN) *TN = t.TN;
+    if (PH) *PH = t.PH;
+    if (PW) *PW = t.PW;
+    if (tiles) *tiles = t.tiles();
+    return GDWS_OK;
+}
+
+size_t gdws_workspace_bytes(const gdws_plan_t *p, gdws_dtype_t dtype, int n, int h, int w)
+{
+    if (!p || n < 1) return 0;
+    const int Ho = gdws_out_dim(h, p->k, p->stride, p->pad);
+    const int Wo = gdws_out_dim(w, p->k, p->stride, p->pad);
+    if (Ho < 1 || Wo < 1) return 0;
+    const size_t px = (size_t)n * Ho * Wo;
+    if (dtype == GDWS_F32) return px * p->G * sizeof(float);
+    if (dtype == GDWS_BF16) return px * p->Gpad * sizeof(uint16_t);
+    return 0;
+}
+
+gdws_status_t gdws_set_workspace(gdws_plan_t *p, void *ws, size_t bytes)
+{
+    if (!p) return fail(GDWS_ERR_INVALID_ARG, "gdws_set_workspace: plan is NULL");
+    if (ws && ((uintptr_t)ws & 255)) return fail(GDWS_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    p->ws = ws;
+    p->ws_bytes = ws ? bytes : 0;
+    return GDWS_OK;
+}
+
+int64_t gdws_launch_count(const gdws_plan_t *p) { return p ? p->launches : 0; }
+
+const char *gdws_last_error(void) { return gdws::g_err; }
+
+const char *gdws_version(void) { return "gdws-b200 0.1.0 (sm_100a)"; }
+
+void gdws_destroy(gdws_plan_t *p)
+{
+    if (!p) return;
+    free_device(p);
+    delete p;
+}
+
+}  // extern "C"

@@ -1,0 +1,192 @@
+"""Parity of the CUDA library (through the C ABI) with the CPU reference, element by
+element on the same seeded inputs.  Bars: max|y - y_ref| / max|y_ref| <= 1e-4 on the
+fp32 path and <= 2e-2 on the bf16-in / fp32-accumulate path."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gdws_oracle as orc
+from paper_2110_14871_b200 import build as gbuild
+from paper_2110_14871_b200 import gdws
+from paper_2110_14871_b200 import inputs as gi
+
+from util import TOL, make_plan, rel_err, run_gpu, run_oracle, small_spec, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    gbuild.build_library()
+    assert torch.cuda.get_device_capability(0)[0] == 10, "these tests need an sm_100 device"
+
+
+# ------------------------------------------------------------------ fp32 path
+F32_SHAPES = [
+    # N, C, D, H, W, k, stride, pad, g_dist
+    (1, 16, 16, 32, 32, 3, 1, 1, ("uniform", 1, 3)),
+    (2, 5, 7, 9, 11, 3, 2, 1, ("uniform", 0, 9)),
+    (3, 4, 130, 7, 6, 5, 1, 2, ("uniform", 1, 25)),
+    (1, 3, 4, 6, 5, 2, 1, 0, ("uniform", 1, 4)),
+    (2, 6, 3, 5, 5, 1, 1, 0, ("const", 1)),
+    (1, 40, 20, 13, 13, 3, 1, 1, ("uniform", 1, 9)),
+]
+
+
+@pytest.mark.parametrize("layout", ["NCHW", "NHWC"])
+@pytest.mark.parametrize("path", [gdws.PATH_FUSED, gdws.PATH_UNFUSED])
+@pytest.mark.parametrize("shape", F32_SHAPES)
+def test_f32_forward_matches_reference(shape, path, layout):
+    N, C, D, H, W, k, s, p, gd = shape
+    spec = small_spec("t", N, C, D, H, W, k, s, p, gd, "f32", layout, relu=(C == 5), seed=sum(shape[:8]))
+    data = gi.make_layer(spec)
+    if data.G == 0:
+        pytest.skip("empty g")
+    y = run_gpu(data, path=path)
+    ref, _ = run_oracle(data)
+    assert rel_err(y, ref) <= TOL["f32"]
+
+
+def test_config0_exact_recipe():
+    data = gi.make_layer(gi.config_layers(0)[0])
+    ref, _ = run_oracle(data)
+    for path in (gdws.PATH_FUSED, gdws.PATH_UNFUSED):
+        assert rel_err(run_gpu(data, path=path), ref) <= TOL["f32"]
+
+
+def test_f32_stages_match_reference():
+    spec = small_spec("t", 2, 6, 10, 9, 8, 3, 2, 1, ("uniform", 1, 9), "f32", "NCHW", seed=5)
+    data = gi.make_layer(spec)
+    plan = make_plan(data)
+    x, dw, pw = to_device(data.x, "f32"), to_device(data.dw_w, "f32"), to_device(data.pw_w, "f32")
+    b = torch.from_numpy(data.bias).cuda()
+    z = torch.full((spec.N, data.G, spec.Ho, spec.Wo), float("nan"), device="cuda")
+    y = torch.full((spec.N, spec.D, spec.Ho, spec.Wo), float("nan"), device="cuda")
+    plan.depthwise(x, z, "NCHW", dw)
+    plan.pointwise(z, y, "NCHW", pw, b)
+    torch.cuda.synchronize()
+    yr, zr, _ = run_oracle(data, return_z=True)
+    assert rel_err(z.cpu().numpy(), zr) <= 1e-5
+    assert rel_err(y.cpu().numpy(), yr) <= TOL["f32"]
+    assert plan.launch_count() == 2
+    plan.destroy()
+
+
+# ------------------------------------------------------------------ bf16 path
+BF16_SHAPES = [
+    # N, C, D, H, W, k, stride, pad, g_dist   (several tiles + ragged tails in n, h and w)
+    (3, 16, 16, 8, 8, 3, 1, 1, ("uniform", 1, 9)),
+    (5, 32, 24, 9, 11, 3, 1, 1, ("uniform", 0, 9)),
+    (2, 24, 40, 20, 17, 3, 2, 1, ("uniform", 1, 9)),
+    (9, 16, 64, 4, 4, 3, 1, 1, ("uniform", 1, 9)),
+    (2, 8, 16, 14, 14, 5, 1, 2, ("uniform", 1, 25)),
+    (1, 16, 8, 12, 10, 2, 1, 0, ("uniform", 1, 4)),
+    (2, 40, 272, 7, 7, 1, 1, 0, ("uniform", 1, 1)),
+    (1, 64, 512, 9, 9, 3, 2, 1, ("heavy",)),
+    (2, 16, 32, 33, 35, 3, 1, 1, ("heavy",)),
+]
+
+
+@pytest.mark.parametrize("path,a_layout", [(gdws.PATH_UNFUSED, 0), (gdws.PATH_FUSED, 0), (gdws.PATH_FUSED, 1)])
+@pytest.mark.parametrize("shape", BF16_SHAPES)
+def test_bf16_forward_matches_reference(shape, path, a_layout):
+    N, C, D, H, W, k, s, p, gd = shape
+    spec = small_spec("t", N, C, D, H, W, k, s, p, gd, "bf16", "NHWC", relu=(C == 24), seed=sum(shape[:8]))
+    data = gi.make_layer(spec)
+    y = run_gpu(data, path=path, a_layout=a_layout)
+    ref, _ = run_oracle(data)
+    err = rel_err(y, ref)
+    assert err <= TOL["bf16"], err
+    # two bf16 roundings (z and y) should sit far inside the bar
+    assert err <= 1e-2, err
+
+
+def test_bf16_depthwise_and_pointwise_stages():
+    spec = small_spec("t", 3, 16, 24, 10, 9, 3, 1, 1, ("uniform", 1, 9), seed=9)
+    data = gi.make_layer(spec)
+    plan = make_plan(data)
+    x, dw, pw = (to_device(a, "bf16") for a in (data.x, data.dw_w, data.pw_w))
+    b = torch.from_numpy(data.bias).cuda()
+    plan.pack_weights(dw, pw, b)
+    G, Gp, _, _ = plan.info()
+    npix = spec.N * spec.Ho * spec.Wo
+    z = torch.full((npix, Gp), float("nan"), dtype=torch.bfloat16, device="cuda")
+    y = torch.full((spec.N, spec.Ho, spec.Wo, spec.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    plan.depthwise(x, z, "NHWC")
+    plan.pointwise(z, y, "NHWC")
+    torch.cuda.synchronize()
+    plan.status()
+    yr, zr, _ = run_oracle(data, return_z=True)
+    zg = z.float().cpu().numpy()
+    assert (zg[:, G:] == 0).all()                      # padding columns are zeros
+    assert rel_err(zg[:, :G].reshape(spec.N, spec.Ho, spec.Wo, G), zr) <= 2 ** -8
+    # the PW stage alone, against the reference PW applied to the GPU's own (rounded) z
+    yr2, _ = orc.pw(zg[:, :G].reshape(spec.N, spec.Ho, spec.Wo, G).astype(np.float64), data.pw_w, data.bias, layout="NHWC")
+    assert rel_err(y.float().cpu().numpy(), yr2) <= 2 ** -7
+    assert rel_err(y.float().cpu().numpy(), yr) <= TOL["bf16"]
+    plan.destroy()
+
+
+def test_bf16_prepacked_weights_and_rerun_is_bitwise_stable():
+    spec = small_spec("t", 4, 32, 32, 8, 8, seed=13)
+    data = gi.make_layer(spec)
+    a = run_gpu(data, path=gdws.PATH_FUSED, prepack=True)
+    b = run_gpu(data, path=gdws.PATH_FUSED, prepack=False)
+    c = run_gpu(data, path=gdws.PATH_FUSED, prepack=True)
+    assert np.array_equal(a, b) and np.array_equal(a, c)
+    ref, _ = run_oracle(data)
+    assert rel_err(a, ref) <= TOL["bf16"]
+
+
+def test_config1_shape_reduced_batch():
+    """Config-1 layer (C=D=256, 8x8, g~U[1,9]) at a batch the reference finishes in seconds."""
+    spec = gi.config_layers(1)[0]
+    data = gi.make_layer(spec, N=20)
+    ref, _ = run_oracle(data)
+    for path in (gdws.PATH_FUSED, gdws.PATH_UNFUSED):
+        err = rel_err(run_gpu(data, path=path), ref)
+        assert err <= TOL["bf16"], (path, err)
+
+
+def test_forward_rejects_bad_tensors():
+    data = gi.make_layer(small_spec("t", 2, 16, 16, 8, 8, seed=3))
+    plan = make_plan(data)
+    x = to_device(data.x, "bf16")
+    y = torch.empty((2, 8, 8, 16), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(gdws.GdwsError) as e:
+        plan.forward(x, y, "NHWC")                                  # no weights yet
+    assert e.value.status == gdws.ERR_INVALID_ARG
+    dw, pw = to_device(data.dw_w, "bf16"), to_device(data.pw_w, "bf16")
+    ybad = torch.empty((2, 7, 8, 16), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(gdws.GdwsError) as e:
+        plan.forward(x, ybad, "NHWC", dw, pw)
+    assert e.value.status == gdws.ERR_INVALID_ARG
+    with pytest.raises(gdws.GdwsError) as e:
+        plan.forward(x, x, "NHWC", dw, pw)                          # aliasing
+    assert e.value.status == gdws.ERR_INVALID_ARG
+    plan.set_option(gdws.OPT_PATH, gdws.PATH_UNFUSED)
+    with pytest.raises(gdws.GdwsError) as e:
+        plan.forward(x, y, "NHWC", dw, pw)                          # no workspace
+    assert e.value.status == gdws.ERR_WORKSPACE
+    before = plan.launch_count()
+    xn = torch.empty((2, 16, 8, 8), dtype=torch.bfloat16, device="cuda")
+    yn = torch.empty((2, 16, 8, 8), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(gdws.GdwsError) as e:
+        plan.forward(xn, yn, "NCHW", dw, pw)
+    assert e.value.status == gdws.ERR_UNSUPPORTED and plan.launch_count() == before
+    plan.destroy()
+
+
+def test_forward_host_matches_device_forward():
+    spec = small_spec("t", 4, 16, 16, 8, 8, seed=21)
+    data = gi.make_layer(spec)
+    plan = make_plan(data)
+    dw, pw = to_device(data.dw_w, "bf16"), to_device(data.pw_w, "bf16")
+    b = torch.from_numpy(data.bias).cuda()
+    plan.pack_weights(dw, pw, b)
+    xh = torch.from_numpy(data.x).to(torch.bfloat16).pin_memory()
+    yh = torch.empty((spec.N, spec.Ho, spec.Wo, spec.D), dtype=torch.bfloat16).pin_memory()
+    plan.forward_host(xh, yh, "NHWC")
+    ref, _ = run_oracle(data)
+    assert rel_err(yh.float().numpy(), ref) <= TOL["bf16"]
+    plan.destroy()
