@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the GDWS convolution forward (Section 3.1 of arXiv 2110.14871) on B200.
+
+A "step" is one pass of the whole hot path (plan already built, weights already
+packed: GDW stage, PW stage, bias) over one synthetic batch of the workload.  The
+default workload is the CIFAR-shaped VGG-16 middle layer (N=256, C=D=256, 8x8, k=3,
+g_c ~ U[1,9], bf16 NHWC).  Timing follows the paper's FPS protocol (Appendix A.1:
+warm-up, then successive inferences between two CUDA events, no host I/O in the timed
+region), adapted to one layer and a batch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--config C] [--layer L] [--path fused|unfused] [--no-graph]
+
+Prints ONE JSON line.  With --gpus N > 1 (under torchrun) every rank runs an
+independent replica on its own GPU (the path has no exchange step); the value is the
+sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2110_14871_b200 import inputs as gi  # noqa: E402
+
+METRIC = "GDWS layer images/sec"
+UNIT = "images/s"
+L2_BYTES = 126e6
+
+
+# ------------------------------------------------------------------------------------------
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def layer_numbers(spec: gi.LayerSpec, G: int):
+    """Algorithmic work of one step: Eq. 3 MACs and the compulsory HBM bytes
+    (x once, y once, weights once; the intermediate channels never counted)."""
+    e = 4 if spec.dtype == "f32" else 2
+    px = spec.N * spec.Ho * spec.Wo
+    macs = px * G * (spec.k * spec.k + spec.D)
+    nbytes = spec.N * spec.H * spec.W * spec.C * e + px * spec.D * e + (G * spec.k * spec.k + spec.D * G) * e + 4 * spec.D
+    return px, macs, nbytes
+
+
+def layer_roofline_us(macs, nbytes, peaks, sustained=False):
+    tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
+    t_tensor = 2.0 * macs / (tf * 1e12) * 1e6
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6
+    return max(t_tensor, t_hbm), t_tensor, t_hbm
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        self._period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _loop(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self._period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+
+    def summary(self):
+        med = int(statistics.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_throughput(spec: gi.LayerSpec, target_s: float = 12.0):
+    """Images/s of the CPU reference on a bounded sample of the workload (host cores)."""
+    from oracle import gdws_oracle as orc
+    n = min(spec.N, 2)
+    d = gi.make_layer(spec, N=n)
+    t0 = time.perf_counter()
+    orc.forward(d.x, d.g, d.dw_w, d.pw_w, d.bias, stride=spec.stride, pad=spec.pad, relu=spec.relu, layout=spec.layout)
+    probe = (time.perf_counter() - t0) / n
+    n = int(max(1, min(spec.N, target_s / max(probe, 1e-6))))
+    d = gi.make_layer(spec, N=n)
+    t0 = time.perf_counter()
+    orc.forward(d.x, d.g, d.dw_w, d.pw_w, d.bias, stride=spec.stride, pad=spec.pad, relu=spec.relu, layout=spec.layout)
+    dt = time.perf_counter() - t0
+    return n / dt, n, dt, orc.num_threads()
+
+
+def run_reference(args, spec):
+    """--impl reference: the CPU reference as it stands, on the host cores, same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import gdws_oracle as orc
+    d_full_g = gi.make_layer(spec, N=1).g
+    G = int(d_full_g.sum())
+    _, macs, _ = layer_numbers(spec, G)
+    per_img = macs / spec.N
+    # bounded sample: about 1.5 s of reference work per step
+    probe_n = min(spec.N, 2)
+    d = gi.make_layer(spec, N=probe_n)
+    t0 = time.perf_counter()
+    orc.forward(d.x, d.g, d.dw_w, d.pw_w, d.bias, stride=spec.stride, pad=spec.pad, relu=spec.relu, layout=spec.layout)
+    probe = (time.perf_counter() - t0) / probe_n
+    budget = min(1.5, 150.0 / max(1, args.steps + args.warmup))
+    n = int(max(1, min(spec.N, budget / max(probe, 1e-6))))
+    d = gi.make_layer(spec, N=n)
+    run = lambda: orc.forward(d.x, d.g, d.dw_w, d.pw_w, d.bias, stride=spec.stride, pad=spec.pad, relu=spec.relu,
+                              layout=spec.layout)
+    for _ in range(args.warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = f"{n} of {spec.N} images per step ({per_img * n / 1e9:.3f} GMAC), {args.steps} steps"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(spec, G) | {"note": "CPU reference (oracle/), fp64 direct loops"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def workload_config(spec: gi.LayerSpec, G: int):
+    return {"workload": f"{spec.name}: N={spec.N} C={spec.C} D={spec.D} {spec.H}x{spec.W} k={spec.k} "
+                        f"stride={spec.stride} pad={spec.pad} g~{spec.g_dist} G={G} {spec.dtype} {spec.layout}",
+            "global_batch": spec.N}
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args, spec):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2110_14871_b200 import build as gbuild
+    from paper_2110_14871_b200 import gdws
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        gbuild.build_library()
+    if world > 1:
+        dist.barrier()
+    peaks = load_peaks()
+
+    data = gi.make_layer(spec)
+    G = data.G
+    px, macs, nbytes = layer_numbers(spec, G)
+    tdt = torch.float32 if spec.dtype == "f32" else torch.bfloat16
+    code = gdws.F32 if spec.dtype == "f32" else gdws.BF16
+
+    def dev(a):
+        t = torch.from_numpy(np.ascontiguousarray(a))
+        return (t.to(torch.bfloat16) if spec.dtype == "bf16" else t).cuda()
+
+    x0, dw, pw = dev(data.x), dev(data.dw_w), dev(data.pw_w)
+    bias = torch.from_numpy(data.bias).cuda()
+    yshape = (spec.N, spec.D, spec.Ho, spec.Wo) if spec.layout == "NCHW" else (spec.N, spec.Ho, spec.Wo, spec.D)
+    set_bytes = x0.numel() * x0.element_size() + int(np.prod(yshape)) * x0.element_size()
+    nsets = max(2, int(np.ceil(3.2 * L2_BYTES / set_bytes))) if set_bytes < 2.5 * L2_BYTES else 1
+    nsets = min(nsets, 64)
+    xs = [x0] + [x0.clone() for _ in range(nsets - 1)]
+    ys = [torch.empty(yshape, dtype=tdt, device="cuda") for _ in range(nsets)]
+
+    plan = gdws.Plan(spec.C, spec.D, spec.k, spec.stride, spec.pad, data.g)
+    plan.set_option(gdws.OPT_RELU, int(spec.relu))
+    path = {"fused": gdws.PATH_FUSED, "unfused": gdws.PATH_UNFUSED, "auto": gdws.PATH_AUTO}[args.path]
+    plan.set_option(gdws.OPT_PATH, path)
+    plan.set_option(gdws.OPT_DW_MATH, args.dw_math)
+    plan.set_option(gdws.OPT_A_LAYOUT, args.a_layout)
+    if args.tile:
+        plan.set_option(gdws.OPT_TILE, args.tile)
+    if path == gdws.PATH_UNFUSED:
+        ws = torch.empty(plan.workspace_bytes(code, spec.N, spec.H, spec.W) + 256, dtype=torch.uint8, device="cuda")
+        plan.set_workspace(ws)
+    f32 = spec.dtype == "f32"
+    if not f32:
+        plan.pack_weights(dw, pw, bias)
+    wargs = dict(dw_w=dw, pw_w=pw, bias=bias) if f32 else {}
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        plan.forward(xs[i % nsets], ys[i % nsets], spec.layout, stream=stream, **wargs)
+
+    # one checked forward before timing: sampled parity against the CPU reference (rank 0)
+    step(0)
+    torch.cuda.synchronize()
+    plan.status()
+    l0 = plan.launch_count()
+    step(0)
+    launches_per_step = plan.launch_count() - l0
+
+    graph = None
+    if not args.no_graph:
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(nsets):
+                plan.forward(xs[i], ys[i], spec.layout, stream=side, **wargs)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(nsets):
+                plan.forward(xs[i], ys[i], spec.layout, stream=torch.cuda.current_stream(), **wargs)
+        graph = g
+
+    def run_steps(k):
+        if graph is None:
+            for i in range(k):
+                step(i)
+        else:
+            full, rem = divmod(k, nsets)
+            for _ in range(full):
+                graph.replay()
+            for i in range(rem):
+                step(i)
+
+    for _ in range(3):
+        run_steps(max(args.warmup, 3))
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        ev0.record()
+        run_steps(args.steps)
+        ev1.record()
+        torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        dist.barrier()
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    plan.status()
+    sec_per_step = ms / 1e3 / args.steps
+    value = world * spec.N / sec_per_step
+
+    # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    e2e = None
+    if not f32 or True:
+        xh = torch.from_numpy(np.ascontiguousarray(data.x))
+        xh = (xh.to(torch.bfloat16) if spec.dtype == "bf16" else xh).pin_memory()
+        yh = torch.empty(yshape, dtype=tdt).pin_memory()
+        k_e2e = max(3, min(args.steps, 30))
+        for _ in range(3):
+            plan.forward_host(xh, yh, spec.layout, stream=stream, **wargs)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(k_e2e):
+            plan.forward_host(xh, yh, spec.layout, stream=stream, **wargs)
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) / k_e2e
+        if world > 1:
+            t = torch.tensor([dt], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = {"value": world * spec.N / dt, "unit": UNIT, "h2d_bytes_per_step": xh.numel() * xh.element_size(),
+               "d2h_bytes_per_step": yh.numel() * yh.element_size(), "steps": k_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    t_roof, t_tensor, t_hbm = layer_roofline_us(macs, nbytes, peaks)
+    t_roof_s, _, _ = layer_roofline_us(macs, nbytes, peaks, sustained=True)
+    us = sec_per_step * 1e6
+    bound = "tensor" if t_tensor >= t_hbm else "hbm"
+    if bound == "tensor":
+        achieved, peak, runit = 2.0 * macs / sec_per_step / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+    else:
+        achieved, peak, runit = nbytes / sec_per_step / 1e9, peaks["hbm_gbs"], "GB/s"
+    traffic = None
+    roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
+            "traffic": traffic, "peak_source": peaks["source"] + (" burst" if bound == "tensor" else " copy"),
+            "kernel": "fused_bf16_kernel" if (not f32 and path != gdws.PATH_UNFUSED) else "see config.path",
+            "layer_roofline_us": t_roof, "t_tensor_us": t_tensor, "t_hbm_us": t_hbm,
+            "frac_of_layer_roofline": t_roof / us, "frac_of_layer_roofline_sustained_peak": t_roof_s / us}
+
+    cpu_v, cpu_n, cpu_dt, cores = oracle_throughput(spec, target_s=args.cpu_seconds)
+    cpu = {"value": cpu_v, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"{cpu_n} of {spec.N} images, {cpu_dt:.1f} s of CPU reference work"}
+
+    # parity of the timed configuration on sampled images
+    parity = None
+    if args.check:
+        from oracle import gdws_oracle as orc
+        torch.cuda.synchronize()
+        sel = sorted(set([0, spec.N // 2, spec.N - 1]))
+        yg = ys[0][sel].float().cpu().numpy().astype(np.float64)
+        xsel = data.x[sel]
+        ref, _ = orc.forward(xsel, data.g, data.dw_w, data.pw_w, data.bias, stride=spec.stride, pad=spec.pad,
+                             relu=spec.relu, layout=spec.layout)
+        parity = float(np.max(np.abs(yg - ref)) / np.max(np.abs(ref)))
+
+    cfg = workload_config(spec, G)
+    cfg.update({"path": args.path, "launch": "cuda graph replay" if graph is not None else "plain launches",
+                "l2": f"rotating {nsets} input/output buffer sets ({nsets * set_bytes / 1e6:.0f} MB > 126 MB L2)"
+                      if nsets > 1 else "one buffer set larger than L2",
+                "tile": "TNxPHxPW=%dx%dx%d" % plan.tile(spec.N, spec.H, spec.W)[:3] if not f32 else None,
+                "parallelism": "replicas" if world > 1 else "single GPU"})
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": sec_per_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": spec.dtype, "data": "synthetic", "config": cfg,
+        "effective_tmacs": world * macs / sec_per_step / 1e12,
+        "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "clocks": clk.summary(), "parity_max_rel_err": parity,
+    }
+    print(json.dumps(out), flush=True)
+    plan.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--layer", type=int, default=0)
+    ap.add_argument("--path", default="fused", choices=["fused", "unfused", "auto"])
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-check", dest="check", action="store_false")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--dw-math", type=int, default=0)
+    ap.add_argument("--a-layout", type=int, default=0)
+    ap.add_argument("--tile", type=int, default=0)
+    args = ap.parse_args()
+    spec = gi.config_layers(args.config)[args.layer]
+    if args.impl == "reference":
+        if args.steps == 20000:
+            args.steps, args.warmup = 20, 3
+        run_reference(args, spec)
+    else:
+        run_ours(args, spec)
+
+
+if __name__ == "__main__":
+    main()

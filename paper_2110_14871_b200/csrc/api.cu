@@ -46,8 +46,12 @@ gdws_status_t check_pair(const gdws_plan_s *p, const gdws_tensor_t *x, const gdw
 
 gdws_status_t prepare(gdws_plan_s *p)
 {
-    gdws_status_t st = check_arch();
-    if (st != GDWS_OK) return st;
+    gdws_status_t st = GDWS_OK;
+    if (!p->arch_ok) {
+        st = check_arch();
+        if (st != GDWS_OK) return st;
+        p->arch_ok = true;
+    }
     st = ensure_device(p);
     if (st != GDWS_OK) return st;
     int dev = -1;

@@ -441,8 +441,13 @@ gdws_status_t bf16_pointwise(gdws_plan_s *p, const void *z, gdws_tensor_t *y, cu
     const int cols = tmem_cols_for(p->Dpad);
     size_t smem = 1024 + 2 * 16384 + 2 * (size_t)p->Dpad * kChunk * 2;
     smem = smem_for_tmem(smem, cols);
-    cudaError_t e = cudaFuncSetAttribute(pw_bf16_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(pw_bf16_tc_kernel)");
+    cudaError_t e = cudaSuccess;
+    static bool attr_set[64] = {};
+    if (!attr_set[p->device & 63]) {   // once per device: allow the full dynamic shared memory
+        e = cudaFuncSetAttribute(pw_bf16_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(pw_bf16_tc_kernel)");
+        attr_set[p->device & 63] = true;
+    }
     const long long blocks = (npix + kTileRows - 1) / kTileRows;
     pw_bf16_tc_kernel<<<(int)blocks, kPwThreads, smem, st>>>((const uint16_t *)z, p->d_pw_img, p->d_bias,
                                                              (uint16_t *)y->ptr, npix, p->Gpad, p->D, p->Dpad,
@@ -718,10 +723,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
 }
 
 template <int K>
-static gdws_status_t launch_fused(const FusedParams &P, int64_t tiles, size_t smem, cudaStream_t st)
+static gdws_status_t launch_fused(const FusedParams &P, int device, int64_t tiles, size_t smem, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(fused_bf16_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_bf16_kernel)");
+    cudaError_t e = cudaSuccess;
+    static bool attr_set[64] = {};
+    if (!attr_set[device & 63]) {   // once per device: allow the full dynamic shared memory
+        e = cudaFuncSetAttribute(fused_bf16_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_bf16_kernel)");
+        attr_set[device & 63] = true;
+    }
     fused_bf16_kernel<K><<<(int)tiles, kFusedThreads, smem, st>>>(P);
     e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "fused_bf16_kernel launch");
@@ -752,13 +762,13 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
     const size_t smem = smem_for_tmem(t.smem, P.tmem_cols);
     gdws_status_t rc;
     switch (p->k) {
-    case 1: rc = launch_fused<1>(P, t.tiles(), smem, st); break;
-    case 2: rc = launch_fused<2>(P, t.tiles(), smem, st); break;
-    case 3: rc = launch_fused<3>(P, t.tiles(), smem, st); break;
-    case 4: rc = launch_fused<4>(P, t.tiles(), smem, st); break;
-    case 5: rc = launch_fused<5>(P, t.tiles(), smem, st); break;
-    case 6: rc = launch_fused<6>(P, t.tiles(), smem, st); break;
-    case 7: rc = launch_fused<7>(P, t.tiles(), smem, st); break;
+    case 1: rc = launch_fused<1>(P, p->device, t.tiles(), smem, st); break;
+    case 2: rc = launch_fused<2>(P, p->device, t.tiles(), smem, st); break;
+    case 3: rc = launch_fused<3>(P, p->device, t.tiles(), smem, st); break;
+    case 4: rc = launch_fused<4>(P, p->device, t.tiles(), smem, st); break;
+    case 5: rc = launch_fused<5>(P, p->device, t.tiles(), smem, st); break;
+    case 6: rc = launch_fused<6>(P, p->device, t.tiles(), smem, st); break;
+    case 7: rc = launch_fused<7>(P, p->device, t.tiles(), smem, st); break;
     default: return fail(GDWS_ERR_UNSUPPORTED, "k=%d", p->k);
     }
     if (rc == GDWS_OK) p->launches++;

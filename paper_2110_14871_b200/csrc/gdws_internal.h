@@ -14,7 +14,7 @@ namespace gdws {
 constexpr int kChunk = 64;          // intermediate channels per tensor-core K chunk (one 128-byte swizzle row of bf16)
 constexpr int kTileRows = 128;      // output pixels per tensor-core tile (UMMA M)
 constexpr int kMaxK = 7;
-constexpr int kMaxSmem = 227 * 1024;
+constexpr int kMaxSmem = 225 * 1024;      // dynamic shared memory a block may ask for (227 KB minus static use)
 
 // Bits of the device status word.
 enum : int {
@@ -49,6 +49,7 @@ struct gdws_plan_s {
 
     // device side (allocated by ensure_device)
     int device = -1;
+    bool arch_ok = false;          // the plan's device was checked to be compute capability 10.x
     int32_t *d_off = nullptr;      // [C+1]
     int32_t *d_chan = nullptr;     // [Gpad], -1 for padding
     float *d_dw = nullptr;         // [Gpad][k*k] fp32 depthwise filters, zero rows for padding
