@@ -1,0 +1,500 @@
+// Fused GDWS forward for bf16 NHWC tensors on sm_100a: the G intermediate channels of the GDW
+// stage go from the ALUs to the tensor cores through shared memory and never reach HBM.
+//
+// One block computes one tile of 128 output pixels (TN images x PH x PW patch) for all D output
+// channels.  The intermediate channels are processed in K chunks of 64 (i = 64q .. 64q+63, in the
+// canonical order i = off_c + j), and three kinds of warps run as a pipeline over the chunks:
+//   * 4 staging warps: chunk q reads the contiguous channel range [c0(q), c0(q)+span); a warp
+//     loads those channels of the tile's input patch (with halo, zero filled outside the image)
+//     with 16-byte loads and writes them channel-major into one of `nslots` slots, so that the
+//     depthwise stage reads runs of consecutive pixels of one channel with 16-byte loads;
+//   * 8 depthwise warps: thread t owns intermediate channel 64q + (t & 63) and a quarter of the
+//     tile's pixels; it keeps its k x k filter in registers, slides down the patch reusing each
+//     input row for up to k output rows, and writes bf16 results as 16-byte pieces into a
+//     pixel-contiguous (MN-major), 128-byte-swizzled tensor-core operand stage;
+//   * 1 control warp: one lane streams the pre-swizzled pointwise-weight chunk (bulk copy with
+//     mbarrier completion) and issues tcgen05.mma into the TMEM accumulator (128 lanes x D
+//     fp32 columns), committing to mbarriers that free the stages.
+// The depthwise warps finally read the accumulator back (tcgen05.ld), add the bias, apply the
+// optional ReLU, round to bf16 and store y.
+#include "sm100.cuh"
+
+namespace gdws {
+
+struct FusedParams {
+    const uint16_t *x;
+    uint16_t *y;
+    const float *dw;
+    const uint32_t *dw2;
+    const uint16_t *pw_img;
+    const float *bias;
+    const int32_t *chan;
+    const int32_t *chunk_c0;
+    int *status;
+    int N, H, W, C, Ho, Wo, D, Dpad, G, nchunks, stride, pad, relu;
+    int TN, PH, PW, tiles_h, tiles_w;
+    int IH, IW, IWp, plane, span, nslots, nsb;
+    int tmem_cols, a_kmajor, dw_math;
+};
+
+constexpr int kDwWarps = 8, kStageWarps = 4;
+constexpr int kDwThreads = kDwWarps * 32;
+constexpr int kStageThreads = kStageWarps * 32;
+constexpr int kFusedThreads = kDwThreads + kStageThreads + 32;
+constexpr int kMaxSlots = 6, kMaxBStages = 4;
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint16_t lds16(uint32_t addr)
+{
+    uint16_t v;
+    asm volatile("ld.shared.b16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Where the 8 bf16 results of pixel group `o` (rows 8o..8o+7 of the tile) and intermediate
+// channel column kk go in a pixel-contiguous (MN-major) stage: K group kk/8 and 64-row block
+// o/8 select a 1024-byte atom, kk%8 the 128-byte row, and the 16-byte piece is swizzled.
+__device__ __forceinline__ uint32_t a_off_mn(int o, int kk)
+{
+    return (uint32_t)(((kk >> 3) * 2 + (o >> 3)) * 1024 + (kk & 7) * 128 + (((o & 7) ^ (kk & 7)) << 4));
+}
+// Channel-contiguous (K-major) stage: byte offset of element (row r, column kk).
+__device__ __forceinline__ uint32_t a_off_k(int r, int kk)
+{
+    return (uint32_t)(r * 128 + (((kk >> 3) ^ (r & 7)) << 4) + (kk & 7) * 2);
+}
+__device__ __forceinline__ void store_group(const FusedParams &P, uint32_t a_stage, int o, int kk, const float (&v)[8])
+{
+    if (!P.a_kmajor) {
+        uint4 q;
+        q.x = pack_bf16x2(v[0], v[1]); q.y = pack_bf16x2(v[2], v[3]);
+        q.z = pack_bf16x2(v[4], v[5]); q.w = pack_bf16x2(v[6], v[7]);
+        sts128(a_stage + a_off_mn(o, kk), q);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sts16(a_stage + a_off_k(o * 8 + e, kk), float_to_bf16_bits(v[e]));
+    }
+}
+
+// ---- depthwise, k = 3, patches at least 8 wide: a thread computes 4 consecutive output rows of one
+// 8-pixel column group, reading each input row once (16-byte loads) and using it for up to 3 rows.
+template <int S>
+__device__ __forceinline__ void dw_rows_k3(const FusedParams &P, uint32_t xs, int cl, const float (&w)[9], int kk,
+                                           int run, bool live_i, uint32_t a_stage)
+{
+    const int nseg = P.PW >> 3;
+    const int seg = run % nseg;
+    const int R0 = (run / nseg) * 4;               // first of the 4 rows (row index = tn*PH + ph)
+    const int o0 = R0 * nseg + seg;
+    float acc[4][8];
+#pragma unroll
+    for (int ro = 0; ro < 4; ++ro)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[ro][e] = 0.f;
+    if (live_i && R0 < P.TN * P.PH) {
+        const int tn = R0 / P.PH, ph0 = R0 - tn * P.PH;
+        const uint32_t rowb = (uint32_t)P.IWp * 2;
+        const uint32_t base = xs + (uint32_t)(cl * P.plane + (tn * P.IH + ph0 * S) * P.IWp + seg * 8 * S) * 2;
+        constexpr int NR = 3 * S + 3;              // input rows feeding 4 output rows
+        constexpr int NX = 7 * S + 3;              // input columns feeding 8 output columns
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+            float xr[NX + 1];
+            const uint4 a = lds128(base + r * rowb);
+            xr[0] = bf_lo(a.x); xr[1] = bf_hi(a.x); xr[2] = bf_lo(a.y); xr[3] = bf_hi(a.y);
+            xr[4] = bf_lo(a.z); xr[5] = bf_hi(a.z); xr[6] = bf_lo(a.w); xr[7] = bf_hi(a.w);
+            if (S == 1) {
+                const uint32_t b = lds32(base + r * rowb + 16);
+                xr[8] = bf_lo(b); xr[9] = bf_hi(b);
+            } else {
+                const uint4 b = lds128(base + r * rowb + 16);
+                const uint32_t c = lds32(base + r * rowb + 32);
+                xr[8] = bf_lo(b.x); xr[9] = bf_hi(b.x); xr[10] = bf_lo(b.y); xr[11] = bf_hi(b.y);
+                xr[12] = bf_lo(b.z); xr[13] = bf_hi(b.z); xr[14] = bf_lo(b.w); xr[15] = bf_hi(b.w);
+                xr[16] = bf_lo(c);
+            }
+#pragma unroll
+            for (int ro = 0; ro < 4; ++ro) {
+                const int u = r - ro * S;
+                if (u >= 0 && u < 3) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+#pragma unroll
+                        for (int v = 0; v < 3; ++v) acc[ro][e] = fmaf(w[u * 3 + v], xr[e * S + v], acc[ro][e]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int ro = 0; ro < 4; ++ro) store_group(P, a_stage, o0 + ro * nseg, kk, acc[ro]);
+}
+
+// ---- depthwise, k = 3, 4-wide patches: a pixel group is 2 output rows x 4 columns of one image.
+template <int S>
+__device__ __forceinline__ void dw_quads_k3(const FusedParams &P, uint32_t xs, int cl, const float (&w)[9], int kk,
+                                            int run, bool live_i, uint32_t a_stage)
+{
+    const int gpi = P.PH >> 1;                      // pixel groups per image
+#pragma unroll 1
+    for (int m = 0; m < 4; ++m) {
+        const int o = run * 4 + m;
+        float acc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+        const int tn = o / gpi, ph0 = (o - tn * gpi) * 2;
+        if (live_i && tn < P.TN) {
+            const uint32_t rowb = (uint32_t)P.IWp * 2;
+            const uint32_t base = xs + (uint32_t)(cl * P.plane + (tn * P.IH + ph0 * S) * P.IWp) * 2;
+            constexpr int NR = S + 3;               // input rows feeding 2 output rows
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+                float xr[10];
+                const uint4 a = lds128(base + r * rowb);
+                xr[0] = bf_lo(a.x); xr[1] = bf_hi(a.x); xr[2] = bf_lo(a.y); xr[3] = bf_hi(a.y);
+                xr[4] = bf_lo(a.z); xr[5] = bf_hi(a.z); xr[6] = bf_lo(a.w); xr[7] = bf_hi(a.w);
+                if (S == 2) {
+                    const uint32_t b = lds32(base + r * rowb + 16);
+                    xr[8] = bf_lo(b); xr[9] = bf_hi(b);
+                }
+#pragma unroll
+                for (int ro = 0; ro < 2; ++ro) {
+                    const int u = r - ro * S;
+                    if (u >= 0 && u < 3) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+#pragma unroll
+                            for (int v = 0; v < 3; ++v)
+                                acc[ro * 4 + e] = fmaf(w[u * 3 + v], xr[e * S + v], acc[ro * 4 + e]);
+                    }
+                }
+            }
+        }
+        store_group(P, a_stage, o, kk, acc);
+    }
+}
+
+// ---- depthwise, any k and stride: one pixel group at a time, 2-byte loads.
+template <int K>
+__device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, int cl, const float *__restrict__ wp, int kk,
+                                           int run, bool live_i, uint32_t a_stage)
+{
+    const int hw = P.PH * P.PW;
+#pragma unroll 1
+    for (int m = 0; m < 4; ++m) {
+        const int o = run * 4 + m;
+        float out[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) out[e] = 0.f;
+        const int r0 = o * 8;
+        const int tn = r0 / hw;
+        if (live_i && tn < P.TN) {
+            const int rem = r0 - tn * hw;
+            const int ph = rem / P.PW, pw0 = rem - ph * P.PW;
+            const uint32_t xc = xs + (uint32_t)(cl * P.plane + tn * P.IH * P.IWp) * 2;
+#pragma unroll 1
+            for (int e = 0; e < 8; ++e) {
+                const int phe = (P.PW >= 8) ? ph : ph + (e >> 2);
+                const int pwe = (P.PW >= 8) ? pw0 + e : (e & 3);
+                const uint32_t xp = xc + (uint32_t)(phe * P.stride * P.IWp + pwe * P.stride) * 2;
+                float acc = 0.f;
+#pragma unroll
+                for (int u = 0; u < K; ++u)
+#pragma unroll
+                    for (int v = 0; v < K; ++v)
+                        acc = fmaf(__ldg(wp + u * K + v), bf16_bits_to_float(lds16(xp + (uint32_t)(u * P.IWp + v) * 2)), acc);
+                out[e] = acc;
+            }
+        }
+        store_group(P, a_stage, o, kk, out);
+    }
+}
+
+// MODE: 0 generic, 1 row runs (k=3), 2 4-wide patches (k=3); S = stride for modes 1/2.
+template <int K, int MODE, int S>
+__global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __grid_constant__ FusedParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    // a_full[2] | mma_done[2] | b_full[4] | b_free[4] | x_full[6] | x_free[6]
+    __shared__ __align__(8) uint64_t bars[2 + 2 + kMaxBStages * 2 + kMaxSlots * 2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t a_s = smem_u32(base);
+    const uint32_t b_bytes = (uint32_t)P.Dpad * kChunk * 2;
+    const uint32_t b_s = a_s + 2 * 16384;
+    const uint32_t x_s = b_s + (uint32_t)P.nsb * b_bytes;
+    const uint32_t slot_bytes = (uint32_t)P.span * P.plane * 2;
+    const uint32_t bar_afull = smem_u32(&bars[0]), bar_done = smem_u32(&bars[2]);
+    const uint32_t bar_bfull = smem_u32(&bars[4]), bar_bfree = smem_u32(&bars[4 + kMaxBStages]);
+    const uint32_t bar_xfull = smem_u32(&bars[4 + 2 * kMaxBStages]);
+    const uint32_t bar_xfree = smem_u32(&bars[4 + 2 * kMaxBStages + kMaxSlots]);
+    constexpr int kCtrlWarp = kDwWarps + kStageWarps;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_afull + 8 * i, kDwThreads); mbar_init(bar_done + 8 * i, 1); }
+        for (int i = 0; i < kMaxBStages; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
+        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(bar_xfull + 8 * i, 32); mbar_init(bar_xfree + 8 * i, kDwThreads); }
+        fence_mbar_init();
+    }
+    if (warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)P.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+
+    // tile -> first image / output row / output column
+    int tile = blockIdx.x;
+    const int bw = tile % P.tiles_w;
+    tile /= P.tiles_w;
+    const int bh = tile % P.tiles_h;
+    const int bn = tile / P.tiles_h;
+    const int n0 = bn * P.TN, ho0 = bh * P.PH, wo0 = bw * P.PW;
+
+    // Pixel table of the tile's input patch: for every pair of horizontally adjacent patch
+    // positions the linear pixel index (n*H + hi)*W + wi in x, or -1 where the patch leaves the image.
+    int2 *pix_tab = reinterpret_cast<int2 *>(base + (x_s - a_s) + (size_t)P.nslots * slot_bytes);
+    {
+        const int hi0 = ho0 * P.stride - P.pad, wi0 = wo0 * P.stride - P.pad;
+        const int npix = P.TN * P.IH * P.IWp;
+        for (int t = tid; t < npix; t += kFusedThreads) {
+            const int iw = t % P.IWp;
+            const int r = t / P.IWp;
+            const int ih = r % P.IH, tn = r / P.IH;
+            const int n = n0 + tn, hi = hi0 + ih, wi = wi0 + iw;
+            const bool in = n < P.N && hi >= 0 && hi < P.H && wi >= 0 && wi < P.W && iw < P.IW;
+            reinterpret_cast<int *>(pix_tab)[t] = in ? (n * P.H + hi) * P.W + wi : -1;
+        }
+    }
+    __syncthreads();
+
+    if (warp == kCtrlWarp) {
+        // ---------------- control warp: weight copies and MMA issue (one lane) ----------------
+        if (lane == 0) {
+            const int pre = P.nchunks < P.nsb ? P.nchunks : P.nsb;
+            for (int q = 0; q < pre; ++q) {
+                mbar_expect_tx(bar_bfull + 8 * q, b_bytes);
+                bulk_g2s(b_s + q * b_bytes, P.pw_img + (size_t)q * P.Dpad * kChunk, b_bytes, bar_bfull + 8 * q);
+            }
+            for (int q = 0; q < P.nchunks; ++q) {
+                const int sa = q & 1, sb = q % P.nsb;
+                mbar_wait(bar_bfull + 8 * sb, (q / P.nsb) & 1, &abort_flag, P.status, kStatusWaitOperand);
+                mbar_wait(bar_afull + 8 * sa, (q >> 1) & 1, &abort_flag, P.status, kStatusWaitOperand);
+                tc_fence_after();
+                issue_chunk(tmem, a_s + sa * 16384, b_s + sb * b_bytes, P.Dpad, !P.a_kmajor, q == 0);
+                umma_commit(bar_done + 8 * sa);
+                umma_commit(bar_bfree + 8 * sb);
+                // refill the weight stage of the previous chunk once its MMAs have finished
+                const int qn = q - 1 + P.nsb;
+                if (q >= 1 && qn < P.nchunks) {
+                    const int sp = (q - 1) % P.nsb;
+                    mbar_wait(bar_bfree + 8 * sp, ((q - 1) / P.nsb) & 1, &abort_flag, P.status, kStatusWaitStage);
+                    mbar_expect_tx(bar_bfull + 8 * sp, b_bytes);
+                    bulk_g2s(b_s + sp * b_bytes, P.pw_img + (size_t)qn * P.Dpad * kChunk, b_bytes, bar_bfull + 8 * sp);
+                }
+            }
+            // every copy issued was awaited above; await the last commits so that nothing is
+            // still arriving on this block's barriers when it exits
+            for (int q = (P.nchunks > P.nsb ? P.nchunks - P.nsb : 0); q < P.nchunks; ++q)
+                mbar_wait_drain(bar_bfree + 8 * (q % P.nsb), (q / P.nsb) & 1);
+        }
+    } else if (warp >= kDwWarps) {
+        // ---------------- staging warps: slot s is always filled by warp s % 4 ----------------
+        const int sw = warp - kDwWarps;
+        const int npair = (P.TN * P.IH * P.IWp) >> 1;
+        for (int q = 0; q < P.nchunks; ++q) {
+            const int slot = q % P.nslots;
+            if ((slot & (kStageWarps - 1)) != sw) continue;
+            const int use = q / P.nslots;
+            if (use >= 1) mbar_wait(bar_xfree + 8 * slot, (use - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+            const int c0 = __ldg(P.chunk_c0 + q);
+            const int ilast = min(P.G, (q + 1) * kChunk) - 1;
+            const int c1 = q * kChunk < P.G ? __ldg(P.chan + ilast) : c0;       // last channel of the chunk
+            const int gr0 = c0 >> 3, ngr = (c1 >> 3) - gr0 + 1;
+            const uint32_t xs = x_s + slot * slot_bytes;
+            for (int gr = 0; gr < ngr; ++gr) {
+                const int cb = (gr0 + gr) * 8 - c0;           // slot channel of the group's first channel
+                const uint16_t *xg = P.x + (gr0 + gr) * 8;
+                const bool whole = cb >= 0 && cb + 8 <= P.span;
+                constexpr int kBatch = 4;                     // pixel pairs per lane in flight
+                for (int p0 = lane; p0 < npair; p0 += 32 * kBatch) {
+                    uint4 va[kBatch], vb[kBatch];
+#pragma unroll
+                    for (int m = 0; m < kBatch; ++m) {
+                        const int pp = p0 + m * 32;
+                        va[m] = make_uint4(0, 0, 0, 0);
+                        vb[m] = make_uint4(0, 0, 0, 0);
+                        if (pp < npair) {
+                            const int2 o = pix_tab[pp];
+                            if (o.x >= 0) va[m] = __ldg(reinterpret_cast<const uint4 *>(xg + (size_t)o.x * P.C));
+                            if (o.y >= 0) vb[m] = __ldg(reinterpret_cast<const uint4 *>(xg + (size_t)o.y * P.C));
+                        }
+                    }
+#pragma unroll
+                    for (int m = 0; m < kBatch; ++m) {
+                        const int pp = p0 + m * 32;
+                        if (pp < npair) {
+                            const uint32_t a4[4] = {va[m].x, va[m].y, va[m].z, va[m].w};
+                            const uint32_t b4[4] = {vb[m].x, vb[m].y, vb[m].z, vb[m].w};
+                            const uint32_t dst = xs + (uint32_t)(cb * P.plane + 2 * pp) * 2;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                // channel cb+e of the two pixels -> one 32-bit store
+                                const uint32_t word = (e & 1) ? __byte_perm(a4[e >> 1], b4[e >> 1], 0x7632)
+                                                              : __byte_perm(a4[e >> 1], b4[e >> 1], 0x5410);
+                                if (whole || (cb + e >= 0 && cb + e < P.span))
+                                    sts32(dst + (uint32_t)(e * P.plane * 2), word);
+                            }
+                        }
+                    }
+                }
+            }
+            mbar_arrive(bar_xfull + 8 * slot);
+        }
+    } else {
+        // ---------------- depthwise warps ----------------
+        const int il = tid & 63, run = tid >> 6;
+        float w[9];
+        int cl = 0;
+        auto load_weights = [&](int q) {
+            const int i = q * kChunk + il;
+            if (MODE != 0) {
+#pragma unroll
+                for (int t = 0; t < 9; ++t) w[t] = __ldg(P.dw + (size_t)i * 9 + t);
+            }
+            const int c = __ldg(P.chan + i);
+            cl = c < 0 ? 0 : c - __ldg(P.chunk_c0 + q);
+        };
+        load_weights(0);
+        for (int q = 0; q < P.nchunks; ++q) {
+            const int sa = q & 1, slot = q % P.nslots;
+            const int i = q * kChunk + il;
+            const bool live_i = i < P.G;
+            float wq[9];
+#pragma unroll
+            for (int t = 0; t < 9; ++t) wq[t] = w[t];
+            const int clq = cl;
+            if (q + 1 < P.nchunks) load_weights(q + 1);     // next chunk's filter while this one computes
+            mbar_wait(bar_xfull + 8 * slot, (q / P.nslots) & 1, &abort_flag, P.status, kStatusWaitOperand);
+            if (q >= 2) mbar_wait(bar_done + 8 * sa, ((q >> 1) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+            const uint32_t xs = x_s + slot * slot_bytes;
+            const uint32_t a_stage = a_s + sa * 16384;
+            if (MODE == 1) dw_rows_k3<S>(P, xs, clq, wq, il, run, live_i, a_stage);
+            else if (MODE == 2) dw_quads_k3<S>(P, xs, clq, wq, il, run, live_i, a_stage);
+            else dw_generic<K>(P, xs, clq, P.dw + (size_t)i * (K * K), il, run, live_i, a_stage);
+            fence_proxy_async();
+            mbar_arrive(bar_afull + 8 * sa);
+            mbar_arrive(bar_xfree + 8 * slot);
+        }
+
+        // ---------------- epilogue: TMEM -> registers -> bias / ReLU -> bf16 -> global ----------------
+        {
+            const int ql = P.nchunks - 1;
+            mbar_wait(bar_done + 8 * (ql & 1), (ql >> 1) & 1, &abort_flag, P.status, kStatusWaitMma);
+            if (P.nchunks >= 2) {
+                const int qo = P.nchunks - 2;
+                mbar_wait(bar_done + 8 * (qo & 1), (qo >> 1) & 1, &abort_flag, P.status, kStatusWaitMma);
+            }
+        }
+        tc_fence_after();
+        const int lg = warp & 3, half = warp >> 2;
+        const int r = lg * 32 + lane;
+        const int hw = P.PH * P.PW;
+        const int tn = r / hw;
+        const int rem = r - tn * hw;
+        const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
+        const int n = n0 + tn, ho = ho0 + ph, wo = wo0 + pw_;
+        const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
+        uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D;
+        for (int d0 = half * 16; d0 < P.Dpad; d0 += 32) {
+            uint32_t acc[16];
+            tmem_ld16(tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)d0, acc);
+            tmem_ld_wait();
+            if (live) store_row16(acc, P.bias, d0, P.D, P.relu, yrow);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    __syncwarp();
+    if (warp == kCtrlWarp) tmem_dealloc(tmem, (uint32_t)P.tmem_cols);
+}
+
+template <int K, int MODE, int S>
+static gdws_status_t launch_fused(const FusedParams &P, int device, int64_t tiles, size_t smem, cudaStream_t st)
+{
+    cudaError_t e = cudaSuccess;
+    static bool attr_set[64] = {};
+    if (!attr_set[device & 63]) {   // once per device: allow the full dynamic shared memory
+        e = cudaFuncSetAttribute(fused_bf16_kernel<K, MODE, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_bf16_kernel)");
+        attr_set[device & 63] = true;
+    }
+    fused_bf16_kernel<K, MODE, S><<<(int)tiles, kFusedThreads, smem, st>>>(P);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "fused_bf16_kernel launch");
+}
+
+gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t st)
+{
+    if (p->Dpad > 512) return fail(GDWS_ERR_UNSUPPORTED, "bf16 fused kernel supports D <= 512 (got %d)", p->D);
+    if (p->D % 8 || p->C % 8)
+        return fail(GDWS_ERR_UNSUPPORTED, "bf16 kernels need C %% 8 == 0 and D %% 8 == 0 (got C=%d, D=%d)", p->C, p->D);
+    Tile t;
+    if (!choose_tile(p, x->n, x->h, x->w, &t))
+        return fail(GDWS_ERR_UNSUPPORTED, "no fused tile fits this shape in shared memory");
+    if (t.tiles() > 0x7fffffffLL) return fail(GDWS_ERR_UNSUPPORTED, "too many tiles");
+    if ((long long)x->n * x->h * x->w > 0x7fffffffLL) return fail(GDWS_ERR_UNSUPPORTED, "more than 2^31 input pixels");
+    FusedParams P;
+    P.x = (const uint16_t *)x->ptr; P.y = (uint16_t *)y->ptr;
+    P.dw = p->d_dw; P.dw2 = p->d_dw2; P.pw_img = p->d_pw_img; P.bias = p->d_bias;
+    P.chan = p->d_chan; P.chunk_c0 = p->d_chunk_c0; P.status = p->d_status;
+    P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = y->h; P.Wo = y->w; P.D = p->D; P.Dpad = p->Dpad;
+    P.G = p->G; P.nchunks = p->nchunks; P.stride = p->stride; P.pad = p->pad;
+    P.relu = p->opt_relu;
+    P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w;
+    P.IH = t.IH; P.IW = t.IW; P.IWp = t.IWp; P.plane = t.plane; P.span = t.span; P.nslots = t.nslots; P.nsb = t.nsb;
+    P.tmem_cols = tmem_cols_for(p->Dpad);
+    P.a_kmajor = p->opt_a_layout;
+    P.dw_math = p->opt_dw_math;
+    const size_t smem = smem_for_tmem(t.smem, P.tmem_cols);
+    const int64_t tiles = t.tiles();
+    gdws_status_t rc;
+    if (t.fast == 1 && p->stride == 1) rc = launch_fused<3, 1, 1>(P, p->device, tiles, smem, st);
+    else if (t.fast == 1 && p->stride == 2) rc = launch_fused<3, 1, 2>(P, p->device, tiles, smem, st);
+    else if (t.fast == 2 && p->stride == 1) rc = launch_fused<3, 2, 1>(P, p->device, tiles, smem, st);
+    else if (t.fast == 2 && p->stride == 2) rc = launch_fused<3, 2, 2>(P, p->device, tiles, smem, st);
+    else {
+        switch (p->k) {
+        case 1: rc = launch_fused<1, 0, 1>(P, p->device, tiles, smem, st); break;
+        case 2: rc = launch_fused<2, 0, 1>(P, p->device, tiles, smem, st); break;
+        case 3: rc = launch_fused<3, 0, 1>(P, p->device, tiles, smem, st); break;
+        case 4: rc = launch_fused<4, 0, 1>(P, p->device, tiles, smem, st); break;
+        case 5: rc = launch_fused<5, 0, 1>(P, p->device, tiles, smem, st); break;
+        case 6: rc = launch_fused<6, 0, 1>(P, p->device, tiles, smem, st); break;
+        case 7: rc = launch_fused<7, 0, 1>(P, p->device, tiles, smem, st); break;
+        default: return fail(GDWS_ERR_UNSUPPORTED, "k=%d", p->k);
+        }
+    }
+    if (rc == GDWS_OK) p->launches++;
+    return rc;
+}
+
+}  // namespace gdws

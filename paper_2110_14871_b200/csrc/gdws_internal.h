@@ -28,8 +28,10 @@ struct Tile {
     int tiles_n = 0, tiles_h = 0, tiles_w = 0;
     int IH = 0, IW = 0, IWp = 0;     // input patch rows / columns / row pitch (elements) per image
     int plane = 0;                   // elements between consecutive channels in the staged input
-    int CB = 0;                      // channels per staged block
+    int span = 0;                    // channels per staged slot (widest channel range of a K chunk)
+    int nslots = 0;                  // staged-input slots
     int nsb = 0;                     // pointwise-weight stages
+    int fast = 0;                    // 1: row-run depthwise path, 2: 4-wide-patch path, 0: generic
     size_t smem = 0;                 // dynamic shared memory of the fused kernel
     int64_t tiles() const { return (int64_t)tiles_n * tiles_h * tiles_w; }
 };
@@ -40,6 +42,8 @@ struct gdws_plan_s {
     int C = 0, D = 0, k = 0, stride = 0, pad = 0;
     int G = 0, Gpad = 0, Dpad = 0, nchunks = 0;
     std::vector<int32_t> g, off, chan;
+    std::vector<int32_t> chunk_c0;   // first input channel read by K chunk q (intermediate channels 64q..64q+63)
+    int span_max = 0;                // widest channel range of one K chunk
 
     int opt_path = GDWS_PATH_AUTO;
     int opt_relu = 0;
@@ -52,6 +56,7 @@ struct gdws_plan_s {
     bool arch_ok = false;          // the plan's device was checked to be compute capability 10.x
     int32_t *d_off = nullptr;      // [C+1]
     int32_t *d_chan = nullptr;     // [Gpad], -1 for padding
+    int32_t *d_chunk_c0 = nullptr; // [nchunks]
     float *d_dw = nullptr;         // [Gpad][k*k] fp32 depthwise filters, zero rows for padding
     uint32_t *d_dw2 = nullptr;     // [Gpad][k*k] the same filters as bf16 pairs (w,w)
     uint16_t *d_pw_img = nullptr;  // [nchunks][Dpad*64] bf16, 128-byte-swizzled K-major operand images

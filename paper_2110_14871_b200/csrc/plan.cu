@@ -57,6 +57,7 @@ static void free_device(gdws_plan_s *p)
     cudaDeviceSynchronize();
     cudaFree(p->d_off);
     cudaFree(p->d_chan);
+    cudaFree(p->d_chunk_c0);
     cudaFree(p->d_dw);
     cudaFree(p->d_dw2);
     cudaFree(p->d_pw_img);
@@ -88,6 +89,7 @@ gdws_status_t ensure_device(gdws_plan_s *p)
     } while (0)
     GDWS_TRY_ALLOC(p->d_off, sizeof(int32_t) * (p->C + 1));
     GDWS_TRY_ALLOC(p->d_chan, sizeof(int32_t) * p->Gpad);
+    GDWS_TRY_ALLOC(p->d_chunk_c0, sizeof(int32_t) * p->nchunks);
     GDWS_TRY_ALLOC(p->d_dw, sizeof(float) * p->Gpad * k2);
     GDWS_TRY_ALLOC(p->d_dw2, sizeof(uint32_t) * p->Gpad * k2);
     GDWS_TRY_ALLOC(p->d_pw_img, img);
@@ -97,6 +99,8 @@ gdws_status_t ensure_device(gdws_plan_s *p)
     p->device = dev;
     e = cudaMemcpy(p->d_off, p->off.data(), sizeof(int32_t) * (p->C + 1), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_chan, p->chan.data(), sizeof(int32_t) * p->Gpad, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(p->d_chunk_c0, p->chunk_c0.data(), sizeof(int32_t) * p->nchunks, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_bias, 0, sizeof(float) * p->Dpad);
     if (e != cudaSuccess) {
@@ -108,13 +112,24 @@ gdws_status_t ensure_device(gdws_plan_s *p)
 
 static int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-// Shared-memory need of the fused bf16 kernel for a candidate tile.
-static size_t fused_smem(const gdws_plan_s *p, const Tile &t)
+// Shared-memory layout of the fused bf16 kernel: two intermediate-tile stages, `nsb` pointwise-weight
+// stages, `nslots` staged-input slots.  Fills t.nsb / t.nslots / t.smem; false if it cannot fit.
+static bool fit_smem(const gdws_plan_s *p, Tile &t)
 {
-    size_t a = 2 * (size_t)kTileRows * kChunk * 2;                 // two intermediate-tile stages
-    size_t b = (size_t)t.nsb * p->Dpad * kChunk * 2;               // pointwise-weight stages
-    size_t x = 2 * (size_t)t.CB * t.plane * 2;                     // two staged input blocks
-    return a + b + x + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    const size_t a = 2 * (size_t)kTileRows * kChunk * 2;
+    const size_t bstage = (size_t)p->Dpad * kChunk * 2;
+    const size_t slot = (size_t)t.span * t.plane * 2;
+    const size_t fixed = a + 1024 /*alignment slack*/ + (size_t)t.TN * t.IH * t.IWp * 4 /*pixel table*/;
+    for (int nsb = (p->Dpad <= 128 ? 3 : 2); nsb >= 2; --nsb) {
+        if (fixed + nsb * bstage + 2 * slot > (size_t)kMaxSmem) continue;
+        int ns = (int)(((size_t)kMaxSmem - fixed - nsb * bstage) / slot);
+        if (ns > 6) ns = 6;
+        t.nsb = nsb;
+        t.nslots = ns;
+        t.smem = fixed + nsb * bstage + ns * slot;
+        return true;
+    }
+    return false;
 }
 
 bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
@@ -125,6 +140,7 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
     double best = 1e300;
     bool found = false;
     const int forced = p->opt_tile;
+    const bool fast_shape = p->k == 3 && (p->stride == 1 || p->stride == 2) && p->opt_a_layout == 0;
     static const int pws[4] = {32, 16, 8, 4};
     for (int pi = 0; pi < 4; ++pi) {
         const int PW = pws[pi];
@@ -133,34 +149,29 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
             const int maxTN = kTileRows / (PH * PW);
             for (int TN = 1; TN <= maxTN; ++TN) {
                 if (TN > 1 && (PH * PW) % 8) continue;
-                if (forced) {
-                    if (TN != ((forced >> 16) & 0xff) || PH != ((forced >> 8) & 0xff) || PW != (forced & 0xff)) continue;
-                }
                 Tile t;
                 t.TN = TN; t.PH = PH; t.PW = PW;
+                if (fast_shape && PW >= 8 && PH % 4 == 0) t.fast = 1;
+                else if (fast_shape && PW == 4) t.fast = 2;
+                if (forced) {
+                    if (TN != ((forced >> 16) & 0xff) || PH != ((forced >> 8) & 0xff) || PW != (forced & 0xff)) continue;
+                } else if (fast_shape && !t.fast) {
+                    continue;                    // a specialised depthwise path exists: only take tiles it covers
+                }
                 t.tiles_w = (Wo + PW - 1) / PW;
                 t.tiles_h = (Ho + PH - 1) / PH;
                 t.tiles_n = (n + TN - 1) / TN;
                 t.IH = (PH - 1) * p->stride + p->k;
                 t.IW = (PW - 1) * p->stride + p->k;
                 t.IWp = round_up(t.IW, 8);
+                if (t.fast == 1 && p->stride == 2) t.IWp = round_up(2 * PW + 2, 8);   // the row path reads 18 columns per group
                 int plane = TN * t.IH * t.IWp;        // elements; make the byte stride = 16 (mod 128)
                 while ((plane * 2) % 128 != 16) plane += 8;
                 t.plane = plane;
-                bool fits = false;
-                for (int CB = 16; CB >= 8 && !fits; CB -= 8) {
-                    // register prefetch of the next block: at most 12 16-byte loads per thread
-                    const int64_t loads = (int64_t)TN * t.IH * t.IWp * (CB / 8);
-                    if (loads > 12 * 256) continue;
-                    for (int nsb = 4; nsb >= 2 && !fits; --nsb) {
-                        t.CB = CB; t.nsb = nsb;
-                        t.smem = fused_smem(p, t);
-                        if (t.smem <= (size_t)kMaxSmem) fits = true;
-                    }
-                }
-                if (!fits) continue;
+                t.span = p->span_max;
+                if (!fit_smem(p, t)) continue;
                 const double tiles = (double)t.tiles();
-                const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IWp) - 1e-3 * PW;
+                const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IWp) * (t.fast ? 1.0 : 4.0) - 1e-3 * PW;
                 if (cost < best) { best = cost; *out = t; found = true; }
             }
         }
@@ -221,6 +232,18 @@ gdws_status_t gdws_plan(int C, int D, int k, int stride, int pad, const int32_t 
         acc += g[c];
     }
     p->off[C] = acc;
+    try {
+        p->chunk_c0.assign(p->nchunks, 0);
+    } catch (...) {
+        delete p;
+        return fail(GDWS_ERR_ALLOC, "gdws_plan: out of host memory");
+    }
+    for (int q = 0; q < p->nchunks; ++q) {   // channel range read by K chunk q
+        const int lo = p->chan[q * kChunk];
+        const int last = std::min(p->G, (q + 1) * kChunk) - 1;
+        p->chunk_c0[q] = lo;
+        p->span_max = std::max(p->span_max, p->chan[last] - lo + 1);
+    }
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
         gdws_status_t st = ensure_device(p);

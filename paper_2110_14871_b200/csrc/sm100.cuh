@@ -1,0 +1,220 @@
+// Device-side building blocks for sm_100a shared by the tensor-core kernels: mbarrier, bulk-copy,
+// tcgen05 (TMEM allocation, MMA, commit, loads) wrappers, operand descriptors, the epilogue.
+//
+// Tensor-core operand conventions used here (sm_100 "UMMA" shared-memory descriptors):
+//   * 128-byte swizzle: within every 1024-byte group of eight 128-byte rows, the 16-byte
+//     column index is XORed with the row index (address bits [4,7) ^= bits [7,10)).
+//   * K-major operand (rows = M or N index, 64 bf16 of K per 128-byte row): row groups
+//     of 8 are 1024 bytes apart (stride byte offset); one MMA of K=16 reads 32 bytes of
+//     each row, so successive K steps advance the start address by 32 bytes.
+//   * MN-major operand (rows = K index, 64 consecutive M per 128-byte row): blocks of
+//     64 M are `leading byte offset` apart, groups of 8 K rows `stride byte offset` apart.
+#pragma once
+
+#include <cuda_bf16.h>
+
+#include "gdws_internal.h"
+
+namespace gdws {
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait.  When the limit runs out (about a second) the thread records `code` in the
+// status word and raises the block's abort flag; from then on every wait in the block returns
+// at once, so that all threads still walk the same control flow, reach the common teardown
+// (barriers stay matched, TMEM is freed) and the kernel ends.
+constexpr uint32_t kSpinLimit = 1u << 22;
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+{
+    if (*abort_flag) return;
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return;
+        if (it > 32) __nanosleep(64);
+        if ((it & 1023) == 1023 && *abort_flag) return;
+    }
+    *abort_flag = 1;
+    atomicOr(status, code);
+}
+// Same, but ignores the abort flag (used in teardown to drain copies that are in flight).
+__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < (1u << 18); ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(64);
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void named_bar_sync(int id, int count)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void sts16(uint32_t addr, uint16_t v)
+{
+    asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+
+// Instruction descriptor of tcgen05.mma kind::f16: fp32 accumulator, bf16 A and B, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(kTileRows >> 4) << 24);
+}
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
+__device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;
+    d |= 2ull << 61;
+    return d;
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+__device__ __forceinline__ uint16_t float_to_bf16_bits(float f)
+{
+    return __bfloat16_as_ushort(__float2bfloat16_rn(f));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    return (uint32_t)float_to_bf16_bits(lo) | ((uint32_t)float_to_bf16_bits(hi) << 16);
+}
+
+// ------------------------------------------------------------------------------------------
+// Epilogue shared by both tensor-core kernels: 16 accumulator columns of one pixel row.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void store_row16(const uint32_t (&acc)[16], const float *__restrict__ bias, int d0, int D,
+                                            int relu, uint16_t *__restrict__ yrow)
+{
+    float v[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        v[j] = __uint_as_float(acc[j]) + __ldg(bias + d0 + j);
+        if (relu) v[j] = fmaxf(v[j], 0.f);
+    }
+    if (d0 + 8 <= D) {
+        uint4 a;
+        a.x = pack_bf16x2(v[0], v[1]); a.y = pack_bf16x2(v[2], v[3]);
+        a.z = pack_bf16x2(v[4], v[5]); a.w = pack_bf16x2(v[6], v[7]);
+        *reinterpret_cast<uint4 *>(yrow + d0) = a;
+    }
+    if (d0 + 16 <= D) {
+        uint4 b;
+        b.x = pack_bf16x2(v[8], v[9]); b.y = pack_bf16x2(v[10], v[11]);
+        b.z = pack_bf16x2(v[12], v[13]); b.w = pack_bf16x2(v[14], v[15]);
+        *reinterpret_cast<uint4 *>(yrow + d0 + 8) = b;
+    }
+}
+
+// Issue the MMAs of one 64-wide K chunk (4 steps of K=16; output channels beyond 256 take a
+// second instruction on the next 256 accumulator columns).
+__device__ __forceinline__ void issue_chunk(uint32_t tmem, uint32_t a_addr, uint32_t b_addr, int Dpad, bool a_mn_major,
+                                            bool first_chunk)
+{
+    const int n0 = Dpad > 256 ? 256 : Dpad;
+    const int n1 = Dpad - n0;
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+        const uint64_t adesc = a_mn_major ? make_sdesc(a_addr + ks * 4096, 1024, 2048)
+                                          : make_sdesc(a_addr + ks * 32, 16, 1024);
+        const uint32_t acc = (first_chunk && ks == 0) ? 0u : 1u;
+        umma_bf16(tmem, adesc, make_sdesc(b_addr + ks * 32, 16, 1024), make_idesc(n0, a_mn_major), acc);
+        if (n1 > 0)
+            umma_bf16(tmem + 256, adesc, make_sdesc(b_addr + 256 * 128 + ks * 32, 16, 1024),
+                      make_idesc(n1, a_mn_major), acc);
+    }
+}
+
+inline int tmem_cols_for(int Dpad)
+{
+    int c = 32;
+    while (c < Dpad) c <<= 1;
+    return c;
+}
+
+// Shared memory to request so that the blocks resident on one SM never ask for more than the
+// 512 TMEM columns together (an allocation that cannot be served would wait).
+inline size_t smem_for_tmem(size_t need, int cols)
+{
+    const int max_ctas = 512 / cols;
+    const size_t floor_bytes = (size_t)kMaxSmem / (max_ctas + 1) + 1024;
+    return need > floor_bytes ? need : floor_bytes;
+}
+
+
+}  // namespace gdws

@@ -84,6 +84,9 @@ BF16_SHAPES = [
     (2, 40, 272, 7, 7, 1, 1, 0, ("uniform", 1, 1)),
     (1, 64, 512, 9, 9, 3, 2, 1, ("heavy",)),
     (2, 16, 32, 33, 35, 3, 1, 1, ("heavy",)),
+    (9, 16, 64, 8, 8, 3, 2, 1, ("uniform", 1, 9)),       # stride 2 onto 4x4 outputs
+    (3, 72, 48, 16, 16, 3, 1, 1, ("const", 1)),            # depthwise-separable special case (g = 1)
+    (1, 8, 16, 40, 70, 3, 1, 1, ("uniform", 5, 9)),
 ]
 
 
@@ -99,6 +102,15 @@ def test_bf16_forward_matches_reference(shape, path, a_layout):
     assert err <= TOL["bf16"], err
     # two bf16 roundings (z and y) should sit far inside the bar
     assert err <= 1e-2, err
+
+
+@pytest.mark.parametrize("tile", [(1 << 16) | (3 << 8) | 32, (2 << 16) | (6 << 8) | 8, (1 << 16) | (1 << 8) | 16])
+def test_bf16_fused_generic_depthwise_path_with_forced_tiles(tile):
+    """Patches the specialised k=3 depthwise code does not cover run the generic code."""
+    spec = small_spec("t", 3, 16, 24, 13, 19, 3, 1, 1, ("uniform", 1, 9), seed=33)
+    data = gi.make_layer(spec)
+    ref, _ = run_oracle(data)
+    assert rel_err(run_gpu(data, path=gdws.PATH_FUSED, tile=tile), ref) <= 1e-2
 
 
 def test_bf16_depthwise_and_pointwise_stages():
