@@ -1,22 +1,26 @@
 // Fused GDWS forward for bf16 NHWC tensors on sm_100a: the G intermediate channels of the GDW
 // stage go from the ALUs to the tensor cores through shared memory and never reach HBM.
 //
-// One block computes one tile of 128 output pixels (TN images x PH x PW patch) for all D output
-// channels.  The intermediate channels are processed in K chunks of 64 (i = 64q .. 64q+63, in the
-// canonical order i = off_c + j), and three kinds of warps run as a pipeline over the chunks:
-//   * 4 staging warps: chunk q reads the contiguous channel range [c0(q), c0(q)+span); a warp
-//     loads those channels of the tile's input patch (with halo, zero filled outside the image)
-//     with 16-byte loads and writes them channel-major into one of `nslots` slots, so that the
+// The kernel is persistent: one block per SM walks over tiles of 128 output pixels (TN images x
+// PH x PW patch, all D output channels).  Within a tile the intermediate channels are processed
+// in K chunks of 64 (i = 64q .. 64q+63, canonical order i = off_c + j).  Five kinds of warps run
+// as one pipeline over the sequence of (tile, chunk) pairs, coupled only by mbarriers:
+//   * 8 staging warps: chunk q reads the contiguous channel range [c0(q), c0(q)+span); the warps
+//     load those channels of the tile's input patch (with halo, zero filled outside the image)
+//     with 16-byte loads and write them channel-major into one of `nslots` slots, so that the
 //     depthwise stage reads runs of consecutive pixels of one channel with 16-byte loads;
 //   * 8 depthwise warps: thread t owns intermediate channel 64q + (t & 63) and a quarter of the
 //     tile's pixels; it keeps its k x k filter in registers, slides down the patch reusing each
 //     input row for up to k output rows, and writes bf16 results as 16-byte pieces into a
 //     pixel-contiguous (MN-major), 128-byte-swizzled tensor-core operand stage;
-//   * 1 control warp: one lane streams the pre-swizzled pointwise-weight chunk (bulk copy with
-//     mbarrier completion) and issues tcgen05.mma into the TMEM accumulator (128 lanes x D
-//     fp32 columns), committing to mbarriers that free the stages.
-// The depthwise warps finally read the accumulator back (tcgen05.ld), add the bias, apply the
-// optional ReLU, round to bf16 and store y.
+//   * 1 control warp: one lane streams the pre-swizzled pointwise weights (bulk copies with
+//     mbarrier completion, a ring of units of at most 256 output channels x 64) and issues
+//     tcgen05.mma into a TMEM accumulator (128 lanes x D fp32 columns; two accumulators when
+//     D <= 256, so that a tile's epilogue overlaps the next tile's main loop);
+//   * 4 epilogue warps: read the finished accumulator (tcgen05.ld), add the bias, apply the
+//     optional ReLU, round to bf16 and store y.
+// Every wait is bounded; a wait that runs out raises a block-wide abort flag that turns all later
+// waits into no-ops, so the block still reaches its teardown, frees TMEM and ends.
 #include "sm100.cuh"
 
 namespace gdws {
@@ -32,16 +36,30 @@ struct FusedParams {
     const int32_t *chunk_c0;
     int *status;
     int N, H, W, C, Ho, Wo, D, Dpad, G, nchunks, stride, pad, relu;
-    int TN, PH, PW, tiles_h, tiles_w;
+    int TN, PH, PW, tiles_h, tiles_w, ntiles;
     int IH, IW, IWp, plane, span, nslots, nsb;
-    int tmem_cols, a_kmajor, dw_math;
+    int nhalf, unit_bytes, nacc, acc_cols;
+    int a_kmajor, dw_math;
 };
 
-constexpr int kDwWarps = 8, kStageWarps = 4;
+// Warp roles, in warpgroups of 4 so that registers can be moved between the roles (setmaxnreg):
+// warps 0-7 depthwise, 8-15 staging, 16 control (17-19 idle), 20-23 epilogue.
+constexpr int kDwWarps = 8, kStageWarps = 8, kEpiWarps = 4;
 constexpr int kDwThreads = kDwWarps * 32;
-constexpr int kStageThreads = kStageWarps * 32;
-constexpr int kFusedThreads = kDwThreads + kStageThreads + 32;
-constexpr int kMaxSlots = 6, kMaxBStages = 4;
+constexpr int kCtrlWarp = kDwWarps + kStageWarps;
+constexpr int kEpiWarp0 = kCtrlWarp + 4;
+constexpr int kFusedThreads = (kEpiWarp0 + kEpiWarps) * 32;
+// Registers per thread after the split.  setmaxnreg.inc can only claim what other warpgroups of the
+// same block released, so the sum must stay within the block's allocation at launch
+// (768 threads x 80 registers, the most that one block of this size can get).
+constexpr int kRegsLaunch = 80, kRegsDw = 112, kRegsStage = 80, kRegsCtrl = 40, kRegsEpi = 56;
+static_assert(kDwThreads * kRegsDw + kStageWarps * 32 * kRegsStage + 128 * kRegsCtrl + kEpiWarps * 32 * kRegsEpi <=
+                  kFusedThreads * kRegsLaunch,
+              "register split exceeds the block's allocation: setmaxnreg.inc would wait forever");
+
+template <int N> __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+constexpr int kMaxSlots = 8, kMaxBUnits = 8;
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr)
 {
@@ -231,146 +249,228 @@ template <int K, int MODE, int S>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __grid_constant__ FusedParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    // a_full[2] | mma_done[2] | b_full[4] | b_free[4] | x_full[6] | x_free[6]
-    __shared__ __align__(8) uint64_t bars[2 + 2 + kMaxBStages * 2 + kMaxSlots * 2];
+    // a_full[2] a_free[2] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2]
+    __shared__ __align__(8) uint64_t bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t a_s = smem_u32(base);
-    const uint32_t b_bytes = (uint32_t)P.Dpad * kChunk * 2;
     const uint32_t b_s = a_s + 2 * 16384;
-    const uint32_t x_s = b_s + (uint32_t)P.nsb * b_bytes;
+    const uint32_t x_s = b_s + (uint32_t)P.nsb * P.unit_bytes;
     const uint32_t slot_bytes = (uint32_t)P.span * P.plane * 2;
-    const uint32_t bar_afull = smem_u32(&bars[0]), bar_done = smem_u32(&bars[2]);
-    const uint32_t bar_bfull = smem_u32(&bars[4]), bar_bfree = smem_u32(&bars[4 + kMaxBStages]);
-    const uint32_t bar_xfull = smem_u32(&bars[4 + 2 * kMaxBStages]);
-    const uint32_t bar_xfree = smem_u32(&bars[4 + 2 * kMaxBStages + kMaxSlots]);
-    constexpr int kCtrlWarp = kDwWarps + kStageWarps;
+    const uint32_t bar_afull = smem_u32(&bars[0]), bar_afree = smem_u32(&bars[2]);
+    const uint32_t bar_bfull = smem_u32(&bars[4]), bar_bfree = smem_u32(&bars[4 + kMaxBUnits]);
+    const uint32_t bar_xfull = smem_u32(&bars[4 + 2 * kMaxBUnits]);
+    const uint32_t bar_xfree = smem_u32(&bars[4 + 2 * kMaxBUnits + kMaxSlots]);
+    const uint32_t bar_accfull = smem_u32(&bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots]);
+    const uint32_t bar_accfree = bar_accfull + 16;
+    const int wps = kStageWarps / P.nslots;               // staging warps that share one slot
+    const int npair = (P.TN * P.IH * P.IWp) >> 1;
 
     if (tid == 0) {
         abort_flag = 0;
-        for (int i = 0; i < 2; ++i) { mbar_init(bar_afull + 8 * i, kDwThreads); mbar_init(bar_done + 8 * i, 1); }
-        for (int i = 0; i < kMaxBStages; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
-        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(bar_xfull + 8 * i, 32); mbar_init(bar_xfree + 8 * i, kDwThreads); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_afull + 8 * i, kDwThreads);
+            mbar_init(bar_afree + 8 * i, 1);
+            mbar_init(bar_accfull + 8 * i, 1);
+            mbar_init(bar_accfree + 8 * i, kEpiWarps * 32);
+        }
+        for (int i = 0; i < kMaxBUnits; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
+        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(bar_xfull + 8 * i, 32 * wps); mbar_init(bar_xfree + 8 * i, kDwThreads); }
         fence_mbar_init();
     }
-    if (warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)P.tmem_cols);
+    if (warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
+
+    // Patch table (the same for every tile): for each pair of horizontally adjacent patch positions
+    // the pixel offset (tn*H + ih)*W + iw relative to the tile's first input pixel, and tn, ih, iw.
+    int2 *pix_tab = reinterpret_cast<int2 *>(base + (x_s - a_s) + (size_t)P.nslots * slot_bytes);
+    for (int pp = tid; pp < npair; pp += kFusedThreads) {
+        const int t = 2 * pp;
+        const int iw = t % P.IWp;
+        const int r = t / P.IWp;
+        const int ih = r % P.IH, tn = r / P.IH;
+        pix_tab[pp] = make_int2((tn * P.H + ih) * P.W + iw, tn | (ih << 8) | (iw << 16));
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
-    // tile -> first image / output row / output column
-    int tile = blockIdx.x;
-    const int bw = tile % P.tiles_w;
-    tile /= P.tiles_w;
-    const int bh = tile % P.tiles_h;
-    const int bn = tile / P.tiles_h;
-    const int n0 = bn * P.TN, ho0 = bh * P.PH, wo0 = bw * P.PW;
+    const int my_tiles = (P.ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int total_chunks = my_tiles * P.nchunks;
+    const int tiles_hw = P.tiles_h * P.tiles_w;
 
-    // Pixel table of the tile's input patch: for every pair of horizontally adjacent patch
-    // positions the linear pixel index (n*H + hi)*W + wi in x, or -1 where the patch leaves the image.
-    int2 *pix_tab = reinterpret_cast<int2 *>(base + (x_s - a_s) + (size_t)P.nslots * slot_bytes);
-    {
-        const int hi0 = ho0 * P.stride - P.pad, wi0 = wo0 * P.stride - P.pad;
-        const int npix = P.TN * P.IH * P.IWp;
-        for (int t = tid; t < npix; t += kFusedThreads) {
-            const int iw = t % P.IWp;
-            const int r = t / P.IWp;
-            const int ih = r % P.IH, tn = r / P.IH;
-            const int n = n0 + tn, hi = hi0 + ih, wi = wi0 + iw;
-            const bool in = n < P.N && hi >= 0 && hi < P.H && wi >= 0 && wi < P.W && iw < P.IW;
-            reinterpret_cast<int *>(pix_tab)[t] = in ? (n * P.H + hi) * P.W + wi : -1;
-        }
-    }
-    __syncthreads();
-
-    if (warp == kCtrlWarp) {
+    if (warp >= kCtrlWarp && warp < kEpiWarp0) {
         // ---------------- control warp: weight copies and MMA issue (one lane) ----------------
-        if (lane == 0) {
-            const int pre = P.nchunks < P.nsb ? P.nchunks : P.nsb;
-            for (int q = 0; q < pre; ++q) {
-                mbar_expect_tx(bar_bfull + 8 * q, b_bytes);
-                bulk_g2s(b_s + q * b_bytes, P.pw_img + (size_t)q * P.Dpad * kChunk, b_bytes, bar_bfull + 8 * q);
-            }
-            for (int q = 0; q < P.nchunks; ++q) {
-                const int sa = q & 1, sb = q % P.nsb;
-                mbar_wait(bar_bfull + 8 * sb, (q / P.nsb) & 1, &abort_flag, P.status, kStatusWaitOperand);
-                mbar_wait(bar_afull + 8 * sa, (q >> 1) & 1, &abort_flag, P.status, kStatusWaitOperand);
+        regs_dec<kRegsCtrl>();
+        if (warp == kCtrlWarp && lane == 0) {
+            const int units_per_tile = P.nchunks * P.nhalf;
+            const int total_units = my_tiles * units_per_tile;
+            const int rows0 = P.Dpad > 256 ? 256 : P.Dpad, rows1 = P.Dpad - rows0;
+            int cu = 0;                                   // next weight unit to copy
+            auto issue_copy = [&](int u) {
+                const int within = u % units_per_tile;
+                const int q = within / P.nhalf, h = within - q * P.nhalf;
+                const int sb = u % P.nsb;
+                const uint32_t bytes = (uint32_t)(h ? rows1 : rows0) * 128u;
+                mbar_expect_tx(bar_bfull + 8 * sb, bytes);
+                bulk_g2s(b_s + sb * P.unit_bytes, P.pw_img + ((size_t)q * P.Dpad + h * 256) * kChunk, bytes,
+                         bar_bfull + 8 * sb);
+            };
+            while (cu < total_units && cu < P.nsb) issue_copy(cu++);
+            int gq = 0, gu = 0;
+            for (int tl = 0; tl < my_tiles; ++tl) {
+                const int buf = tl % P.nacc;
+                if (tl >= P.nacc)
+                    mbar_wait(bar_accfree + 8 * buf, ((tl / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
                 tc_fence_after();
-                issue_chunk(tmem, a_s + sa * 16384, b_s + sb * b_bytes, P.Dpad, !P.a_kmajor, q == 0);
-                umma_commit(bar_done + 8 * sa);
-                umma_commit(bar_bfree + 8 * sb);
-                // refill the weight stage of the previous chunk once its MMAs have finished
-                const int qn = q - 1 + P.nsb;
-                if (q >= 1 && qn < P.nchunks) {
-                    const int sp = (q - 1) % P.nsb;
-                    mbar_wait(bar_bfree + 8 * sp, ((q - 1) / P.nsb) & 1, &abort_flag, P.status, kStatusWaitStage);
-                    mbar_expect_tx(bar_bfull + 8 * sp, b_bytes);
-                    bulk_g2s(b_s + sp * b_bytes, P.pw_img + (size_t)qn * P.Dpad * kChunk, b_bytes, bar_bfull + 8 * sp);
+                for (int q = 0; q < P.nchunks; ++q, ++gq) {
+                    const int sa = gq & 1;
+                    mbar_wait(bar_afull + 8 * sa, (gq >> 1) & 1, &abort_flag, P.status, kStatusWaitOperand);
+                    for (int h = 0; h < P.nhalf; ++h, ++gu) {
+                        const int sb = gu % P.nsb;
+                        mbar_wait(bar_bfull + 8 * sb, (gu / P.nsb) & 1, &abort_flag, P.status, kStatusWaitOperand);
+                        tc_fence_after();
+                        const uint32_t d_tmem = tmem + (uint32_t)(buf * P.acc_cols + h * 256);
+                        const uint32_t a_addr = a_s + sa * 16384, b_addr = b_s + sb * P.unit_bytes;
+                        const uint32_t idesc = make_idesc(h ? rows1 : rows0, !P.a_kmajor);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t adesc = !P.a_kmajor ? make_sdesc(a_addr + ks * 4096, 1024, 2048)
+                                                               : make_sdesc(a_addr + ks * 32, 16, 1024);
+                            umma_bf16(d_tmem, adesc, make_sdesc(b_addr + ks * 32, 16, 1024), idesc,
+                                      (q == 0 && ks == 0) ? 0u : 1u);
+                        }
+                        umma_commit(bar_bfree + 8 * sb);
+                        // refill the ring: unit cu reuses the slot of unit cu - nsb, whose MMAs were
+                        // issued at least one unit ago
+                        while (cu < total_units && cu <= gu + P.nsb - 1) {
+                            mbar_wait(bar_bfree + 8 * (cu % P.nsb), ((cu / P.nsb) - 1) & 1, &abort_flag, P.status,
+                                      kStatusWaitStage);
+                            issue_copy(cu++);
+                        }
+                    }
+                    umma_commit(bar_afree + 8 * sa);
                 }
+                umma_commit(bar_accfull + 8 * buf);
             }
-            // every copy issued was awaited above; await the last commits so that nothing is
-            // still arriving on this block's barriers when it exits
-            for (int q = (P.nchunks > P.nsb ? P.nchunks - P.nsb : 0); q < P.nchunks; ++q)
-                mbar_wait_drain(bar_bfree + 8 * (q % P.nsb), (q / P.nsb) & 1);
+        }
+    } else if (warp >= kEpiWarp0) {
+        // ---------------- epilogue warps: TMEM -> registers -> bias / ReLU -> bf16 -> global ----------------
+        regs_dec<kRegsEpi>();
+        const int lg = warp & 3;                          // TMEM lanes 32*lg .. 32*lg+31 belong to this warp
+        const int r = lg * 32 + lane;
+        const int hw = P.PH * P.PW;
+        const int tn = r / hw;
+        const int rem = r - tn * hw;
+        const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
+        for (int tl = 0; tl < my_tiles; ++tl) {
+            int tile = (int)blockIdx.x + tl * (int)gridDim.x;
+            const int bn = tile / tiles_hw;
+            tile -= bn * tiles_hw;
+            const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+            const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
+            const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
+            uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D;
+            const int buf = tl % P.nacc;
+            mbar_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
+            tc_fence_after();
+            const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * P.acc_cols);
+            for (int d0 = 0; d0 < P.Dpad; d0 += 16) {
+                uint32_t acc[16];
+                tmem_ld16(t_base + (uint32_t)d0, acc);
+                tmem_ld_wait();
+                if (live) store_row16(acc, P.bias, d0, P.D, P.relu, yrow);
+            }
+            tc_fence_before();
+            mbar_arrive(bar_accfree + 8 * buf);
         }
     } else if (warp >= kDwWarps) {
-        // ---------------- staging warps: slot s is always filled by warp s % 4 ----------------
+        // ---------------- staging warps: slot s is filled by the warps w with w % nslots == s ----------------
+        if (kRegsStage < kRegsLaunch) regs_dec<kRegsStage>();
         const int sw = warp - kDwWarps;
-        const int npair = (P.TN * P.IH * P.IWp) >> 1;
-        for (int q = 0; q < P.nchunks; ++q) {
-            const int slot = q % P.nslots;
-            if ((slot & (kStageWarps - 1)) != sw) continue;
-            const int use = q / P.nslots;
+        const int slot = sw % P.nslots, share = sw / P.nslots;
+        const uint32_t xs = x_s + slot * slot_bytes;
+        for (int gq = slot; gq < total_chunks; gq += P.nslots) {
+            const int tl = gq / P.nchunks, q = gq - tl * P.nchunks;
+            int tile = (int)blockIdx.x + tl * (int)gridDim.x;
+            const int bn = tile / tiles_hw;
+            tile -= bn * tiles_hw;
+            const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+            const int n0 = bn * P.TN, hi0 = bh * P.PH * P.stride - P.pad, wi0 = bw * P.PW * P.stride - P.pad;
+            const long long pbase = ((long long)n0 * P.H + hi0) * P.W + wi0;
+            const int use = gq / P.nslots;
             if (use >= 1) mbar_wait(bar_xfree + 8 * slot, (use - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
             const int c0 = __ldg(P.chunk_c0 + q);
             const int ilast = min(P.G, (q + 1) * kChunk) - 1;
             const int c1 = q * kChunk < P.G ? __ldg(P.chan + ilast) : c0;       // last channel of the chunk
             const int gr0 = c0 >> 3, ngr = (c1 >> 3) - gr0 + 1;
-            const uint32_t xs = x_s + slot * slot_bytes;
-            for (int gr = 0; gr < ngr; ++gr) {
-                const int cb = (gr0 + gr) * 8 - c0;           // slot channel of the group's first channel
-                const uint16_t *xg = P.x + (gr0 + gr) * 8;
-                const bool whole = cb >= 0 && cb + 8 <= P.span;
-                constexpr int kBatch = 4;                     // pixel pairs per lane in flight
-                for (int p0 = lane; p0 < npair; p0 += 32 * kBatch) {
-                    uint4 va[kBatch], vb[kBatch];
+            const int items = ngr * npair;                    // (channel group, pixel pair), pixel pair fastest
+            constexpr int kBatch = 4;                         // pixel pairs per lane in flight (8 loads)
+            for (int t0 = share * 32 * kBatch + lane; t0 < items; t0 += 32 * kBatch * wps) {
+                uint4 va[kBatch], vb[kBatch];
 #pragma unroll
-                    for (int m = 0; m < kBatch; ++m) {
-                        const int pp = p0 + m * 32;
-                        va[m] = make_uint4(0, 0, 0, 0);
-                        vb[m] = make_uint4(0, 0, 0, 0);
-                        if (pp < npair) {
-                            const int2 o = pix_tab[pp];
-                            if (o.x >= 0) va[m] = __ldg(reinterpret_cast<const uint4 *>(xg + (size_t)o.x * P.C));
-                            if (o.y >= 0) vb[m] = __ldg(reinterpret_cast<const uint4 *>(xg + (size_t)o.y * P.C));
-                        }
+                for (int m = 0; m < kBatch; ++m) {
+                    const int t = t0 + m * 32;
+                    va[m] = make_uint4(0, 0, 0, 0);
+                    vb[m] = make_uint4(0, 0, 0, 0);
+                    if (t < items) {
+                        const int gr = t / npair, pp = t - gr * npair;
+                        const int2 e = pix_tab[pp];
+                        const int tn = e.y & 0xff, ih = (e.y >> 8) & 0xff, iw = e.y >> 16;
+                        const int hi = hi0 + ih, wi = wi0 + iw;
+                        const bool rowok = n0 + tn < P.N && hi >= 0 && hi < P.H;
+                        const uint16_t *xp = P.x + (pbase + e.x) * P.C + (gr0 + gr) * 8;
+                        if (rowok && wi >= 0 && wi < P.W && iw < P.IW) va[m] = __ldg(reinterpret_cast<const uint4 *>(xp));
+                        if (rowok && wi + 1 >= 0 && wi + 1 < P.W && iw + 1 < P.IW)
+                            vb[m] = __ldg(reinterpret_cast<const uint4 *>(xp + P.C));
                     }
+                }
 #pragma unroll
-                    for (int m = 0; m < kBatch; ++m) {
-                        const int pp = p0 + m * 32;
-                        if (pp < npair) {
-                            const uint32_t a4[4] = {va[m].x, va[m].y, va[m].z, va[m].w};
-                            const uint32_t b4[4] = {vb[m].x, vb[m].y, vb[m].z, vb[m].w};
-                            const uint32_t dst = xs + (uint32_t)(cb * P.plane + 2 * pp) * 2;
+                for (int m = 0; m < kBatch; ++m) {
+                    const int t = t0 + m * 32;
+                    if (t < items) {
+                        const int gr = t / npair, pp = t - gr * npair;
+                        const int cb = (gr0 + gr) * 8 - c0;   // slot channel of the group's first channel
+                        const bool whole = cb >= 0 && cb + 8 <= P.span;
+                        const uint32_t a4[4] = {va[m].x, va[m].y, va[m].z, va[m].w};
+                        const uint32_t b4[4] = {vb[m].x, vb[m].y, vb[m].z, vb[m].w};
+                        const uint32_t dst = xs + (uint32_t)(cb * P.plane + 2 * pp) * 2;
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                // channel cb+e of the two pixels -> one 32-bit store
-                                const uint32_t word = (e & 1) ? __byte_perm(a4[e >> 1], b4[e >> 1], 0x7632)
-                                                              : __byte_perm(a4[e >> 1], b4[e >> 1], 0x5410);
-                                if (whole || (cb + e >= 0 && cb + e < P.span))
-                                    sts32(dst + (uint32_t)(e * P.plane * 2), word);
-                            }
+                        for (int e = 0; e < 8; ++e) {
+                            // channel cb+e of the two pixels -> one 32-bit store
+                            const uint32_t word = (e & 1) ? __byte_perm(a4[e >> 1], b4[e >> 1], 0x7632)
+                                                          : __byte_perm(a4[e >> 1], b4[e >> 1], 0x5410);
+                            if (whole || (cb + e >= 0 && cb + e < P.span))
+                                sts32(dst + (uint32_t)(e * P.plane * 2), word);
                         }
                     }
                 }
             }
             mbar_arrive(bar_xfull + 8 * slot);
+            // first chunk of a tile: pull the next tile's input patch towards L2
+            if (q == 0 && share == 0 && tl + 1 < my_tiles) {
+                int nt = (int)blockIdx.x + (tl + 1) * (int)gridDim.x;
+                const int nbn = nt / tiles_hw;
+                nt -= nbn * tiles_hw;
+                const int nbh = nt / P.tiles_w, nbw = nt - nbh * P.tiles_w;
+                const int nn0 = nbn * P.TN, nhi0 = nbh * P.PH * P.stride - P.pad, nwi0 = nbw * P.PW * P.stride - P.pad;
+                const long long nbase = ((long long)nn0 * P.H + nhi0) * P.W + nwi0;
+                for (int pp = lane; pp < npair; pp += 32) {
+                    const int2 e = pix_tab[pp];
+                    const int tn = e.y & 0xff, ih = (e.y >> 8) & 0xff, iw = e.y >> 16;
+                    const int hi = nhi0 + ih, wi = nwi0 + iw;
+                    if (nn0 + tn < P.N && hi >= 0 && hi < P.H && wi >= 0 && wi + 1 < P.W && iw + 1 < P.IW) {
+                        const char *px = reinterpret_cast<const char *>(P.x + (nbase + e.x) * P.C);
+                        for (int b = 0; b < P.C * 4; b += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(px + b));
+                    }
+                }
+            }
         }
     } else {
         // ---------------- depthwise warps ----------------
+        regs_inc<kRegsDw>();
         const int il = tid & 63, run = tid >> 6;
         float w[9];
         int cl = 0;
@@ -384,17 +484,19 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             cl = c < 0 ? 0 : c - __ldg(P.chunk_c0 + q);
         };
         load_weights(0);
-        for (int q = 0; q < P.nchunks; ++q) {
-            const int sa = q & 1, slot = q % P.nslots;
+        int q = 0;
+        for (int gq = 0; gq < total_chunks; ++gq) {
+            const int sa = gq & 1, slot = gq % P.nslots;
             const int i = q * kChunk + il;
             const bool live_i = i < P.G;
             float wq[9];
 #pragma unroll
             for (int t = 0; t < 9; ++t) wq[t] = w[t];
             const int clq = cl;
-            if (q + 1 < P.nchunks) load_weights(q + 1);     // next chunk's filter while this one computes
-            mbar_wait(bar_xfull + 8 * slot, (q / P.nslots) & 1, &abort_flag, P.status, kStatusWaitOperand);
-            if (q >= 2) mbar_wait(bar_done + 8 * sa, ((q >> 1) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+            const int qn = (q + 1 == P.nchunks) ? 0 : q + 1;
+            if (gq + 1 < total_chunks) load_weights(qn);    // next chunk's filter while this one computes
+            mbar_wait(bar_xfull + 8 * slot, (gq / P.nslots) & 1, &abort_flag, P.status, kStatusWaitOperand);
+            if (gq >= 2) mbar_wait(bar_afree + 8 * sa, ((gq >> 1) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
             const uint32_t xs = x_s + slot * slot_bytes;
             const uint32_t a_stage = a_s + sa * 16384;
             if (MODE == 1) dw_rows_k3<S>(P, xs, clq, wq, il, run, live_i, a_stage);
@@ -403,42 +505,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             fence_proxy_async();
             mbar_arrive(bar_afull + 8 * sa);
             mbar_arrive(bar_xfree + 8 * slot);
-        }
-
-        // ---------------- epilogue: TMEM -> registers -> bias / ReLU -> bf16 -> global ----------------
-        {
-            const int ql = P.nchunks - 1;
-            mbar_wait(bar_done + 8 * (ql & 1), (ql >> 1) & 1, &abort_flag, P.status, kStatusWaitMma);
-            if (P.nchunks >= 2) {
-                const int qo = P.nchunks - 2;
-                mbar_wait(bar_done + 8 * (qo & 1), (qo >> 1) & 1, &abort_flag, P.status, kStatusWaitMma);
-            }
-        }
-        tc_fence_after();
-        const int lg = warp & 3, half = warp >> 2;
-        const int r = lg * 32 + lane;
-        const int hw = P.PH * P.PW;
-        const int tn = r / hw;
-        const int rem = r - tn * hw;
-        const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
-        const int n = n0 + tn, ho = ho0 + ph, wo = wo0 + pw_;
-        const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
-        uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D;
-        for (int d0 = half * 16; d0 < P.Dpad; d0 += 32) {
-            uint32_t acc[16];
-            tmem_ld16(tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)d0, acc);
-            tmem_ld_wait();
-            if (live) store_row16(acc, P.bias, d0, P.D, P.relu, yrow);
+            q = qn;
         }
     }
     tc_fence_before();
     __syncthreads();
     __syncwarp();
-    if (warp == kCtrlWarp) tmem_dealloc(tmem, (uint32_t)P.tmem_cols);
+    if (warp == kCtrlWarp) tmem_dealloc(tmem, (uint32_t)(P.nacc * P.acc_cols));
 }
 
 template <int K, int MODE, int S>
-static gdws_status_t launch_fused(const FusedParams &P, int device, int64_t tiles, size_t smem, cudaStream_t st)
+static gdws_status_t launch_fused(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
 {
     cudaError_t e = cudaSuccess;
     static bool attr_set[64] = {};
@@ -447,7 +524,7 @@ static gdws_status_t launch_fused(const FusedParams &P, int device, int64_t tile
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_bf16_kernel)");
         attr_set[device & 63] = true;
     }
-    fused_bf16_kernel<K, MODE, S><<<(int)tiles, kFusedThreads, smem, st>>>(P);
+    fused_bf16_kernel<K, MODE, S><<<grid, kFusedThreads, smem, st>>>(P);
     e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "fused_bf16_kernel launch");
 }
@@ -462,6 +539,10 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
         return fail(GDWS_ERR_UNSUPPORTED, "no fused tile fits this shape in shared memory");
     if (t.tiles() > 0x7fffffffLL) return fail(GDWS_ERR_UNSUPPORTED, "too many tiles");
     if ((long long)x->n * x->h * x->w > 0x7fffffffLL) return fail(GDWS_ERR_UNSUPPORTED, "more than 2^31 input pixels");
+    if (p->sm_count <= 0) {
+        cudaError_t e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute(MultiProcessorCount)");
+    }
     FusedParams P;
     P.x = (const uint16_t *)x->ptr; P.y = (uint16_t *)y->ptr;
     P.dw = p->d_dw; P.dw2 = p->d_dw2; P.pw_img = p->d_pw_img; P.bias = p->d_bias;
@@ -469,27 +550,30 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
     P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = y->h; P.Wo = y->w; P.D = p->D; P.Dpad = p->Dpad;
     P.G = p->G; P.nchunks = p->nchunks; P.stride = p->stride; P.pad = p->pad;
     P.relu = p->opt_relu;
-    P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w;
+    P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
     P.IH = t.IH; P.IW = t.IW; P.IWp = t.IWp; P.plane = t.plane; P.span = t.span; P.nslots = t.nslots; P.nsb = t.nsb;
-    P.tmem_cols = tmem_cols_for(p->Dpad);
+    P.nhalf = p->Dpad > 256 ? 2 : 1;
+    P.unit_bytes = (p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
+    P.acc_cols = tmem_cols_for(p->Dpad);
+    P.nacc = P.acc_cols <= 256 ? 2 : 1;
     P.a_kmajor = p->opt_a_layout;
     P.dw_math = p->opt_dw_math;
-    const size_t smem = smem_for_tmem(t.smem, P.tmem_cols);
-    const int64_t tiles = t.tiles();
+    const size_t smem = t.smem;     // one block per SM (register file), so the TMEM columns are never oversubscribed
+    const int grid = P.ntiles < p->sm_count ? P.ntiles : p->sm_count;
     gdws_status_t rc;
-    if (t.fast == 1 && p->stride == 1) rc = launch_fused<3, 1, 1>(P, p->device, tiles, smem, st);
-    else if (t.fast == 1 && p->stride == 2) rc = launch_fused<3, 1, 2>(P, p->device, tiles, smem, st);
-    else if (t.fast == 2 && p->stride == 1) rc = launch_fused<3, 2, 1>(P, p->device, tiles, smem, st);
-    else if (t.fast == 2 && p->stride == 2) rc = launch_fused<3, 2, 2>(P, p->device, tiles, smem, st);
+    if (t.fast == 1 && p->stride == 1) rc = launch_fused<3, 1, 1>(P, p->device, grid, smem, st);
+    else if (t.fast == 1 && p->stride == 2) rc = launch_fused<3, 1, 2>(P, p->device, grid, smem, st);
+    else if (t.fast == 2 && p->stride == 1) rc = launch_fused<3, 2, 1>(P, p->device, grid, smem, st);
+    else if (t.fast == 2 && p->stride == 2) rc = launch_fused<3, 2, 2>(P, p->device, grid, smem, st);
     else {
         switch (p->k) {
-        case 1: rc = launch_fused<1, 0, 1>(P, p->device, tiles, smem, st); break;
-        case 2: rc = launch_fused<2, 0, 1>(P, p->device, tiles, smem, st); break;
-        case 3: rc = launch_fused<3, 0, 1>(P, p->device, tiles, smem, st); break;
-        case 4: rc = launch_fused<4, 0, 1>(P, p->device, tiles, smem, st); break;
-        case 5: rc = launch_fused<5, 0, 1>(P, p->device, tiles, smem, st); break;
-        case 6: rc = launch_fused<6, 0, 1>(P, p->device, tiles, smem, st); break;
-        case 7: rc = launch_fused<7, 0, 1>(P, p->device, tiles, smem, st); break;
+        case 1: rc = launch_fused<1, 0, 1>(P, p->device, grid, smem, st); break;
+        case 2: rc = launch_fused<2, 0, 1>(P, p->device, grid, smem, st); break;
+        case 3: rc = launch_fused<3, 0, 1>(P, p->device, grid, smem, st); break;
+        case 4: rc = launch_fused<4, 0, 1>(P, p->device, grid, smem, st); break;
+        case 5: rc = launch_fused<5, 0, 1>(P, p->device, grid, smem, st); break;
+        case 6: rc = launch_fused<6, 0, 1>(P, p->device, grid, smem, st); break;
+        case 7: rc = launch_fused<7, 0, 1>(P, p->device, grid, smem, st); break;
         default: return fail(GDWS_ERR_UNSUPPORTED, "k=%d", p->k);
         }
     }

@@ -53,6 +53,7 @@ struct gdws_plan_s {
 
     // device side (allocated by ensure_device)
     int device = -1;
+    int sm_count = 0;              // SMs of the plan's device (grid size of the persistent kernel)
     bool arch_ok = false;          // the plan's device was checked to be compute capability 10.x
     int32_t *d_off = nullptr;      // [C+1]
     int32_t *d_chan = nullptr;     // [Gpad], -1 for padding

@@ -112,24 +112,32 @@ gdws_status_t ensure_device(gdws_plan_s *p)
 
 static int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-// Shared-memory layout of the fused bf16 kernel: two intermediate-tile stages, `nsb` pointwise-weight
-// stages, `nslots` staged-input slots.  Fills t.nsb / t.nslots / t.smem; false if it cannot fit.
+// Shared-memory layout of the fused bf16 kernel: two intermediate-tile stages, a ring of `nsb`
+// pointwise-weight units (a unit = one K chunk x up to 256 output channels, at most 32 KB), `nslots`
+// staged-input slots (2, 4 or 8) and the patch table.  Fills t.nsb / t.nslots / t.smem; false if
+// it cannot fit.  Prefers at least 3 chunks of weights and 4 input slots in flight.
 static bool fit_smem(const gdws_plan_s *p, Tile &t)
 {
     const size_t a = 2 * (size_t)kTileRows * kChunk * 2;
-    const size_t bstage = (size_t)p->Dpad * kChunk * 2;
+    const int nhalf = p->Dpad > 256 ? 2 : 1;
+    const size_t unit = (size_t)(p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
     const size_t slot = (size_t)t.span * t.plane * 2;
-    const size_t fixed = a + 1024 /*alignment slack*/ + (size_t)t.TN * t.IH * t.IWp * 4 /*pixel table*/;
-    for (int nsb = (p->Dpad <= 128 ? 3 : 2); nsb >= 2; --nsb) {
-        if (fixed + nsb * bstage + 2 * slot > (size_t)kMaxSmem) continue;
-        int ns = (int)(((size_t)kMaxSmem - fixed - nsb * bstage) / slot);
-        if (ns > 6) ns = 6;
-        t.nsb = nsb;
-        t.nslots = ns;
-        t.smem = fixed + nsb * bstage + ns * slot;
-        return true;
+    const size_t fixed = a + 1024 /*alignment slack*/ + (size_t)t.TN * t.IH * t.IWp * 4 /*patch table*/;
+    int best_score = -1;
+    for (int ns = 2; ns <= 8; ns *= 2) {
+        if (fixed + ns * slot + (size_t)(nhalf + 1) * unit > (size_t)kMaxSmem) break;
+        int nsb = (int)(((size_t)kMaxSmem - fixed - ns * slot) / unit);
+        if (nsb > 8) nsb = 8;
+        const int depth_b = nsb / nhalf;
+        const int score = 100 * std::min(std::min(depth_b, ns), 4) + 10 * std::min(depth_b, 6) + ns;
+        if (score > best_score) {
+            best_score = score;
+            t.nsb = nsb;
+            t.nslots = ns;
+            t.smem = fixed + nsb * unit + ns * slot;
+        }
     }
-    return false;
+    return best_score >= 0;
 }
 
 bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)

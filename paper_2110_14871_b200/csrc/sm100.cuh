@@ -152,7 +152,9 @@ __device__ __forceinline__ uint16_t float_to_bf16_bits(float f)
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
-    return (uint32_t)float_to_bf16_bits(lo) | ((uint32_t)float_to_bf16_bits(hi) << 16);
+    uint32_t r;   // one packed conversion: low half <- lo, high half <- hi (round to nearest even)
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
 }
 
 // ------------------------------------------------------------------------------------------
