@@ -208,6 +208,39 @@ GDWS_API gdws_status_t gdws_forward_host(gdws_plan_t *plan, const gdws_tensor_t 
                                          gdws_tensor_t *y_host, void *stream);
 
 /*
+ * gdws_forward_static -- gdws_forward on the unfused path, for callers that cannot allocate device
+ * memory.  (The paper has no counterpart; this is an addition of the library.)
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region whose memory plan
+ * was fixed up front (a real-time or safety-checked inference loop that forbids allocation after
+ * start-up, a process whose device memory is handed out entirely by another framework's pool, a
+ * callback that may not block on the allocator) -- and that therefore can neither size a workspace
+ * with gdws_workspace_bytes / gdws_set_workspace nor let the library grow one.
+ * What it does: the GDW kernel writes the G intermediate channels z into a fixed scratch array that
+ * is part of the library image (GDWS_STATIC_SCRATCH_BYTES, 16 MiB; every GPU that loads the library
+ * holds it until the process ends), and the PW kernel reads them from there.  Arguments, supported
+ * tensors, weight rules and results are those of gdws_forward with GDWS_PATH_UNFUSED; the plan's
+ * workspace and path options are ignored.  The call itself, and the kernels it launches, allocate
+ * nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ * Limits and rules:
+ *   - z must fit: gdws_workspace_bytes(plan, dtype, n, h, w) <= gdws_static_scratch_bytes(), else
+ *     GDWS_ERR_UNSUPPORTED (nothing is launched).
+ *   - The plan must have been built with its device current (that is where the plan's own tables
+ *     were allocated); otherwise GDWS_ERR_INVALID_ARG.
+ *   - The first call on each device looks up the scratch array's device address
+ *     (cudaGetSymbolAddress).  Make that first call outside any stream capture.
+ *   - All calls on one GPU share the one array, whatever the plan or stream, and it keeps what the
+ *     last call left there.  Nothing has to be cleared: each call overwrites every element of z that
+ *     it reads.  Two calls whose kernels may overlap on the GPU (different streams) race on it:
+ *     order them on one stream or with events.
+ */
+#define GDWS_STATIC_SCRATCH_BYTES (16u << 20)
+GDWS_API gdws_status_t gdws_forward_static(gdws_plan_t *plan, const gdws_tensor_t *x, const void *dw_w,
+                                           const void *pw_w, const float *bias, gdws_tensor_t *y,
+                                           void *stream);
+/* Size in bytes of the built-in scratch array used by gdws_forward_static. */
+GDWS_API size_t gdws_static_scratch_bytes(void);
+
+/*
  * gdws_status -- read (and clear) the plan's device status word; synchronises with the
  * device.  GDWS_OK, or GDWS_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel expired
  * (the kernel then skipped its remaining work; outputs of that launch are undefined).

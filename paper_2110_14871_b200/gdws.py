@@ -27,7 +27,7 @@ EXPORTS = [
     "gdws_plan", "gdws_plan_set_option", "gdws_plan_info", "gdws_plan_tables", "gdws_plan_tile",
     "gdws_out_dim", "gdws_pack_weights", "gdws_workspace_bytes", "gdws_set_workspace", "gdws_forward",
     "gdws_depthwise", "gdws_pointwise", "gdws_forward_host", "gdws_status", "gdws_launch_count",
-    "gdws_last_error", "gdws_version", "gdws_destroy",
+    "gdws_last_error", "gdws_version", "gdws_destroy", "gdws_forward_static", "gdws_static_scratch_bytes",
 ]
 
 
@@ -87,6 +87,10 @@ def lib() -> ctypes.CDLL:
     L.gdws_pointwise.restype = ci
     L.gdws_forward_host.argtypes = [vp, pt, vp, vp, vp, pt, vp]
     L.gdws_forward_host.restype = ci
+    L.gdws_forward_static.argtypes = [vp, pt, vp, vp, vp, pt, vp]
+    L.gdws_forward_static.restype = ci
+    L.gdws_static_scratch_bytes.argtypes = []
+    L.gdws_static_scratch_bytes.restype = ctypes.c_size_t
     L.gdws_status.argtypes = [vp]
     L.gdws_status.restype = ci
     L.gdws_launch_count.argtypes = [vp]
@@ -107,6 +111,10 @@ def last_error() -> str:
 
 def version() -> str:
     return lib().gdws_version().decode()
+
+
+def static_scratch_bytes() -> int:
+    return int(lib().gdws_static_scratch_bytes())
 
 
 def out_dim(size: int, k: int, stride: int, pad: int) -> int:
@@ -242,6 +250,13 @@ class Plan:
         xd, yd = tensor_desc(x_host, layout), tensor_desc(y_host, layout)
         _check(lib().gdws_forward_host(self._h, ctypes.byref(xd), _ptr(dw_w), _ptr(pw_w), _ptr(bias), ctypes.byref(yd),
                                        _stream(stream)))
+
+    def forward_static(self, x, y, layout: str, dw_w=None, pw_w=None, bias=None, stream=None) -> None:
+        """gdws_forward_static: the unfused forward with the intermediate in the library's built-in
+        scratch array; for callers that must not allocate device memory."""
+        xd, yd = tensor_desc(x, layout), tensor_desc(y, layout)
+        _check(lib().gdws_forward_static(self._h, ctypes.byref(xd), _ptr(dw_w), _ptr(pw_w), _ptr(bias),
+                                         ctypes.byref(yd), _stream(stream)))
 
     def status(self) -> None:
         _check(lib().gdws_status(self._h))
