@@ -33,17 +33,27 @@ __global__ void pack_pw_kernel(const void *__restrict__ pw, int is_bf16, int D, 
     }
 }
 
-__global__ void pack_dw_kernel(const void *__restrict__ dw, int is_bf16, int G, int Gpad, int k2,
-                               float *__restrict__ out, uint32_t *__restrict__ out2)
+// dw_w[G][k][k] -> (1) fp32 taps [Gpad][k*k] (zero rows for the padding) for the unfused kernel,
+// (2) [Gpad][wstride] words for the fused kernel: the taps, then the index of the channel inside the
+// slot staged for its K chunk (chan[i] - first channel of chunk i/64).
+__global__ void pack_dw_kernel(const void *__restrict__ dw, int is_bf16, int G, int Gpad, int k2, int wstride,
+                               const int32_t *__restrict__ chan, const int32_t *__restrict__ chunk_c0,
+                               float *__restrict__ out, uint32_t *__restrict__ outp)
 {
-    const int total = Gpad * k2;
+    const int total = Gpad * wstride;
     for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
-        const int i = t / k2;
-        float v = 0.f;
-        if (i < G) v = load_weight(dw, t, is_bf16);
-        const uint32_t b = float_to_bf16_bits(v);
-        out[t] = bf16_bits_to_float((uint16_t)b);
-        out2[t] = b | (b << 16);
+        const int i = t / wstride, j = t - i * wstride;
+        uint32_t word = 0;
+        if (j < k2) {
+            float v = 0.f;
+            if (i < G) v = load_weight(dw, (size_t)i * k2 + j, is_bf16);
+            v = bf16_bits_to_float(float_to_bf16_bits(v));
+            out[(size_t)i * k2 + j] = v;
+            word = __float_as_uint(v);
+        } else if (j == k2 && i < G) {
+            word = (uint32_t)(chan[i] - chunk_c0[i / kChunk]);
+        }
+        outp[t] = word;
     }
 }
 
@@ -62,8 +72,9 @@ gdws_status_t bf16_pack(gdws_plan_s *p, const void *dw_w, const void *pw_w, cons
     int blocks = (int)((tot_pw + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
     pack_pw_kernel<<<blocks, 256, 0, st>>>(pw_w, is_bf16, p->D, p->Dpad, p->G, p->nchunks, p->d_pw_img);
-    int blocks2 = (p->Gpad * k2 + 255) / 256;
-    pack_dw_kernel<<<blocks2, 256, 0, st>>>(dw_w, is_bf16, p->G, p->Gpad, k2, p->d_dw, p->d_dw2);
+    int blocks2 = (p->Gpad * p->wstride + 255) / 256;
+    pack_dw_kernel<<<blocks2, 256, 0, st>>>(dw_w, is_bf16, p->G, p->Gpad, k2, p->wstride, p->d_chan, p->d_chunk_c0,
+                                            p->d_dw, p->d_dwpack);
     pack_bias_kernel<<<(p->Dpad + 255) / 256, 256, 0, st>>>(bias, p->D, p->Dpad, p->d_bias);
     p->launches += 3;
     cudaError_t e = cudaGetLastError();

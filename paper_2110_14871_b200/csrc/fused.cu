@@ -13,8 +13,8 @@
 //     tile's pixels; it keeps its k x k filter in registers, slides down the patch reusing each
 //     input row for up to k output rows, and writes bf16 results as 16-byte pieces into a
 //     pixel-contiguous (MN-major), 128-byte-swizzled tensor-core operand stage;
-//   * 1 control warp: one lane streams the pre-swizzled pointwise weights (bulk copies with
-//     mbarrier completion, a ring of units of at most 256 output channels x 64) and issues
+//   * 2 control threads: one streams the pre-swizzled pointwise weights (bulk copies with mbarrier
+//     completion, a ring of units of at most 256 output channels x 64), the other issues
 //     tcgen05.mma into a TMEM accumulator (128 lanes x D fp32 columns; two accumulators when
 //     D <= 256, so that a tile's epilogue overlaps the next tile's main loop);
 //   * 4 epilogue warps: read the finished accumulator (tcgen05.ld), add the bias, apply the
@@ -28,8 +28,7 @@ namespace gdws {
 struct FusedParams {
     const uint16_t *x;
     uint16_t *y;
-    const float *dw;
-    const uint32_t *dw2;
+    const uint32_t *dwpack;
     const uint16_t *pw_img;
     const float *bias;
     const int32_t *chan;
@@ -37,13 +36,13 @@ struct FusedParams {
     int *status;
     int N, H, W, C, Ho, Wo, D, Dpad, G, nchunks, stride, pad, relu;
     int TN, PH, PW, tiles_h, tiles_w, ntiles;
-    int IH, IW, IWp, plane, span, nslots, nsb;
+    int IH, IW, IWp, plane, span, nslots, nsb, wstride;
     int nhalf, unit_bytes, nacc, acc_cols;
     int a_kmajor, dw_math;
 };
 
 // Warp roles, in warpgroups of 4 so that registers can be moved between the roles (setmaxnreg):
-// warps 0-7 depthwise, 8-15 staging, 16 control (17-19 idle), 20-23 epilogue.
+// warps 0-7 depthwise, 8-15 staging, 16 MMA issue, 17 weight loader (18-19 idle), 20-23 epilogue.
 constexpr int kDwWarps = 8, kStageWarps = 8, kEpiWarps = 4;
 constexpr int kDwThreads = kDwWarps * 32;
 constexpr int kCtrlWarp = kDwWarps + kStageWarps;
@@ -56,6 +55,18 @@ constexpr int kRegsLaunch = 80, kRegsDw = 112, kRegsStage = 80, kRegsCtrl = 40, 
 static_assert(kDwThreads * kRegsDw + kStageWarps * 32 * kRegsStage + 128 * kRegsCtrl + kEpiWarps * 32 * kRegsEpi <=
                   kFusedThreads * kRegsLaunch,
               "register split exceeds the block's allocation: setmaxnreg.inc would wait forever");
+
+// Barrier traffic is per warp, not per thread: one lane waits or arrives for its warp.
+__device__ __forceinline__ void warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+{
+    if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, abort_flag, status, code);
+    __syncwarp();
+}
+__device__ __forceinline__ void warp_arrive(uint32_t bar)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
 
 template <int N> __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -210,7 +221,7 @@ __device__ __forceinline__ void dw_quads_k3(const FusedParams &P, uint32_t xs, i
 
 // ---- depthwise, any k and stride: one pixel group at a time, 2-byte loads.
 template <int K>
-__device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, int cl, const float *__restrict__ wp, int kk,
+__device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, int cl, uint32_t wsm, int kk,
                                            int run, bool live_i, uint32_t a_stage)
 {
     const int hw = P.PH * P.PW;
@@ -236,7 +247,8 @@ __device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, in
                 for (int u = 0; u < K; ++u)
 #pragma unroll
                     for (int v = 0; v < K; ++v)
-                        acc = fmaf(__ldg(wp + u * K + v), bf16_bits_to_float(lds16(xp + (uint32_t)(u * P.IWp + v) * 2)), acc);
+                        acc = fmaf(__uint_as_float(lds32(wsm + (uint32_t)(u * K + v) * 4)),
+                                   bf16_bits_to_float(lds16(xp + (uint32_t)(u * P.IWp + v) * 2)), acc);
                 out[e] = acc;
             }
         }
@@ -258,26 +270,26 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const uint32_t a_s = smem_u32(base);
     const uint32_t b_s = a_s + 2 * 16384;
     const uint32_t x_s = b_s + (uint32_t)P.nsb * P.unit_bytes;
-    const uint32_t slot_bytes = (uint32_t)P.span * P.plane * 2;
+    const uint32_t xplanes_bytes = (uint32_t)P.span * P.plane * 2;       // a slot: channel planes, then the chunk's filters
+    const uint32_t slot_bytes = xplanes_bytes + (uint32_t)kChunk * P.wstride * 4;
     const uint32_t bar_afull = smem_u32(&bars[0]), bar_afree = smem_u32(&bars[2]);
     const uint32_t bar_bfull = smem_u32(&bars[4]), bar_bfree = smem_u32(&bars[4 + kMaxBUnits]);
     const uint32_t bar_xfull = smem_u32(&bars[4 + 2 * kMaxBUnits]);
     const uint32_t bar_xfree = smem_u32(&bars[4 + 2 * kMaxBUnits + kMaxSlots]);
     const uint32_t bar_accfull = smem_u32(&bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots]);
     const uint32_t bar_accfree = bar_accfull + 16;
-    const int wps = kStageWarps / P.nslots;               // staging warps that share one slot
     const int npair = (P.TN * P.IH * P.IWp) >> 1;
 
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_afull + 8 * i, kDwThreads);
+            mbar_init(bar_afull + 8 * i, kDwWarps);
             mbar_init(bar_afree + 8 * i, 1);
             mbar_init(bar_accfull + 8 * i, 1);
-            mbar_init(bar_accfree + 8 * i, kEpiWarps * 32);
+            mbar_init(bar_accfree + 8 * i, kEpiWarps);
         }
         for (int i = 0; i < kMaxBUnits; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
-        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(bar_xfull + 8 * i, 32 * wps); mbar_init(bar_xfree + 8 * i, kDwThreads); }
+        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(bar_xfull + 8 * i, kStageWarps); mbar_init(bar_xfree + 8 * i, kDwWarps); }
         fence_mbar_init();
     }
     if (warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
@@ -292,6 +304,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int ih = r % P.IH, tn = r / P.IH;
         pix_tab[pp] = make_int2((tn * P.H + ih) * P.W + iw, tn | (ih << 8) | (iw << 16));
     }
+    // Channel range [c0, c1] read by every K chunk.
+    int2 *chunk_rng = pix_tab + npair;
+    for (int q = tid; q < P.nchunks; q += kFusedThreads) {
+        const int c0 = __ldg(P.chunk_c0 + q);
+        const int ilast = min(P.G, (q + 1) * kChunk) - 1;
+        chunk_rng[q] = make_int2(c0, q * kChunk < P.G ? __ldg(P.chan + ilast) : c0);
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -302,58 +321,58 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const int tiles_hw = P.tiles_h * P.tiles_w;
 
     if (warp >= kCtrlWarp && warp < kEpiWarp0) {
-        // ---------------- control warp: weight copies and MMA issue (one lane) ----------------
         regs_dec<kRegsCtrl>();
+        const int units_per_tile = P.nchunks * P.nhalf;
+        const int total_units = my_tiles * units_per_tile;
+        const int rows0 = P.Dpad > 256 ? 256 : P.Dpad, rows1 = P.Dpad - rows0;
         if (warp == kCtrlWarp && lane == 0) {
-            const int units_per_tile = P.nchunks * P.nhalf;
-            const int total_units = my_tiles * units_per_tile;
-            const int rows0 = P.Dpad > 256 ? 256 : P.Dpad, rows1 = P.Dpad - rows0;
-            int cu = 0;                                   // next weight unit to copy
-            auto issue_copy = [&](int u) {
-                const int within = u % units_per_tile;
-                const int q = within / P.nhalf, h = within - q * P.nhalf;
-                const int sb = u % P.nsb;
-                const uint32_t bytes = (uint32_t)(h ? rows1 : rows0) * 128u;
-                mbar_expect_tx(bar_bfull + 8 * sb, bytes);
-                bulk_g2s(b_s + sb * P.unit_bytes, P.pw_img + ((size_t)q * P.Dpad + h * 256) * kChunk, bytes,
-                         bar_bfull + 8 * sb);
-            };
-            while (cu < total_units && cu < P.nsb) issue_copy(cu++);
-            int gq = 0, gu = 0;
+            // ---------------- MMA issue (one thread) ----------------
+            const bool a_mn = !P.a_kmajor;
+            const uint64_t adesc0 = a_mn ? make_sdesc(a_s, 1024, 2048) : make_sdesc(a_s, 16, 1024);
+            const uint64_t bdesc0 = make_sdesc(b_s, 16, 1024);
+            const uint32_t a_step = a_mn ? (4096u >> 4) : (32u >> 4);     // descriptor advance per K step of 16
+            const uint32_t idesc0 = make_idesc(rows0, a_mn), idesc1 = make_idesc(rows1 > 0 ? rows1 : 16, a_mn);
+            uint32_t sa = 0, pa = 0;          // intermediate-tile stage and its phase parity
+            uint32_t sb = 0, pb = 0;          // weight-ring slot and its phase parity
             for (int tl = 0; tl < my_tiles; ++tl) {
                 const int buf = tl % P.nacc;
                 if (tl >= P.nacc)
                     mbar_wait(bar_accfree + 8 * buf, ((tl / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
                 tc_fence_after();
-                for (int q = 0; q < P.nchunks; ++q, ++gq) {
-                    const int sa = gq & 1;
-                    mbar_wait(bar_afull + 8 * sa, (gq >> 1) & 1, &abort_flag, P.status, kStatusWaitOperand);
-                    for (int h = 0; h < P.nhalf; ++h, ++gu) {
-                        const int sb = gu % P.nsb;
-                        mbar_wait(bar_bfull + 8 * sb, (gu / P.nsb) & 1, &abort_flag, P.status, kStatusWaitOperand);
+                for (int q = 0; q < P.nchunks; ++q) {
+                    mbar_wait(bar_afull + 8 * sa, pa, &abort_flag, P.status, kStatusWaitOperand);
+                    const uint64_t adesc = adesc0 + (uint64_t)(sa * (16384u >> 4));
+                    for (int h = 0; h < P.nhalf; ++h) {
+                        mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
                         tc_fence_after();
                         const uint32_t d_tmem = tmem + (uint32_t)(buf * P.acc_cols + h * 256);
-                        const uint32_t a_addr = a_s + sa * 16384, b_addr = b_s + sb * P.unit_bytes;
-                        const uint32_t idesc = make_idesc(h ? rows1 : rows0, !P.a_kmajor);
+                        const uint64_t bdesc = bdesc0 + (uint64_t)(sb * ((uint32_t)P.unit_bytes >> 4));
+                        const uint32_t idesc = h ? idesc1 : idesc0;
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {
-                            const uint64_t adesc = !P.a_kmajor ? make_sdesc(a_addr + ks * 4096, 1024, 2048)
-                                                               : make_sdesc(a_addr + ks * 32, 16, 1024);
-                            umma_bf16(d_tmem, adesc, make_sdesc(b_addr + ks * 32, 16, 1024), idesc,
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_bf16(d_tmem, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * 2), idesc,
                                       (q == 0 && ks == 0) ? 0u : 1u);
-                        }
                         umma_commit(bar_bfree + 8 * sb);
-                        // refill the ring: unit cu reuses the slot of unit cu - nsb, whose MMAs were
-                        // issued at least one unit ago
-                        while (cu < total_units && cu <= gu + P.nsb - 1) {
-                            mbar_wait(bar_bfree + 8 * (cu % P.nsb), ((cu / P.nsb) - 1) & 1, &abort_flag, P.status,
-                                      kStatusWaitStage);
-                            issue_copy(cu++);
-                        }
+                        if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
                     }
                     umma_commit(bar_afree + 8 * sa);
+                    sa ^= 1;
+                    if (sa == 0) pa ^= 1;
                 }
                 umma_commit(bar_accfull + 8 * buf);
+            }
+        } else if (warp == kCtrlWarp + 1 && lane == 0) {
+            // ---------------- pointwise-weight loader (one thread): ring of nsb units ----------------
+            uint32_t sb = 0, pb = 1;          // parity of the "slot free" phase awaited (first round: nothing to wait for)
+            int q = 0, h = 0;
+            for (int u = 0; u < total_units; ++u) {
+                if (u >= P.nsb) mbar_wait(bar_bfree + 8 * sb, pb, &abort_flag, P.status, kStatusWaitStage);
+                const uint32_t bytes = (uint32_t)(h ? rows1 : rows0) * 128u;
+                mbar_expect_tx(bar_bfull + 8 * sb, bytes);
+                bulk_g2s(b_s + sb * P.unit_bytes, P.pw_img + ((size_t)q * P.Dpad + h * 256) * kChunk, bytes,
+                         bar_bfull + 8 * sb);
+                if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
+                if (++h == P.nhalf) { h = 0; if (++q == P.nchunks) q = 0; }
             }
         }
     } else if (warp >= kEpiWarp0) {
@@ -374,7 +393,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
             uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D;
             const int buf = tl % P.nacc;
-            mbar_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
+            warp_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
             tc_fence_after();
             const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * P.acc_cols);
             for (int d0 = 0; d0 < P.Dpad; d0 += 16) {
@@ -384,128 +403,163 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 if (live) store_row16(acc, P.bias, d0, P.D, P.relu, yrow);
             }
             tc_fence_before();
-            mbar_arrive(bar_accfree + 8 * buf);
+            warp_arrive(bar_accfree + 8 * buf);
         }
     } else if (warp >= kDwWarps) {
-        // ---------------- staging warps: slot s is filled by the warps w with w % nslots == s ----------------
+        // ---------------- staging warps: all 8 work on every chunk, software-pipelined ----------------
+        // A chunk is staged in rounds of 256 x kSet pixel pairs (one channel group of 8 each).  The loads of
+        // round e+1 are issued before the stores of round e, also across chunk and tile boundaries, so the
+        // global-memory latency is overlapped with the shared-memory scatter of the previous round.
         if (kRegsStage < kRegsLaunch) regs_dec<kRegsStage>();
-        const int sw = warp - kDwWarps;
-        const int slot = sw % P.nslots, share = sw / P.nslots;
-        const uint32_t xs = x_s + slot * slot_bytes;
-        for (int gq = slot; gq < total_chunks; gq += P.nslots) {
-            const int tl = gq / P.nchunks, q = gq - tl * P.nchunks;
+        const int st = tid - kDwThreads;                       // 0..255
+        constexpr int kSet = 3;                                // pixel pairs per thread and round (6 loads)
+        struct ChunkInfo {
+            int gq, q, n0, hi0, wi0, c0, gr0, items, rounds;
+            long long pbase;
+        };
+        auto chunk_info = [&](int gq, ChunkInfo &ci) {
+            ci.gq = gq;
+            const int tl = gq / P.nchunks;
+            ci.q = gq - tl * P.nchunks;
             int tile = (int)blockIdx.x + tl * (int)gridDim.x;
             const int bn = tile / tiles_hw;
             tile -= bn * tiles_hw;
             const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
-            const int n0 = bn * P.TN, hi0 = bh * P.PH * P.stride - P.pad, wi0 = bw * P.PW * P.stride - P.pad;
-            const long long pbase = ((long long)n0 * P.H + hi0) * P.W + wi0;
-            const int use = gq / P.nslots;
-            if (use >= 1) mbar_wait(bar_xfree + 8 * slot, (use - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
-            const int c0 = __ldg(P.chunk_c0 + q);
-            const int ilast = min(P.G, (q + 1) * kChunk) - 1;
-            const int c1 = q * kChunk < P.G ? __ldg(P.chan + ilast) : c0;       // last channel of the chunk
-            const int gr0 = c0 >> 3, ngr = (c1 >> 3) - gr0 + 1;
-            const int items = ngr * npair;                    // (channel group, pixel pair), pixel pair fastest
-            constexpr int kBatch = 4;                         // pixel pairs per lane in flight (8 loads)
-            for (int t0 = share * 32 * kBatch + lane; t0 < items; t0 += 32 * kBatch * wps) {
-                uint4 va[kBatch], vb[kBatch];
+            ci.n0 = bn * P.TN;
+            ci.hi0 = bh * P.PH * P.stride - P.pad;
+            ci.wi0 = bw * P.PW * P.stride - P.pad;
+            ci.pbase = ((long long)ci.n0 * P.H + ci.hi0) * P.W + ci.wi0;
+            const int2 rng = chunk_rng[ci.q];
+            ci.c0 = rng.x;
+            ci.gr0 = rng.x >> 3;
+            ci.items = ((rng.y >> 3) - ci.gr0 + 1) * npair;    // (channel group, pixel pair), pixel pair fastest
+            ci.rounds = (ci.items + kStageWarps * 32 * kSet - 1) / (kStageWarps * 32 * kSet);
+        };
+        uint4 va[2][kSet], vb[2][kSet];
+        auto load_round = [&](const ChunkInfo &ci, int r, int set) {
 #pragma unroll
-                for (int m = 0; m < kBatch; ++m) {
-                    const int t = t0 + m * 32;
-                    va[m] = make_uint4(0, 0, 0, 0);
-                    vb[m] = make_uint4(0, 0, 0, 0);
-                    if (t < items) {
-                        const int gr = t / npair, pp = t - gr * npair;
-                        const int2 e = pix_tab[pp];
-                        const int tn = e.y & 0xff, ih = (e.y >> 8) & 0xff, iw = e.y >> 16;
-                        const int hi = hi0 + ih, wi = wi0 + iw;
-                        const bool rowok = n0 + tn < P.N && hi >= 0 && hi < P.H;
-                        const uint16_t *xp = P.x + (pbase + e.x) * P.C + (gr0 + gr) * 8;
-                        if (rowok && wi >= 0 && wi < P.W && iw < P.IW) va[m] = __ldg(reinterpret_cast<const uint4 *>(xp));
-                        if (rowok && wi + 1 >= 0 && wi + 1 < P.W && iw + 1 < P.IW)
-                            vb[m] = __ldg(reinterpret_cast<const uint4 *>(xp + P.C));
-                    }
+            for (int m = 0; m < kSet; ++m) {
+                const int t = (r * kSet + m) * (kStageWarps * 32) + st;
+                va[set][m] = make_uint4(0, 0, 0, 0);
+                vb[set][m] = make_uint4(0, 0, 0, 0);
+                if (t < ci.items) {
+                    const int gr = t / npair, pp = t - gr * npair;
+                    const int2 e = pix_tab[pp];
+                    const int tn = e.y & 0xff, ih = (e.y >> 8) & 0xff, iw = e.y >> 16;
+                    const int hi = ci.hi0 + ih, wi = ci.wi0 + iw;
+                    const bool rowok = ci.n0 + tn < P.N && hi >= 0 && hi < P.H;
+                    const uint16_t *xp = P.x + (ci.pbase + e.x) * P.C + (ci.gr0 + gr) * 8;
+                    if (rowok && wi >= 0 && wi < P.W && iw < P.IW) va[set][m] = __ldg(reinterpret_cast<const uint4 *>(xp));
+                    if (rowok && wi + 1 >= 0 && wi + 1 < P.W && iw + 1 < P.IW)
+                        vb[set][m] = __ldg(reinterpret_cast<const uint4 *>(xp + P.C));
                 }
+            }
+        };
+        auto store_round = [&](const ChunkInfo &ci, int r, int set, uint32_t xs) {
 #pragma unroll
-                for (int m = 0; m < kBatch; ++m) {
-                    const int t = t0 + m * 32;
-                    if (t < items) {
-                        const int gr = t / npair, pp = t - gr * npair;
-                        const int cb = (gr0 + gr) * 8 - c0;   // slot channel of the group's first channel
-                        const bool whole = cb >= 0 && cb + 8 <= P.span;
-                        const uint32_t a4[4] = {va[m].x, va[m].y, va[m].z, va[m].w};
-                        const uint32_t b4[4] = {vb[m].x, vb[m].y, vb[m].z, vb[m].w};
-                        const uint32_t dst = xs + (uint32_t)(cb * P.plane + 2 * pp) * 2;
+            for (int m = 0; m < kSet; ++m) {
+                const int t = (r * kSet + m) * (kStageWarps * 32) + st;
+                if (t < ci.items) {
+                    const int gr = t / npair, pp = t - gr * npair;
+                    const int cb = (ci.gr0 + gr) * 8 - ci.c0;   // slot channel of the group's first channel
+                    const bool whole = cb >= 0 && cb + 8 <= P.span;
+                    const uint32_t a4[4] = {va[set][m].x, va[set][m].y, va[set][m].z, va[set][m].w};
+                    const uint32_t b4[4] = {vb[set][m].x, vb[set][m].y, vb[set][m].z, vb[set][m].w};
+                    const uint32_t dst = xs + (uint32_t)(cb * P.plane + 2 * pp) * 2;
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            // channel cb+e of the two pixels -> one 32-bit store
-                            const uint32_t word = (e & 1) ? __byte_perm(a4[e >> 1], b4[e >> 1], 0x7632)
-                                                          : __byte_perm(a4[e >> 1], b4[e >> 1], 0x5410);
-                            if (whole || (cb + e >= 0 && cb + e < P.span))
-                                sts32(dst + (uint32_t)(e * P.plane * 2), word);
-                        }
+                    for (int e = 0; e < 8; ++e) {
+                        // channel cb+e of the two pixels -> one 32-bit store
+                        const uint32_t word = (e & 1) ? __byte_perm(a4[e >> 1], b4[e >> 1], 0x7632)
+                                                      : __byte_perm(a4[e >> 1], b4[e >> 1], 0x5410);
+                        if (whole || (cb + e >= 0 && cb + e < P.span)) sts32(dst + (uint32_t)(e * P.plane * 2), word);
                     }
                 }
             }
-            mbar_arrive(bar_xfull + 8 * slot);
-            // first chunk of a tile: pull the next tile's input patch towards L2
-            if (q == 0 && share == 0 && tl + 1 < my_tiles) {
-                int nt = (int)blockIdx.x + (tl + 1) * (int)gridDim.x;
-                const int nbn = nt / tiles_hw;
-                nt -= nbn * tiles_hw;
-                const int nbh = nt / P.tiles_w, nbw = nt - nbh * P.tiles_w;
-                const int nn0 = nbn * P.TN, nhi0 = nbh * P.PH * P.stride - P.pad, nwi0 = nbw * P.PW * P.stride - P.pad;
-                const long long nbase = ((long long)nn0 * P.H + nhi0) * P.W + nwi0;
-                for (int pp = lane; pp < npair; pp += 32) {
-                    const int2 e = pix_tab[pp];
-                    const int tn = e.y & 0xff, ih = (e.y >> 8) & 0xff, iw = e.y >> 16;
-                    const int hi = nhi0 + ih, wi = nwi0 + iw;
-                    if (nn0 + tn < P.N && hi >= 0 && hi < P.H && wi >= 0 && wi + 1 < P.W && iw + 1 < P.IW) {
-                        const char *px = reinterpret_cast<const char *>(P.x + (nbase + e.x) * P.C);
-                        for (int b = 0; b < P.C * 4; b += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(px + b));
+        };
+        if (total_chunks > 0) {
+            ChunkInfo LC, SC;
+            chunk_info(0, LC);
+            SC = LC;
+            int lr = 0, sr = 0, set = 0;
+            load_round(LC, 0, 0);
+            while (true) {
+                // advance the load cursor and issue its loads into the other register set
+                bool more = true;
+                if (++lr == LC.rounds) {
+                    lr = 0;
+                    if (LC.gq + 1 < total_chunks) chunk_info(LC.gq + 1, LC);
+                    else more = false;
+                }
+                if (more) {
+                    if (set == 0) load_round(LC, lr, 1);
+                    else load_round(LC, lr, 0);
+                    if (lr == 0 && LC.q == 0 && warp == kDwWarps + 1) {
+                        // first chunk of a tile: pull the rest of that tile's input patch towards L2
+                        for (int pp = lane; pp < npair; pp += 32) {
+                            const int2 e = pix_tab[pp];
+                            const int tn = e.y & 0xff, ih = (e.y >> 8) & 0xff, iw = e.y >> 16;
+                            const int hi = LC.hi0 + ih, wi = LC.wi0 + iw;
+                            if (LC.n0 + tn < P.N && hi >= 0 && hi < P.H && wi >= 0 && wi + 1 < P.W && iw + 1 < P.IW) {
+                                const char *px = reinterpret_cast<const char *>(P.x + (LC.pbase + e.x) * P.C);
+                                for (int bb = 0; bb < P.C * 4; bb += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(px + bb));
+                            }
+                        }
                     }
                 }
+                // store the round loaded one step earlier
+                const int slot = SC.gq % P.nslots;
+                const uint32_t xs = x_s + slot * slot_bytes;
+                if (sr == 0) {
+                    const int use = SC.gq / P.nslots;
+                    if (use >= 1) warp_wait(bar_xfree + 8 * slot, (use - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                    if (st == 0) {   // the chunk's filters and slot-channel indices: one bulk copy, counted by the slot's barrier
+                        const uint32_t wbytes = (uint32_t)kChunk * P.wstride * 4;
+                        mbar_expect_tx_only(bar_xfull + 8 * slot, wbytes);
+                        bulk_g2s(xs + xplanes_bytes, P.dwpack + (size_t)SC.q * kChunk * P.wstride, wbytes, bar_xfull + 8 * slot);
+                    }
+                }
+                if (set == 0) store_round(SC, sr, 0, xs);
+                else store_round(SC, sr, 1, xs);
+                if (++sr == SC.rounds) {
+                    sr = 0;
+                    warp_arrive(bar_xfull + 8 * slot);
+                    if (SC.gq + 1 >= total_chunks) break;
+                    chunk_info(SC.gq + 1, SC);
+                }
+                set ^= 1;
             }
         }
     } else {
         // ---------------- depthwise warps ----------------
         regs_inc<kRegsDw>();
         const int il = tid & 63, run = tid >> 6;
-        float w[9];
-        int cl = 0;
-        auto load_weights = [&](int q) {
-            const int i = q * kChunk + il;
-            if (MODE != 0) {
-#pragma unroll
-                for (int t = 0; t < 9; ++t) w[t] = __ldg(P.dw + (size_t)i * 9 + t);
-            }
-            const int c = __ldg(P.chan + i);
-            cl = c < 0 ? 0 : c - __ldg(P.chunk_c0 + q);
-        };
-        load_weights(0);
         int q = 0;
         for (int gq = 0; gq < total_chunks; ++gq) {
             const int sa = gq & 1, slot = gq % P.nslots;
-            const int i = q * kChunk + il;
-            const bool live_i = i < P.G;
-            float wq[9];
-#pragma unroll
-            for (int t = 0; t < 9; ++t) wq[t] = w[t];
-            const int clq = cl;
-            const int qn = (q + 1 == P.nchunks) ? 0 : q + 1;
-            if (gq + 1 < total_chunks) load_weights(qn);    // next chunk's filter while this one computes
-            mbar_wait(bar_xfull + 8 * slot, (gq / P.nslots) & 1, &abort_flag, P.status, kStatusWaitOperand);
-            if (gq >= 2) mbar_wait(bar_afree + 8 * sa, ((gq >> 1) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+            const bool live_i = q * kChunk + il < P.G;
+            warp_wait(bar_xfull + 8 * slot, (gq / P.nslots) & 1, &abort_flag, P.status, kStatusWaitOperand);
             const uint32_t xs = x_s + slot * slot_bytes;
+            const uint32_t wsm = xs + xplanes_bytes + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
+            float w[9];
+            int cl;
+            if (MODE != 0) {
+                const uint4 w0 = lds128(wsm), w1 = lds128(wsm + 16), w2 = lds128(wsm + 32);
+                w[0] = __uint_as_float(w0.x); w[1] = __uint_as_float(w0.y); w[2] = __uint_as_float(w0.z);
+                w[3] = __uint_as_float(w0.w); w[4] = __uint_as_float(w1.x); w[5] = __uint_as_float(w1.y);
+                w[6] = __uint_as_float(w1.z); w[7] = __uint_as_float(w1.w); w[8] = __uint_as_float(w2.x);
+                cl = (int)w2.y;
+            } else {
+                cl = (int)lds32(wsm + (uint32_t)(K * K) * 4);
+            }
+            if (gq >= 2) warp_wait(bar_afree + 8 * sa, ((gq >> 1) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
             const uint32_t a_stage = a_s + sa * 16384;
-            if (MODE == 1) dw_rows_k3<S>(P, xs, clq, wq, il, run, live_i, a_stage);
-            else if (MODE == 2) dw_quads_k3<S>(P, xs, clq, wq, il, run, live_i, a_stage);
-            else dw_generic<K>(P, xs, clq, P.dw + (size_t)i * (K * K), il, run, live_i, a_stage);
-            fence_proxy_async();
-            mbar_arrive(bar_afull + 8 * sa);
-            mbar_arrive(bar_xfree + 8 * slot);
-            q = qn;
+            if (MODE == 1) dw_rows_k3<S>(P, xs, cl, w, il, run, live_i, a_stage);
+            else if (MODE == 2) dw_quads_k3<S>(P, xs, cl, w, il, run, live_i, a_stage);
+            else dw_generic<K>(P, xs, cl, wsm, il, run, live_i, a_stage);
+            fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
+            warp_arrive(bar_afull + 8 * sa);
+            warp_arrive(bar_xfree + 8 * slot);
+            q = (q + 1 == P.nchunks) ? 0 : q + 1;
         }
     }
     tc_fence_before();
@@ -545,13 +599,13 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
     }
     FusedParams P;
     P.x = (const uint16_t *)x->ptr; P.y = (uint16_t *)y->ptr;
-    P.dw = p->d_dw; P.dw2 = p->d_dw2; P.pw_img = p->d_pw_img; P.bias = p->d_bias;
+    P.dwpack = p->d_dwpack; P.pw_img = p->d_pw_img; P.bias = p->d_bias;
     P.chan = p->d_chan; P.chunk_c0 = p->d_chunk_c0; P.status = p->d_status;
     P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = y->h; P.Wo = y->w; P.D = p->D; P.Dpad = p->Dpad;
     P.G = p->G; P.nchunks = p->nchunks; P.stride = p->stride; P.pad = p->pad;
     P.relu = p->opt_relu;
     P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
-    P.IH = t.IH; P.IW = t.IW; P.IWp = t.IWp; P.plane = t.plane; P.span = t.span; P.nslots = t.nslots; P.nsb = t.nsb;
+    P.IH = t.IH; P.IW = t.IW; P.IWp = t.IWp; P.plane = t.plane; P.span = t.span; P.nslots = t.nslots; P.nsb = t.nsb; P.wstride = p->wstride;
     P.nhalf = p->Dpad > 256 ? 2 : 1;
     P.unit_bytes = (p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
     P.acc_cols = tmem_cols_for(p->Dpad);

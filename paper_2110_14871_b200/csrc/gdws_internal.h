@@ -41,6 +41,7 @@ struct Tile {
 struct gdws_plan_s {
     int C = 0, D = 0, k = 0, stride = 0, pad = 0;
     int G = 0, Gpad = 0, Dpad = 0, nchunks = 0;
+    int wstride = 0;                 // 32-bit words per intermediate channel in d_dwpack (multiple of 4)
     std::vector<int32_t> g, off, chan;
     std::vector<int32_t> chunk_c0;   // first input channel read by K chunk q (intermediate channels 64q..64q+63)
     int span_max = 0;                // widest channel range of one K chunk
@@ -59,7 +60,7 @@ struct gdws_plan_s {
     int32_t *d_chan = nullptr;     // [Gpad], -1 for padding
     int32_t *d_chunk_c0 = nullptr; // [nchunks]
     float *d_dw = nullptr;         // [Gpad][k*k] fp32 depthwise filters, zero rows for padding
-    uint32_t *d_dw2 = nullptr;     // [Gpad][k*k] the same filters as bf16 pairs (w,w)
+    uint32_t *d_dwpack = nullptr;  // [Gpad][wstride]: k*k fp32 filter taps, then the channel's index within its K chunk's slot
     uint16_t *d_pw_img = nullptr;  // [nchunks][Dpad*64] bf16, 128-byte-swizzled K-major operand images
     float *d_bias = nullptr;       // [Dpad]
     int *d_status = nullptr;       // device status word

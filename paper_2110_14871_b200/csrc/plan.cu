@@ -59,7 +59,7 @@ static void free_device(gdws_plan_s *p)
     cudaFree(p->d_chan);
     cudaFree(p->d_chunk_c0);
     cudaFree(p->d_dw);
-    cudaFree(p->d_dw2);
+    cudaFree(p->d_dwpack);
     cudaFree(p->d_pw_img);
     cudaFree(p->d_bias);
     cudaFree(p->d_status);
@@ -91,7 +91,7 @@ gdws_status_t ensure_device(gdws_plan_s *p)
     GDWS_TRY_ALLOC(p->d_chan, sizeof(int32_t) * p->Gpad);
     GDWS_TRY_ALLOC(p->d_chunk_c0, sizeof(int32_t) * p->nchunks);
     GDWS_TRY_ALLOC(p->d_dw, sizeof(float) * p->Gpad * k2);
-    GDWS_TRY_ALLOC(p->d_dw2, sizeof(uint32_t) * p->Gpad * k2);
+    GDWS_TRY_ALLOC(p->d_dwpack, sizeof(uint32_t) * p->Gpad * p->wstride);
     GDWS_TRY_ALLOC(p->d_pw_img, img);
     GDWS_TRY_ALLOC(p->d_bias, sizeof(float) * p->Dpad);
     GDWS_TRY_ALLOC(p->d_status, sizeof(int));
@@ -121,8 +121,9 @@ static bool fit_smem(const gdws_plan_s *p, Tile &t)
     const size_t a = 2 * (size_t)kTileRows * kChunk * 2;
     const int nhalf = p->Dpad > 256 ? 2 : 1;
     const size_t unit = (size_t)(p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
-    const size_t slot = (size_t)t.span * t.plane * 2;
-    const size_t fixed = a + 1024 /*alignment slack*/ + (size_t)t.TN * t.IH * t.IWp * 4 /*patch table*/;
+    const size_t slot = (size_t)t.span * t.plane * 2 + (size_t)kChunk * p->wstride * 4 /*the chunk's filters*/;
+    const size_t fixed = a + 1024 /*alignment slack*/ + (size_t)t.TN * t.IH * t.IWp * 4 /*patch table*/ +
+                         (size_t)p->nchunks * 8 /*channel range of every chunk*/;
     int best_score = -1;
     for (int ns = 2; ns <= 8; ns *= 2) {
         if (fixed + ns * slot + (size_t)(nhalf + 1) * unit > (size_t)kMaxSmem) break;
@@ -225,6 +226,7 @@ gdws_status_t gdws_plan(int C, int D, int k, int stride, int pad, const int32_t 
     p->Gpad = round_up((int)G, kChunk);
     p->Dpad = round_up(D, 16);
     p->nchunks = p->Gpad / kChunk;
+    p->wstride = round_up(k * k + 1, 4);
     try {
         p->g.assign(g, g + C);
         p->off.resize(C + 1);
