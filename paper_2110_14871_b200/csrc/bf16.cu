@@ -35,7 +35,7 @@ __global__ void pack_pw_kernel(const void *__restrict__ pw, int is_bf16, int D, 
 
 // dw_w[G][k][k] -> (1) fp32 taps [Gpad][k*k] (zero rows for the padding) for the unfused kernel,
 // (2) [Gpad][wstride] words for the fused kernel: the taps, then the index of the channel inside the
-// slot staged for its K chunk (chan[i] - first channel of chunk i/64).
+// box staged for its K chunk (chan[i] - first channel of chunk i/64 rounded down to a multiple of 8).
 __global__ void pack_dw_kernel(const void *__restrict__ dw, int is_bf16, int G, int Gpad, int k2, int wstride,
                                const int32_t *__restrict__ chan, const int32_t *__restrict__ chunk_c0,
                                float *__restrict__ out, uint32_t *__restrict__ outp)
@@ -51,7 +51,7 @@ __global__ void pack_dw_kernel(const void *__restrict__ dw, int is_bf16, int G, 
             out[(size_t)i * k2 + j] = v;
             word = __float_as_uint(v);
         } else if (j == k2 && i < G) {
-            word = (uint32_t)(chan[i] - chunk_c0[i / kChunk]);
+            word = (uint32_t)(chan[i] - (chunk_c0[i / kChunk] & ~7));
         }
         outp[t] = word;
     }

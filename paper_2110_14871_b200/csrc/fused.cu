@@ -3,58 +3,62 @@
 //
 // The kernel is persistent: one block per SM walks over tiles of 128 output pixels (TN images x
 // PH x PW patch, all D output channels).  Within a tile the intermediate channels are processed
-// in K chunks of 64 (i = 64q .. 64q+63, canonical order i = off_c + j).  Five kinds of warps run
-// as one pipeline over the sequence of (tile, chunk) pairs, coupled only by mbarriers:
-//   * 8 staging warps: chunk q reads the contiguous channel range [c0(q), c0(q)+span); the warps
-//     load those channels of the tile's input patch (with halo, zero filled outside the image)
-//     with 16-byte loads and write them channel-major into one of `nslots` slots, so that the
-//     depthwise stage reads runs of consecutive pixels of one channel with 16-byte loads;
-//   * 8 depthwise warps: thread t owns intermediate channel 64q + (t & 63) and a quarter of the
-//     tile's pixels; it keeps its k x k filter in registers, slides down the patch reusing each
-//     input row for up to k output rows, and writes bf16 results as 16-byte pieces into a
-//     pixel-contiguous (MN-major), 128-byte-swizzled tensor-core operand stage;
-//   * 2 control threads: one streams the pre-swizzled pointwise weights (bulk copies with mbarrier
-//     completion, a ring of units of at most 256 output channels x 64), the other issues
-//     tcgen05.mma into a TMEM accumulator (128 lanes x D fp32 columns; two accumulators when
-//     D <= 256, so that a tile's epilogue overlaps the next tile's main loop);
+// in K chunks of 64 (i = 64q .. 64q+63, canonical order i = off_c + j).  The warps form one
+// pipeline over the sequence of (tile, chunk) pairs, coupled only by mbarriers:
+//   * input loader (one thread): chunk q reads a contiguous range of input channels; one TMA
+//     tiled load (x seen as a rank-4 tensor C x W x H x N, box = channels x patch with halo,
+//     out-of-image positions filled with zeros) brings those channels of the tile's input patch
+//     into one of `nslots` shared-memory slots, and one bulk copy adds the chunk's 64 filters;
+//   * 16 depthwise warps in two groups that take alternate chunks: thread t of a group owns
+//     intermediate channel 64q + (t & 63) and a quarter of the tile's pixels; it keeps its k x k
+//     filter in registers, slides down the patch reusing each input row for up to k output rows,
+//     and writes bf16 results as 16-byte pieces into the group's pixel-contiguous (MN-major),
+//     128-byte-swizzled tensor-core operand stage;
+//   * weight loader (one thread): streams the pre-swizzled pointwise weights (bulk copies with
+//     mbarrier completion, a ring of units of at most 256 output channels x 64);
+//   * MMA issuer (one thread): tcgen05.mma into a TMEM accumulator (128 lanes x D fp32 columns;
+//     two accumulators when D <= 256, so that a tile's epilogue overlaps the next tile's main loop);
 //   * 4 epilogue warps: read the finished accumulator (tcgen05.ld), add the bias, apply the
 //     optional ReLU, round to bf16 and store y.
 // Every wait is bounded; a wait that runs out raises a block-wide abort flag that turns all later
 // waits into no-ops, so the block still reaches its teardown, frees TMEM and ends.
+#include <cuda.h>
+
 #include "sm100.cuh"
 
 namespace gdws {
 
-struct FusedParams {
-    const uint16_t *x;
+struct alignas(64) FusedParams {
+    CUtensorMap tmap;            // x as (C, W, H, N) bf16, box (cbox, IW, IH, TN)
     uint16_t *y;
     const uint32_t *dwpack;
     const uint16_t *pw_img;
     const float *bias;
-    const int32_t *chan;
     const int32_t *chunk_c0;
     int *status;
     int N, H, W, C, Ho, Wo, D, Dpad, G, nchunks, stride, pad, relu;
     int TN, PH, PW, tiles_h, tiles_w, ntiles;
-    int IH, IW, IWp, plane, span, nslots, nsb, wstride;
+    int IH, IW, ps, nslots, nsb, wstride;
+    int box_bytes, slot_bytes;
     int nhalf, unit_bytes, nacc, acc_cols;
     int a_kmajor, dw_math;
 };
 
 // Warp roles, in warpgroups of 4 so that registers can be moved between the roles (setmaxnreg):
-// warps 0-7 depthwise, 8-15 staging, 16 MMA issue, 17 weight loader (18-19 idle), 20-23 epilogue.
-constexpr int kDwWarps = 8, kStageWarps = 8, kEpiWarps = 4;
+// warps 0-15 depthwise (two groups of 8), 16 MMA issue, 17 weight loader, 18 input loader
+// (19 idle), 20-23 epilogue.
+constexpr int kDwWarps = 16, kDwGroupWarps = 8, kEpiWarps = 4;
 constexpr int kDwThreads = kDwWarps * 32;
-constexpr int kCtrlWarp = kDwWarps + kStageWarps;
+constexpr int kCtrlWarp = kDwWarps;
 constexpr int kEpiWarp0 = kCtrlWarp + 4;
 constexpr int kFusedThreads = (kEpiWarp0 + kEpiWarps) * 32;
 // Registers per thread after the split.  setmaxnreg.inc can only claim what other warpgroups of the
 // same block released, so the sum must stay within the block's allocation at launch
 // (768 threads x 80 registers, the most that one block of this size can get).
-constexpr int kRegsLaunch = 80, kRegsDw = 112, kRegsStage = 80, kRegsCtrl = 40, kRegsEpi = 56;
-static_assert(kDwThreads * kRegsDw + kStageWarps * 32 * kRegsStage + 128 * kRegsCtrl + kEpiWarps * 32 * kRegsEpi <=
-                  kFusedThreads * kRegsLaunch,
+constexpr int kRegsLaunch = 80, kRegsDw = 96, kRegsCtrl = 40, kRegsEpi = 56;
+static_assert(kDwThreads * kRegsDw + 128 * kRegsCtrl + kEpiWarps * 32 * kRegsEpi <= kFusedThreads * kRegsLaunch,
               "register split exceeds the block's allocation: setmaxnreg.inc would wait forever");
+constexpr int kMaxSlots = 8, kMaxBUnits = 8;
 
 // Barrier traffic is per warp, not per thread: one lane waits or arrives for its warp.
 __device__ __forceinline__ void warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
@@ -70,7 +74,16 @@ __device__ __forceinline__ void warp_arrive(uint32_t bar)
 
 template <int N> __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-constexpr int kMaxSlots = 8, kMaxBUnits = 8;
+
+// TMA tiled load of a rank-4 box; coordinates innermost first.  The innermost coordinate times the
+// element size must be a multiple of 16 bytes (here: a multiple of 8 channels).
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tmap, int c0, int c1, int c2, int c3,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr)
 {
@@ -84,18 +97,13 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
     asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v)
+// One bf16 element of the staged input as fp32.
+__device__ __forceinline__ float lds_bf16(uint32_t addr)
 {
-    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+    uint32_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));
+    return __uint_as_float(v << 16);
 }
-__device__ __forceinline__ uint16_t lds16(uint32_t addr)
-{
-    uint16_t v;
-    asm volatile("ld.shared.b16 %0, [%1];" : "=h"(v) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 // Where the 8 bf16 results of pixel group `o` (rows 8o..8o+7 of the tile) and intermediate
 // channel column kk go in a pixel-contiguous (MN-major) stage: K group kk/8 and 64-row block
@@ -122,10 +130,14 @@ __device__ __forceinline__ void store_group(const FusedParams &P, uint32_t a_sta
     }
 }
 
+// The staged input of a slot is the TMA box as it lies in x: [tn][ih][iw][channel], PS bytes per
+// pixel.  Lanes of a warp read different channels of the same pixel, i.e. one or two 32-byte
+// sectors: a single shared-memory wavefront per load.
+
 // ---- depthwise, k = 3, patches at least 8 wide: a thread computes 4 consecutive output rows of one
-// 8-pixel column group, reading each input row once (16-byte loads) and using it for up to 3 rows.
-template <int S>
-__device__ __forceinline__ void dw_rows_k3(const FusedParams &P, uint32_t xs, int cl, const float (&w)[9], int kk,
+// 8-pixel column group, reading each input row once and using it for up to 3 output rows.
+template <int S, int PS>
+__device__ __forceinline__ void dw_rows_k3(const FusedParams &P, uint32_t xs, int clb, const float (&w)[9], int kk,
                                            int run, bool live_i, uint32_t a_stage)
 {
     const int nseg = P.PW >> 3;
@@ -139,26 +151,15 @@ __device__ __forceinline__ void dw_rows_k3(const FusedParams &P, uint32_t xs, in
         for (int e = 0; e < 8; ++e) acc[ro][e] = 0.f;
     if (live_i && R0 < P.TN * P.PH) {
         const int tn = R0 / P.PH, ph0 = R0 - tn * P.PH;
-        const uint32_t rowb = (uint32_t)P.IWp * 2;
-        const uint32_t base = xs + (uint32_t)(cl * P.plane + (tn * P.IH + ph0 * S) * P.IWp + seg * 8 * S) * 2;
+        const uint32_t rowb = (uint32_t)P.IW * PS;
+        const uint32_t base = xs + (uint32_t)((tn * P.IH + ph0 * S) * P.IW + seg * 8 * S) * PS + (uint32_t)clb * 2;
         constexpr int NR = 3 * S + 3;              // input rows feeding 4 output rows
         constexpr int NX = 7 * S + 3;              // input columns feeding 8 output columns
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
-            float xr[NX + 1];
-            const uint4 a = lds128(base + r * rowb);
-            xr[0] = bf_lo(a.x); xr[1] = bf_hi(a.x); xr[2] = bf_lo(a.y); xr[3] = bf_hi(a.y);
-            xr[4] = bf_lo(a.z); xr[5] = bf_hi(a.z); xr[6] = bf_lo(a.w); xr[7] = bf_hi(a.w);
-            if (S == 1) {
-                const uint32_t b = lds32(base + r * rowb + 16);
-                xr[8] = bf_lo(b); xr[9] = bf_hi(b);
-            } else {
-                const uint4 b = lds128(base + r * rowb + 16);
-                const uint32_t c = lds32(base + r * rowb + 32);
-                xr[8] = bf_lo(b.x); xr[9] = bf_hi(b.x); xr[10] = bf_lo(b.y); xr[11] = bf_hi(b.y);
-                xr[12] = bf_lo(b.z); xr[13] = bf_hi(b.z); xr[14] = bf_lo(b.w); xr[15] = bf_hi(b.w);
-                xr[16] = bf_lo(c);
-            }
+            float xr[NX];
+#pragma unroll
+            for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * rowb + j * PS);
 #pragma unroll
             for (int ro = 0; ro < 4; ++ro) {
                 const int u = r - ro * S;
@@ -176,8 +177,8 @@ __device__ __forceinline__ void dw_rows_k3(const FusedParams &P, uint32_t xs, in
 }
 
 // ---- depthwise, k = 3, 4-wide patches: a pixel group is 2 output rows x 4 columns of one image.
-template <int S>
-__device__ __forceinline__ void dw_quads_k3(const FusedParams &P, uint32_t xs, int cl, const float (&w)[9], int kk,
+template <int S, int PS>
+__device__ __forceinline__ void dw_quads_k3(const FusedParams &P, uint32_t xs, int clb, const float (&w)[9], int kk,
                                             int run, bool live_i, uint32_t a_stage)
 {
     const int gpi = P.PH >> 1;                      // pixel groups per image
@@ -189,19 +190,15 @@ __device__ __forceinline__ void dw_quads_k3(const FusedParams &P, uint32_t xs, i
         for (int e = 0; e < 8; ++e) acc[e] = 0.f;
         const int tn = o / gpi, ph0 = (o - tn * gpi) * 2;
         if (live_i && tn < P.TN) {
-            const uint32_t rowb = (uint32_t)P.IWp * 2;
-            const uint32_t base = xs + (uint32_t)(cl * P.plane + (tn * P.IH + ph0 * S) * P.IWp) * 2;
+            const uint32_t rowb = (uint32_t)P.IW * PS;
+            const uint32_t base = xs + (uint32_t)((tn * P.IH + ph0 * S) * P.IW) * PS + (uint32_t)clb * 2;
             constexpr int NR = S + 3;               // input rows feeding 2 output rows
+            constexpr int NX = 3 * S + 3;           // input columns feeding 4 output columns
 #pragma unroll
             for (int r = 0; r < NR; ++r) {
-                float xr[10];
-                const uint4 a = lds128(base + r * rowb);
-                xr[0] = bf_lo(a.x); xr[1] = bf_hi(a.x); xr[2] = bf_lo(a.y); xr[3] = bf_hi(a.y);
-                xr[4] = bf_lo(a.z); xr[5] = bf_hi(a.z); xr[6] = bf_lo(a.w); xr[7] = bf_hi(a.w);
-                if (S == 2) {
-                    const uint32_t b = lds32(base + r * rowb + 16);
-                    xr[8] = bf_lo(b); xr[9] = bf_hi(b);
-                }
+                float xr[NX];
+#pragma unroll
+                for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * rowb + j * PS);
 #pragma unroll
                 for (int ro = 0; ro < 2; ++ro) {
                     const int u = r - ro * S;
@@ -219,9 +216,9 @@ __device__ __forceinline__ void dw_quads_k3(const FusedParams &P, uint32_t xs, i
     }
 }
 
-// ---- depthwise, any k and stride: one pixel group at a time, 2-byte loads.
+// ---- depthwise, any k and stride: one pixel group at a time.
 template <int K>
-__device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, int cl, uint32_t wsm, int kk,
+__device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, int clb, uint32_t wsm, int kk,
                                            int run, bool live_i, uint32_t a_stage)
 {
     const int hw = P.PH * P.PW;
@@ -236,19 +233,19 @@ __device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, in
         if (live_i && tn < P.TN) {
             const int rem = r0 - tn * hw;
             const int ph = rem / P.PW, pw0 = rem - ph * P.PW;
-            const uint32_t xc = xs + (uint32_t)(cl * P.plane + tn * P.IH * P.IWp) * 2;
+            const uint32_t xc = xs + (uint32_t)(tn * P.IH * P.IW) * P.ps + (uint32_t)clb * 2;
 #pragma unroll 1
             for (int e = 0; e < 8; ++e) {
                 const int phe = (P.PW >= 8) ? ph : ph + (e >> 2);
                 const int pwe = (P.PW >= 8) ? pw0 + e : (e & 3);
-                const uint32_t xp = xc + (uint32_t)(phe * P.stride * P.IWp + pwe * P.stride) * 2;
+                const uint32_t xp = xc + (uint32_t)(phe * P.stride * P.IW + pwe * P.stride) * P.ps;
                 float acc = 0.f;
 #pragma unroll
                 for (int u = 0; u < K; ++u)
 #pragma unroll
                     for (int v = 0; v < K; ++v)
                         acc = fmaf(__uint_as_float(lds32(wsm + (uint32_t)(u * K + v) * 4)),
-                                   bf16_bits_to_float(lds16(xp + (uint32_t)(u * P.IWp + v) * 2)), acc);
+                                   lds_bf16(xp + (uint32_t)(u * P.IW + v) * P.ps), acc);
                 out[e] = acc;
             }
         }
@@ -256,8 +253,9 @@ __device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, in
     }
 }
 
-// MODE: 0 generic, 1 row runs (k=3), 2 4-wide patches (k=3); S = stride for modes 1/2.
-template <int K, int MODE, int S>
+// MODE: 0 generic, 1 row runs (k=3), 2 4-wide patches (k=3); S = stride and PS = bytes per staged
+// pixel for modes 1/2 (mode 0 reads both from the parameters).
+template <int K, int MODE, int S, int PS>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __grid_constant__ FusedParams P)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -270,47 +268,26 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const uint32_t a_s = smem_u32(base);
     const uint32_t b_s = a_s + 2 * 16384;
     const uint32_t x_s = b_s + (uint32_t)P.nsb * P.unit_bytes;
-    const uint32_t xplanes_bytes = (uint32_t)P.span * P.plane * 2;       // a slot: channel planes, then the chunk's filters
-    const uint32_t slot_bytes = xplanes_bytes + (uint32_t)kChunk * P.wstride * 4;
     const uint32_t bar_afull = smem_u32(&bars[0]), bar_afree = smem_u32(&bars[2]);
     const uint32_t bar_bfull = smem_u32(&bars[4]), bar_bfree = smem_u32(&bars[4 + kMaxBUnits]);
     const uint32_t bar_xfull = smem_u32(&bars[4 + 2 * kMaxBUnits]);
     const uint32_t bar_xfree = smem_u32(&bars[4 + 2 * kMaxBUnits + kMaxSlots]);
     const uint32_t bar_accfull = smem_u32(&bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots]);
     const uint32_t bar_accfree = bar_accfull + 16;
-    const int npair = (P.TN * P.IH * P.IWp) >> 1;
 
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_afull + 8 * i, kDwWarps);
+            mbar_init(bar_afull + 8 * i, kDwGroupWarps);
             mbar_init(bar_afree + 8 * i, 1);
             mbar_init(bar_accfull + 8 * i, 1);
             mbar_init(bar_accfree + 8 * i, kEpiWarps);
         }
         for (int i = 0; i < kMaxBUnits; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
-        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(bar_xfull + 8 * i, kStageWarps); mbar_init(bar_xfree + 8 * i, kDwWarps); }
+        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(bar_xfull + 8 * i, 1); mbar_init(bar_xfree + 8 * i, kDwGroupWarps); }
         fence_mbar_init();
     }
     if (warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
-
-    // Patch table (the same for every tile): for each pair of horizontally adjacent patch positions
-    // the pixel offset (tn*H + ih)*W + iw relative to the tile's first input pixel, and tn, ih, iw.
-    int2 *pix_tab = reinterpret_cast<int2 *>(base + (x_s - a_s) + (size_t)P.nslots * slot_bytes);
-    for (int pp = tid; pp < npair; pp += kFusedThreads) {
-        const int t = 2 * pp;
-        const int iw = t % P.IWp;
-        const int r = t / P.IWp;
-        const int ih = r % P.IH, tn = r / P.IH;
-        pix_tab[pp] = make_int2((tn * P.H + ih) * P.W + iw, tn | (ih << 8) | (iw << 16));
-    }
-    // Channel range [c0, c1] read by every K chunk.
-    int2 *chunk_rng = pix_tab + npair;
-    for (int q = tid; q < P.nchunks; q += kFusedThreads) {
-        const int c0 = __ldg(P.chunk_c0 + q);
-        const int ilast = min(P.G, (q + 1) * kChunk) - 1;
-        chunk_rng[q] = make_int2(c0, q * kChunk < P.G ? __ldg(P.chan + ilast) : c0);
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -374,6 +351,28 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
                 if (++h == P.nhalf) { h = 0; if (++q == P.nchunks) q = 0; }
             }
+        } else if (warp == kCtrlWarp + 2 && lane == 0) {
+            // ---------------- input loader (one thread): ring of nslots slots ----------------
+            const uint32_t wbytes = (uint32_t)kChunk * P.wstride * 4;
+            uint32_t slot = 0, px = 1;        // parity of the "slot free" phase awaited
+            int gq = 0;
+            for (int tl = 0; tl < my_tiles; ++tl) {
+                int tile = (int)blockIdx.x + tl * (int)gridDim.x;
+                const int bn = tile / tiles_hw;
+                tile -= bn * tiles_hw;
+                const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+                const int n0 = bn * P.TN, hi0 = bh * P.PH * P.stride - P.pad, wi0 = bw * P.PW * P.stride - P.pad;
+                for (int q = 0; q < P.nchunks; ++q, ++gq) {
+                    if (gq >= P.nslots) mbar_wait(bar_xfree + 8 * slot, px, &abort_flag, P.status, kStatusWaitStage);
+                    const uint32_t xs = x_s + slot * (uint32_t)P.slot_bytes;
+                    const int cbase = __ldg(P.chunk_c0 + q) & ~7;          // first channel of the box (16-byte aligned)
+                    mbar_expect_tx(bar_xfull + 8 * slot, (uint32_t)P.box_bytes + wbytes);
+                    tma_load_4d(xs, &P.tmap, cbase, wi0, hi0, n0, bar_xfull + 8 * slot);
+                    bulk_g2s(xs + (uint32_t)P.box_bytes, P.dwpack + (size_t)q * kChunk * P.wstride, wbytes,
+                             bar_xfull + 8 * slot);
+                    if (++slot == (uint32_t)P.nslots) { slot = 0; px ^= 1; }
+                }
+            }
         }
     } else if (warp >= kEpiWarp0) {
         // ---------------- epilogue warps: TMEM -> registers -> bias / ReLU -> bf16 -> global ----------------
@@ -405,161 +404,39 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             tc_fence_before();
             warp_arrive(bar_accfree + 8 * buf);
         }
-    } else if (warp >= kDwWarps) {
-        // ---------------- staging warps: all 8 work on every chunk, software-pipelined ----------------
-        // A chunk is staged in rounds of 256 x kSet pixel pairs (one channel group of 8 each).  The loads of
-        // round e+1 are issued before the stores of round e, also across chunk and tile boundaries, so the
-        // global-memory latency is overlapped with the shared-memory scatter of the previous round.
-        if (kRegsStage < kRegsLaunch) regs_dec<kRegsStage>();
-        const int st = tid - kDwThreads;                       // 0..255
-        constexpr int kSet = 3;                                // pixel pairs per thread and round (6 loads)
-        struct ChunkInfo {
-            int gq, q, n0, hi0, wi0, c0, gr0, items, rounds;
-            long long pbase;
-        };
-        auto chunk_info = [&](int gq, ChunkInfo &ci) {
-            ci.gq = gq;
-            const int tl = gq / P.nchunks;
-            ci.q = gq - tl * P.nchunks;
-            int tile = (int)blockIdx.x + tl * (int)gridDim.x;
-            const int bn = tile / tiles_hw;
-            tile -= bn * tiles_hw;
-            const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
-            ci.n0 = bn * P.TN;
-            ci.hi0 = bh * P.PH * P.stride - P.pad;
-            ci.wi0 = bw * P.PW * P.stride - P.pad;
-            ci.pbase = ((long long)ci.n0 * P.H + ci.hi0) * P.W + ci.wi0;
-            const int2 rng = chunk_rng[ci.q];
-            ci.c0 = rng.x;
-            ci.gr0 = rng.x >> 3;
-            ci.items = ((rng.y >> 3) - ci.gr0 + 1) * npair;    // (channel group, pixel pair), pixel pair fastest
-            ci.rounds = (ci.items + kStageWarps * 32 * kSet - 1) / (kStageWarps * 32 * kSet);
-        };
-        uint4 va[2][kSet], vb[2][kSet];
-        auto load_round = [&](const ChunkInfo &ci, int r, int set) {
-#pragma unroll
-            for (int m = 0; m < kSet; ++m) {
-                const int t = (r * kSet + m) * (kStageWarps * 32) + st;
-                va[set][m] = make_uint4(0, 0, 0, 0);
-                vb[set][m] = make_uint4(0, 0, 0, 0);
-                if (t < ci.items) {
-                    const int gr = t / npair, pp = t - gr * npair;
-                    const int2 e = pix_tab[pp];
-                    const int tn = e.y & 0xff, ih = (e.y >> 8) & 0xff, iw = e.y >> 16;
-                    const int hi = ci.hi0 + ih, wi = ci.wi0 + iw;
-                    const bool rowok = ci.n0 + tn < P.N && hi >= 0 && hi < P.H;
-                    const uint16_t *xp = P.x + (ci.pbase + e.x) * P.C + (ci.gr0 + gr) * 8;
-                    if (rowok && wi >= 0 && wi < P.W && iw < P.IW) va[set][m] = __ldg(reinterpret_cast<const uint4 *>(xp));
-                    if (rowok && wi + 1 >= 0 && wi + 1 < P.W && iw + 1 < P.IW)
-                        vb[set][m] = __ldg(reinterpret_cast<const uint4 *>(xp + P.C));
-                }
-            }
-        };
-        auto store_round = [&](const ChunkInfo &ci, int r, int set, uint32_t xs) {
-#pragma unroll
-            for (int m = 0; m < kSet; ++m) {
-                const int t = (r * kSet + m) * (kStageWarps * 32) + st;
-                if (t < ci.items) {
-                    const int gr = t / npair, pp = t - gr * npair;
-                    const int cb = (ci.gr0 + gr) * 8 - ci.c0;   // slot channel of the group's first channel
-                    const bool whole = cb >= 0 && cb + 8 <= P.span;
-                    const uint32_t a4[4] = {va[set][m].x, va[set][m].y, va[set][m].z, va[set][m].w};
-                    const uint32_t b4[4] = {vb[set][m].x, vb[set][m].y, vb[set][m].z, vb[set][m].w};
-                    const uint32_t dst = xs + (uint32_t)(cb * P.plane + 2 * pp) * 2;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        // channel cb+e of the two pixels -> one 32-bit store
-                        const uint32_t word = (e & 1) ? __byte_perm(a4[e >> 1], b4[e >> 1], 0x7632)
-                                                      : __byte_perm(a4[e >> 1], b4[e >> 1], 0x5410);
-                        if (whole || (cb + e >= 0 && cb + e < P.span)) sts32(dst + (uint32_t)(e * P.plane * 2), word);
-                    }
-                }
-            }
-        };
-        if (total_chunks > 0) {
-            ChunkInfo LC, SC;
-            chunk_info(0, LC);
-            SC = LC;
-            int lr = 0, sr = 0, set = 0;
-            load_round(LC, 0, 0);
-            while (true) {
-                // advance the load cursor and issue its loads into the other register set
-                bool more = true;
-                if (++lr == LC.rounds) {
-                    lr = 0;
-                    if (LC.gq + 1 < total_chunks) chunk_info(LC.gq + 1, LC);
-                    else more = false;
-                }
-                if (more) {
-                    if (set == 0) load_round(LC, lr, 1);
-                    else load_round(LC, lr, 0);
-                    if (lr == 0 && LC.q == 0 && warp == kDwWarps + 1) {
-                        // first chunk of a tile: pull the rest of that tile's input patch towards L2
-                        for (int pp = lane; pp < npair; pp += 32) {
-                            const int2 e = pix_tab[pp];
-                            const int tn = e.y & 0xff, ih = (e.y >> 8) & 0xff, iw = e.y >> 16;
-                            const int hi = LC.hi0 + ih, wi = LC.wi0 + iw;
-                            if (LC.n0 + tn < P.N && hi >= 0 && hi < P.H && wi >= 0 && wi + 1 < P.W && iw + 1 < P.IW) {
-                                const char *px = reinterpret_cast<const char *>(P.x + (LC.pbase + e.x) * P.C);
-                                for (int bb = 0; bb < P.C * 4; bb += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(px + bb));
-                            }
-                        }
-                    }
-                }
-                // store the round loaded one step earlier
-                const int slot = SC.gq % P.nslots;
-                const uint32_t xs = x_s + slot * slot_bytes;
-                if (sr == 0) {
-                    const int use = SC.gq / P.nslots;
-                    if (use >= 1) warp_wait(bar_xfree + 8 * slot, (use - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
-                    if (st == 0) {   // the chunk's filters and slot-channel indices: one bulk copy, counted by the slot's barrier
-                        const uint32_t wbytes = (uint32_t)kChunk * P.wstride * 4;
-                        mbar_expect_tx_only(bar_xfull + 8 * slot, wbytes);
-                        bulk_g2s(xs + xplanes_bytes, P.dwpack + (size_t)SC.q * kChunk * P.wstride, wbytes, bar_xfull + 8 * slot);
-                    }
-                }
-                if (set == 0) store_round(SC, sr, 0, xs);
-                else store_round(SC, sr, 1, xs);
-                if (++sr == SC.rounds) {
-                    sr = 0;
-                    warp_arrive(bar_xfull + 8 * slot);
-                    if (SC.gq + 1 >= total_chunks) break;
-                    chunk_info(SC.gq + 1, SC);
-                }
-                set ^= 1;
-            }
-        }
     } else {
-        // ---------------- depthwise warps ----------------
+        // ---------------- depthwise warps: group g takes the chunks gq = g, g+2, ... ----------------
         regs_inc<kRegsDw>();
-        const int il = tid & 63, run = tid >> 6;
-        int q = 0;
-        for (int gq = 0; gq < total_chunks; ++gq) {
-            const int sa = gq & 1, slot = gq % P.nslots;
+        const int g = warp >> 3;
+        const int il = tid & 63, run = (tid >> 6) & 3;
+        const uint32_t a_stage = a_s + g * 16384;
+        int q = g % P.nchunks;
+        for (int gq = g, k = 0; gq < total_chunks; gq += 2, ++k) {
+            const int slot = gq % P.nslots;
             const bool live_i = q * kChunk + il < P.G;
             warp_wait(bar_xfull + 8 * slot, (gq / P.nslots) & 1, &abort_flag, P.status, kStatusWaitOperand);
-            const uint32_t xs = x_s + slot * slot_bytes;
-            const uint32_t wsm = xs + xplanes_bytes + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
+            const uint32_t xs = x_s + slot * (uint32_t)P.slot_bytes;
+            const uint32_t wsm = xs + (uint32_t)P.box_bytes + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
             float w[9];
-            int cl;
+            int clb;                                      // channel index inside the staged box
             if (MODE != 0) {
                 const uint4 w0 = lds128(wsm), w1 = lds128(wsm + 16), w2 = lds128(wsm + 32);
                 w[0] = __uint_as_float(w0.x); w[1] = __uint_as_float(w0.y); w[2] = __uint_as_float(w0.z);
                 w[3] = __uint_as_float(w0.w); w[4] = __uint_as_float(w1.x); w[5] = __uint_as_float(w1.y);
                 w[6] = __uint_as_float(w1.z); w[7] = __uint_as_float(w1.w); w[8] = __uint_as_float(w2.x);
-                cl = (int)w2.y;
+                clb = (int)w2.y;
             } else {
-                cl = (int)lds32(wsm + (uint32_t)(K * K) * 4);
+                clb = (int)lds32(wsm + (uint32_t)(K * K) * 4);
             }
-            if (gq >= 2) warp_wait(bar_afree + 8 * sa, ((gq >> 1) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
-            const uint32_t a_stage = a_s + sa * 16384;
-            if (MODE == 1) dw_rows_k3<S>(P, xs, cl, w, il, run, live_i, a_stage);
-            else if (MODE == 2) dw_quads_k3<S>(P, xs, cl, w, il, run, live_i, a_stage);
-            else dw_generic<K>(P, xs, cl, wsm, il, run, live_i, a_stage);
+            if (k >= 1) warp_wait(bar_afree + 8 * g, (k - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+            if (MODE == 1) dw_rows_k3<S, PS>(P, xs, clb, w, il, run, live_i, a_stage);
+            else if (MODE == 2) dw_quads_k3<S, PS>(P, xs, clb, w, il, run, live_i, a_stage);
+            else dw_generic<K>(P, xs, clb, wsm, il, run, live_i, a_stage);
             fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
-            warp_arrive(bar_afull + 8 * sa);
+            warp_arrive(bar_afull + 8 * g);
             warp_arrive(bar_xfree + 8 * slot);
-            q = (q + 1 == P.nchunks) ? 0 : q + 1;
+            q += 2;
+            while (q >= P.nchunks) q -= P.nchunks;
         }
     }
     tc_fence_before();
@@ -568,19 +445,51 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     if (warp == kCtrlWarp) tmem_dealloc(tmem, (uint32_t)(P.nacc * P.acc_cols));
 }
 
-template <int K, int MODE, int S>
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*tensor_map_encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                         const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                         CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                         CUtensorMapFloatOOBfill);
+
+static tensor_map_encode_fn encode_fn()
+{
+    static tensor_map_encode_fn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (tensor_map_encode_fn)p;
+    }
+    return fn;
+}
+
+template <int K, int MODE, int S, int PS>
 static gdws_status_t launch_fused(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
 {
     cudaError_t e = cudaSuccess;
     static bool attr_set[64] = {};
     if (!attr_set[device & 63]) {   // once per device: allow the full dynamic shared memory
-        e = cudaFuncSetAttribute(fused_bf16_kernel<K, MODE, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        e = cudaFuncSetAttribute(fused_bf16_kernel<K, MODE, S, PS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_bf16_kernel)");
         attr_set[device & 63] = true;
     }
-    fused_bf16_kernel<K, MODE, S><<<grid, kFusedThreads, smem, st>>>(P);
+    fused_bf16_kernel<K, MODE, S, PS><<<grid, kFusedThreads, smem, st>>>(P);
     e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "fused_bf16_kernel launch");
+}
+
+template <int MODE, int S>
+static gdws_status_t launch_fast(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
+{
+    switch (P.ps) {
+    case 64: return launch_fused<3, MODE, S, 64>(P, device, grid, smem, st);
+    case 128: return launch_fused<3, MODE, S, 128>(P, device, grid, smem, st);
+    case 256: return launch_fused<3, MODE, S, 256>(P, device, grid, smem, st);
+    default: return fail(GDWS_ERR_UNSUPPORTED, "staged pixel size %d", P.ps);
+    }
 }
 
 gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t st)
@@ -592,20 +501,34 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
     if (!choose_tile(p, x->n, x->h, x->w, &t))
         return fail(GDWS_ERR_UNSUPPORTED, "no fused tile fits this shape in shared memory");
     if (t.tiles() > 0x7fffffffLL) return fail(GDWS_ERR_UNSUPPORTED, "too many tiles");
-    if ((long long)x->n * x->h * x->w > 0x7fffffffLL) return fail(GDWS_ERR_UNSUPPORTED, "more than 2^31 input pixels");
     if (p->sm_count <= 0) {
         cudaError_t e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
         if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute(MultiProcessorCount)");
     }
+    tensor_map_encode_fn encode = encode_fn();
+    if (!encode) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
     FusedParams P;
-    P.x = (const uint16_t *)x->ptr; P.y = (uint16_t *)y->ptr;
+    {
+        // x as a rank-4 tensor, innermost first: channels, width, height, batch
+        const cuuint64_t dims[4] = {(cuuint64_t)p->C, (cuuint64_t)x->w, (cuuint64_t)x->h, (cuuint64_t)x->n};
+        const cuuint64_t strides[3] = {(cuuint64_t)p->C * 2, (cuuint64_t)x->w * p->C * 2,
+                                       (cuuint64_t)x->h * x->w * p->C * 2};
+        const cuuint32_t box[4] = {(cuuint32_t)t.cbox, (cuuint32_t)t.IW, (cuuint32_t)t.IH, (cuuint32_t)t.TN};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        const CUresult r = encode(&P.tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, x->ptr, dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    }
+    P.y = (uint16_t *)y->ptr;
     P.dwpack = p->d_dwpack; P.pw_img = p->d_pw_img; P.bias = p->d_bias;
-    P.chan = p->d_chan; P.chunk_c0 = p->d_chunk_c0; P.status = p->d_status;
+    P.chunk_c0 = p->d_chunk_c0; P.status = p->d_status;
     P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = y->h; P.Wo = y->w; P.D = p->D; P.Dpad = p->Dpad;
     P.G = p->G; P.nchunks = p->nchunks; P.stride = p->stride; P.pad = p->pad;
     P.relu = p->opt_relu;
     P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
-    P.IH = t.IH; P.IW = t.IW; P.IWp = t.IWp; P.plane = t.plane; P.span = t.span; P.nslots = t.nslots; P.nsb = t.nsb; P.wstride = p->wstride;
+    P.IH = t.IH; P.IW = t.IW; P.ps = t.cbox * 2; P.nslots = t.nslots; P.nsb = t.nsb; P.wstride = p->wstride;
+    P.box_bytes = t.box_bytes; P.slot_bytes = t.slot_bytes;
     P.nhalf = p->Dpad > 256 ? 2 : 1;
     P.unit_bytes = (p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
     P.acc_cols = tmem_cols_for(p->Dpad);
@@ -614,20 +537,21 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
     P.dw_math = p->opt_dw_math;
     const size_t smem = t.smem;     // one block per SM (register file), so the TMEM columns are never oversubscribed
     const int grid = P.ntiles < p->sm_count ? P.ntiles : p->sm_count;
+    const int dev = p->device;
     gdws_status_t rc;
-    if (t.fast == 1 && p->stride == 1) rc = launch_fused<3, 1, 1>(P, p->device, grid, smem, st);
-    else if (t.fast == 1 && p->stride == 2) rc = launch_fused<3, 1, 2>(P, p->device, grid, smem, st);
-    else if (t.fast == 2 && p->stride == 1) rc = launch_fused<3, 2, 1>(P, p->device, grid, smem, st);
-    else if (t.fast == 2 && p->stride == 2) rc = launch_fused<3, 2, 2>(P, p->device, grid, smem, st);
+    if (t.fast == 1 && p->stride == 1) rc = launch_fast<1, 1>(P, dev, grid, smem, st);
+    else if (t.fast == 1 && p->stride == 2) rc = launch_fast<1, 2>(P, dev, grid, smem, st);
+    else if (t.fast == 2 && p->stride == 1) rc = launch_fast<2, 1>(P, dev, grid, smem, st);
+    else if (t.fast == 2 && p->stride == 2) rc = launch_fast<2, 2>(P, dev, grid, smem, st);
     else {
         switch (p->k) {
-        case 1: rc = launch_fused<1, 0, 1>(P, p->device, grid, smem, st); break;
-        case 2: rc = launch_fused<2, 0, 1>(P, p->device, grid, smem, st); break;
-        case 3: rc = launch_fused<3, 0, 1>(P, p->device, grid, smem, st); break;
-        case 4: rc = launch_fused<4, 0, 1>(P, p->device, grid, smem, st); break;
-        case 5: rc = launch_fused<5, 0, 1>(P, p->device, grid, smem, st); break;
-        case 6: rc = launch_fused<6, 0, 1>(P, p->device, grid, smem, st); break;
-        case 7: rc = launch_fused<7, 0, 1>(P, p->device, grid, smem, st); break;
+        case 1: rc = launch_fused<1, 0, 1, 0>(P, dev, grid, smem, st); break;
+        case 2: rc = launch_fused<2, 0, 1, 0>(P, dev, grid, smem, st); break;
+        case 3: rc = launch_fused<3, 0, 1, 0>(P, dev, grid, smem, st); break;
+        case 4: rc = launch_fused<4, 0, 1, 0>(P, dev, grid, smem, st); break;
+        case 5: rc = launch_fused<5, 0, 1, 0>(P, dev, grid, smem, st); break;
+        case 6: rc = launch_fused<6, 0, 1, 0>(P, dev, grid, smem, st); break;
+        case 7: rc = launch_fused<7, 0, 1, 0>(P, dev, grid, smem, st); break;
         default: return fail(GDWS_ERR_UNSUPPORTED, "k=%d", p->k);
         }
     }

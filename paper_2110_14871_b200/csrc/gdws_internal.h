@@ -26,11 +26,12 @@ enum : int {
 struct Tile {
     int TN = 0, PH = 0, PW = 0;      // images x rows x columns of output pixels per 128-row tile
     int tiles_n = 0, tiles_h = 0, tiles_w = 0;
-    int IH = 0, IW = 0, IWp = 0;     // input patch rows / columns / row pitch (elements) per image
-    int plane = 0;                   // elements between consecutive channels in the staged input
-    int span = 0;                    // channels per staged slot (widest channel range of a K chunk)
+    int IH = 0, IW = 0;              // input patch rows / columns per image (with halo)
+    int cbox = 0;                    // channels per staged box (32, 64 or 128)
+    int box_bytes = 0;               // TN*IH*IW*cbox*2: one TMA box
+    int slot_bytes = 0;              // box + the chunk's filters, rounded up to 128
     int nslots = 0;                  // staged-input slots
-    int nsb = 0;                     // pointwise-weight stages
+    int nsb = 0;                     // pointwise-weight units in the ring
     int fast = 0;                    // 1: row-run depthwise path, 2: 4-wide-patch path, 0: generic
     size_t smem = 0;                 // dynamic shared memory of the fused kernel
     int64_t tiles() const { return (int64_t)tiles_n * tiles_h * tiles_w; }
@@ -44,7 +45,8 @@ struct gdws_plan_s {
     int wstride = 0;                 // 32-bit words per intermediate channel in d_dwpack (multiple of 4)
     std::vector<int32_t> g, off, chan;
     std::vector<int32_t> chunk_c0;   // first input channel read by K chunk q (intermediate channels 64q..64q+63)
-    int span_max = 0;                // widest channel range of one K chunk
+    int span_max = 0;                // widest channel range of one K chunk, counted from the chunk's first
+                                     // channel rounded down to a multiple of 8 (the staged box starts there)
 
     int opt_path = GDWS_PATH_AUTO;
     int opt_relu = 0;

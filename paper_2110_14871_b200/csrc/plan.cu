@@ -113,19 +113,18 @@ gdws_status_t ensure_device(gdws_plan_s *p)
 static int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
 // Shared-memory layout of the fused bf16 kernel: two intermediate-tile stages, a ring of `nsb`
-// pointwise-weight units (a unit = one K chunk x up to 256 output channels, at most 32 KB), `nslots`
-// staged-input slots (2, 4 or 8) and the patch table.  Fills t.nsb / t.nslots / t.smem; false if
-// it cannot fit.  Prefers at least 3 chunks of weights and 4 input slots in flight.
+// pointwise-weight units (a unit = one K chunk x up to 256 output channels, at most 32 KB) and
+// `nslots` staged-input slots (one TMA box plus the chunk's filters).  Fills t.nsb / t.nslots /
+// t.smem; false if it cannot fit.  Prefers at least 3 chunks of weights and 4 input slots in flight.
 static bool fit_smem(const gdws_plan_s *p, Tile &t)
 {
     const size_t a = 2 * (size_t)kTileRows * kChunk * 2;
     const int nhalf = p->Dpad > 256 ? 2 : 1;
     const size_t unit = (size_t)(p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
-    const size_t slot = (size_t)t.span * t.plane * 2 + (size_t)kChunk * p->wstride * 4 /*the chunk's filters*/;
-    const size_t fixed = a + 1024 /*alignment slack*/ + (size_t)t.TN * t.IH * t.IWp * 4 /*patch table*/ +
-                         (size_t)p->nchunks * 8 /*channel range of every chunk*/;
+    const size_t slot = (size_t)t.slot_bytes;
+    const size_t fixed = a + 1024 /*alignment slack*/;
     int best_score = -1;
-    for (int ns = 2; ns <= 8; ns *= 2) {
+    for (int ns = 2; ns <= 8; ++ns) {
         if (fixed + ns * slot + (size_t)(nhalf + 1) * unit > (size_t)kMaxSmem) break;
         int nsb = (int)(((size_t)kMaxSmem - fixed - ns * slot) / unit);
         if (nsb > 8) nsb = 8;
@@ -146,6 +145,10 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
     const int Ho = gdws_out_dim(h, p->k, p->stride, p->pad);
     const int Wo = gdws_out_dim(w, p->k, p->stride, p->pad);
     if (n < 1 || Ho < 1 || Wo < 1) return false;
+    // channels per staged box: the widest aligned channel range of a chunk, as 32, 64 or 128
+    int cbox = 32;
+    while (cbox < p->span_max) cbox *= 2;
+    if (cbox > 128) return false;
     double best = 1e300;
     bool found = false;
     const int forced = p->opt_tile;
@@ -172,15 +175,13 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
                 t.tiles_n = (n + TN - 1) / TN;
                 t.IH = (PH - 1) * p->stride + p->k;
                 t.IW = (PW - 1) * p->stride + p->k;
-                t.IWp = round_up(t.IW, 8);
-                if (t.fast == 1 && p->stride == 2) t.IWp = round_up(2 * PW + 2, 8);   // the row path reads 18 columns per group
-                int plane = TN * t.IH * t.IWp;        // elements; make the byte stride = 16 (mod 128)
-                while ((plane * 2) % 128 != 16) plane += 8;
-                t.plane = plane;
-                t.span = p->span_max;
+                if (t.IH > 256 || t.IW > 256 || TN > 256) continue;      // TMA box extents
+                t.cbox = cbox;
+                t.box_bytes = TN * t.IH * t.IW * cbox * 2;
+                t.slot_bytes = round_up(t.box_bytes + kChunk * p->wstride * 4, 128);
                 if (!fit_smem(p, t)) continue;
                 const double tiles = (double)t.tiles();
-                const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IWp) * (t.fast ? 1.0 : 4.0) - 1e-3 * PW;
+                const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IW) * (t.fast ? 1.0 : 4.0) - 1e-3 * PW;
                 if (cost < best) { best = cost; *out = t; found = true; }
             }
         }
@@ -252,7 +253,7 @@ gdws_status_t gdws_plan(int C, int D, int k, int stride, int pad, const int32_t 
         const int lo = p->chan[q * kChunk];
         const int last = std::min(p->G, (q + 1) * kChunk) - 1;
         p->chunk_c0[q] = lo;
-        p->span_max = std::max(p->span_max, p->chan[last] - lo + 1);
+        p->span_max = std::max(p->span_max, p->chan[last] - (lo & ~7) + 1);
     }
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
