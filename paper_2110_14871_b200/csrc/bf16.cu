@@ -35,9 +35,9 @@ __global__ void pack_pw_kernel(const void *__restrict__ pw, int is_bf16, int D, 
 
 // dw_w[G][k][k] -> (1) fp32 taps [Gpad][k*k] (zero rows for the padding) for the unfused kernel,
 // (2) [Gpad][wstride] words for the fused kernel: the taps, then the index of the channel inside the
-// box staged for its K chunk (chan[i] - first channel of chunk i/64 rounded down to a multiple of 8).
+// input box staged for its K chunk (chan[i] - first channel of that box).
 __global__ void pack_dw_kernel(const void *__restrict__ dw, int is_bf16, int G, int Gpad, int k2, int wstride,
-                               const int32_t *__restrict__ chan, const int32_t *__restrict__ chunk_c0,
+                               const int32_t *__restrict__ chan, const int32_t *__restrict__ chunk_meta,
                                float *__restrict__ out, uint32_t *__restrict__ outp)
 {
     const int total = Gpad * wstride;
@@ -51,7 +51,7 @@ __global__ void pack_dw_kernel(const void *__restrict__ dw, int is_bf16, int G, 
             out[(size_t)i * k2 + j] = v;
             word = __float_as_uint(v);
         } else if (j == k2 && i < G) {
-            word = (uint32_t)(chan[i] - (chunk_c0[i / kChunk] & ~7));
+            word = (uint32_t)(chan[i] - chunk_meta[4 * (i / kChunk) + 2]);
         }
         outp[t] = word;
     }
@@ -73,7 +73,7 @@ gdws_status_t bf16_pack(gdws_plan_s *p, const void *dw_w, const void *pw_w, cons
     if (blocks > 148 * 8) blocks = 148 * 8;
     pack_pw_kernel<<<blocks, 256, 0, st>>>(pw_w, is_bf16, p->D, p->Dpad, p->G, p->nchunks, p->d_pw_img);
     int blocks2 = (p->Gpad * p->wstride + 255) / 256;
-    pack_dw_kernel<<<blocks2, 256, 0, st>>>(dw_w, is_bf16, p->G, p->Gpad, k2, p->wstride, p->d_chan, p->d_chunk_c0,
+    pack_dw_kernel<<<blocks2, 256, 0, st>>>(dw_w, is_bf16, p->G, p->Gpad, k2, p->wstride, p->d_chan, p->d_chunk_meta,
                                             p->d_dw, p->d_dwpack);
     pack_bias_kernel<<<(p->Dpad + 255) / 256, 256, 0, st>>>(bias, p->D, p->Dpad, p->d_bias);
     p->launches += 3;

@@ -5,10 +5,11 @@
 // PH x PW patch, all D output channels).  Within a tile the intermediate channels are processed
 // in K chunks of 64 (i = 64q .. 64q+63, canonical order i = off_c + j).  The warps form one
 // pipeline over the sequence of (tile, chunk) pairs, coupled only by mbarriers:
-//   * input loader (one thread): chunk q reads a contiguous range of input channels; one TMA
-//     tiled load (x seen as a rank-4 tensor C x W x H x N, box = channels x patch with halo,
-//     out-of-image positions filled with zeros) brings those channels of the tile's input patch
-//     into one of `nslots` shared-memory slots, and one bulk copy adds the chunk's 64 filters;
+//   * input loader (one thread): chunk q reads a contiguous range of input channels, and
+//     consecutive chunks whose ranges fit into one box of `cbox` channels share it; one TMA
+//     tiled load per box (x seen as a rank-4 tensor C x W x H x N, box = channels x patch with
+//     halo, out-of-image positions filled with zeros) brings those channels of the tile's input
+//     patch into one of `nslots` shared-memory slots; one bulk copy per chunk adds its 64 filters;
 //   * 16 depthwise warps in two groups that take alternate chunks: thread t of a group owns
 //     intermediate channel 64q + (t & 63) and a quarter of the tile's pixels; it keeps its k x k
 //     filter in registers, slides down the patch reusing each input row for up to k output rows,
@@ -34,11 +35,11 @@ struct alignas(64) FusedParams {
     const uint32_t *dwpack;
     const uint16_t *pw_img;
     const float *bias;
-    const int32_t *chunk_c0;
+    const int4 *chunk_meta;      // per chunk: {box index, flags, first channel of the box, 0}
     int *status;
     int N, H, W, C, Ho, Wo, D, Dpad, G, nchunks, stride, pad, relu;
     int TN, PH, PW, tiles_h, tiles_w, ntiles;
-    int IH, IW, ps, nslots, nsb, wstride;
+    int IH, IW, ps, nslots, nwslots, nboxes, nsb, wstride;
     int box_bytes, slot_bytes;
     int nhalf, unit_bytes, nacc, acc_cols;
     int a_kmajor, dw_math;
@@ -105,6 +106,23 @@ __device__ __forceinline__ float lds_bf16(uint32_t addr)
     return __uint_as_float(v << 16);
 }
 
+// Packed fp32 arithmetic: one instruction does two independent fused multiply-adds (same rounding as two
+// scalar FMAs), which halves the issue slots of the depthwise stage.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void ffma2(uint64_t &d, uint64_t a, uint64_t b)
+{
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
+}
+
 // Where the 8 bf16 results of pixel group `o` (rows 8o..8o+7 of the tile) and intermediate
 // channel column kk go in a pixel-contiguous (MN-major) stage: K group kk/8 and 64-row block
 // o/8 select a 1024-byte atom, kk%8 the 128-byte row, and the 16-byte piece is swizzled.
@@ -144,36 +162,49 @@ __device__ __forceinline__ void dw_rows_k3(const FusedParams &P, uint32_t xs, in
     const int seg = run % nseg;
     const int R0 = (run / nseg) * 4;               // first of the 4 rows (row index = tn*PH + ph)
     const int o0 = R0 * nseg + seg;
-    float acc[4][8];
+    uint64_t acc2[4][4];                           // pairs of adjacent output columns
 #pragma unroll
     for (int ro = 0; ro < 4; ++ro)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[ro][e] = 0.f;
+        for (int p = 0; p < 4; ++p) acc2[ro][p] = 0ull;
     if (live_i && R0 < P.TN * P.PH) {
         const int tn = R0 / P.PH, ph0 = R0 - tn * P.PH;
         const uint32_t rowb = (uint32_t)P.IW * PS;
         const uint32_t base = xs + (uint32_t)((tn * P.IH + ph0 * S) * P.IW + seg * 8 * S) * PS + (uint32_t)clb * 2;
         constexpr int NR = 3 * S + 3;              // input rows feeding 4 output rows
         constexpr int NX = 7 * S + 3;              // input columns feeding 8 output columns
+        uint64_t w2[9];
+#pragma unroll
+        for (int t = 0; t < 9; ++t) w2[t] = pack2(w[t], w[t]);
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
             float xr[NX];
 #pragma unroll
             for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * rowb + j * PS);
+            uint64_t xp[3][4];                     // inputs of output columns (2p, 2p+1) for tap column v
+#pragma unroll
+            for (int v = 0; v < 3; ++v)
+#pragma unroll
+                for (int p = 0; p < 4; ++p) xp[v][p] = pack2(xr[(2 * p) * S + v], xr[(2 * p + 1) * S + v]);
 #pragma unroll
             for (int ro = 0; ro < 4; ++ro) {
                 const int u = r - ro * S;
                 if (u >= 0 && u < 3) {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e)
+                    for (int p = 0; p < 4; ++p)
 #pragma unroll
-                        for (int v = 0; v < 3; ++v) acc[ro][e] = fmaf(w[u * 3 + v], xr[e * S + v], acc[ro][e]);
+                        for (int v = 0; v < 3; ++v) ffma2(acc2[ro][p], w2[u * 3 + v], xp[v][p]);
                 }
             }
         }
     }
 #pragma unroll
-    for (int ro = 0; ro < 4; ++ro) store_group(P, a_stage, o0 + ro * nseg, kk, acc[ro]);
+    for (int ro = 0; ro < 4; ++ro) {
+        float out[8];
+#pragma unroll
+        for (int p = 0; p < 4; ++p) unpack2(acc2[ro][p], out[2 * p], out[2 * p + 1]);
+        store_group(P, a_stage, o0 + ro * nseg, kk, out);
+    }
 }
 
 // ---- depthwise, k = 3, 4-wide patches: a pixel group is 2 output rows x 4 columns of one image.
@@ -259,10 +290,11 @@ template <int K, int MODE, int S, int PS>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __grid_constant__ FusedParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    // a_full[2] a_free[2] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2]
-    __shared__ __align__(8) uint64_t bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots + 4];
+    // a_full[2] a_free[2] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2] | w_full[8] w_free[8]
+    __shared__ __align__(8) uint64_t bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots + 4 + 2 * kMaxSlots];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ uint32_t xinfo[kMaxSlots];      // per filter-ring slot: input slot (bits 0-7) and phase parity (bit 8) of the chunk's box
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t a_s = smem_u32(base);
@@ -274,6 +306,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const uint32_t bar_xfree = smem_u32(&bars[4 + 2 * kMaxBUnits + kMaxSlots]);
     const uint32_t bar_accfull = smem_u32(&bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots]);
     const uint32_t bar_accfree = bar_accfull + 16;
+    const uint32_t bar_wfull = bar_accfull + 32, bar_wfree = bar_wfull + 8 * kMaxSlots;
+    const uint32_t wblock = (uint32_t)kChunk * P.wstride * 4;             // one chunk's filters
+    const uint32_t w_s = x_s + (uint32_t)P.nslots * P.slot_bytes;         // ring of nwslots filter blocks
+    int4 *meta_tab = reinterpret_cast<int4 *>(base + (w_s - a_s) + (size_t)P.nwslots * wblock);
 
     if (tid == 0) {
         abort_flag = 0;
@@ -284,10 +320,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             mbar_init(bar_accfree + 8 * i, kEpiWarps);
         }
         for (int i = 0; i < kMaxBUnits; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
-        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(bar_xfull + 8 * i, 1); mbar_init(bar_xfree + 8 * i, kDwGroupWarps); }
+        for (int i = 0; i < kMaxSlots; ++i) {
+            mbar_init(bar_xfull + 8 * i, 1);
+            mbar_init(bar_xfree + 8 * i, 2 * kDwGroupWarps);   // the last two chunks that use a box release it
+            mbar_init(bar_wfull + 8 * i, 1);
+            mbar_init(bar_wfree + 8 * i, kDwGroupWarps);
+        }
         fence_mbar_init();
     }
     if (warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
+    for (int q = tid; q < P.nchunks; q += kFusedThreads) meta_tab[q] = __ldg(P.chunk_meta + q);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -352,10 +394,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 if (++h == P.nhalf) { h = 0; if (++q == P.nchunks) q = 0; }
             }
         } else if (warp == kCtrlWarp + 2 && lane == 0) {
-            // ---------------- input loader (one thread): ring of nslots slots ----------------
-            const uint32_t wbytes = (uint32_t)kChunk * P.wstride * 4;
-            uint32_t slot = 0, px = 1;        // parity of the "slot free" phase awaited
-            int gq = 0;
+            // ---------------- input loader (one thread): ring of boxes, ring of filter blocks ----------------
+            uint32_t xslot = 0, xpar = 1;     // next box slot; parity of the "slot free" phase awaited
+            uint32_t wslot = 0, wpar = 1;
+            uint32_t cur_x = 0;               // slot and "full" phase parity of the box the current chunks read
+            int gq = 0, gb = 0;
             for (int tl = 0; tl < my_tiles; ++tl) {
                 int tile = (int)blockIdx.x + tl * (int)gridDim.x;
                 const int bn = tile / tiles_hw;
@@ -363,14 +406,20 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
                 const int n0 = bn * P.TN, hi0 = bh * P.PH * P.stride - P.pad, wi0 = bw * P.PW * P.stride - P.pad;
                 for (int q = 0; q < P.nchunks; ++q, ++gq) {
-                    if (gq >= P.nslots) mbar_wait(bar_xfree + 8 * slot, px, &abort_flag, P.status, kStatusWaitStage);
-                    const uint32_t xs = x_s + slot * (uint32_t)P.slot_bytes;
-                    const int cbase = __ldg(P.chunk_c0 + q) & ~7;          // first channel of the box (16-byte aligned)
-                    mbar_expect_tx(bar_xfull + 8 * slot, (uint32_t)P.box_bytes + wbytes);
-                    tma_load_4d(xs, &P.tmap, cbase, wi0, hi0, n0, bar_xfull + 8 * slot);
-                    bulk_g2s(xs + (uint32_t)P.box_bytes, P.dwpack + (size_t)q * kChunk * P.wstride, wbytes,
-                             bar_xfull + 8 * slot);
-                    if (++slot == (uint32_t)P.nslots) { slot = 0; px ^= 1; }
+                    const int4 meta = meta_tab[q];
+                    if (meta.y & 4) {         // first chunk of a box: fetch the box
+                        if (gb >= P.nslots) mbar_wait(bar_xfree + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitStage);
+                        mbar_expect_tx(bar_xfull + 8 * xslot, (uint32_t)P.box_bytes);
+                        tma_load_4d(x_s + xslot * (uint32_t)P.slot_bytes, &P.tmap, meta.z, wi0, hi0, n0, bar_xfull + 8 * xslot);
+                        cur_x = xslot | ((xpar ^ 1u) << 8);   // "full" phase parity = the opposite of the "free" parity awaited
+                        ++gb;
+                        if (++xslot == (uint32_t)P.nslots) { xslot = 0; xpar ^= 1; }
+                    }
+                    if (gq >= P.nwslots) mbar_wait(bar_wfree + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitStage);
+                    xinfo[wslot] = cur_x;                     // published by the arrive below
+                    mbar_expect_tx(bar_wfull + 8 * wslot, wblock);
+                    bulk_g2s(w_s + wslot * wblock, P.dwpack + (size_t)q * kChunk * P.wstride, wblock, bar_wfull + 8 * wslot);
+                    if (++wslot == (uint32_t)P.nwslots) { wslot = 0; wpar ^= 1; }
                 }
             }
         }
@@ -410,13 +459,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int g = warp >> 3;
         const int il = tid & 63, run = (tid >> 6) & 3;
         const uint32_t a_stage = a_s + g * 16384;
-        int q = g % P.nchunks;
+        int q = g;
+        while (q >= P.nchunks) q -= P.nchunks;
+        int wslot = g;
+        uint32_t wpar = 0;
+        while (wslot >= P.nwslots) { wslot -= P.nwslots; wpar ^= 1; }
         for (int gq = g, k = 0; gq < total_chunks; gq += 2, ++k) {
-            const int slot = gq % P.nslots;
+            const int flags = meta_tab[q].y;
             const bool live_i = q * kChunk + il < P.G;
-            warp_wait(bar_xfull + 8 * slot, (gq / P.nslots) & 1, &abort_flag, P.status, kStatusWaitOperand);
-            const uint32_t xs = x_s + slot * (uint32_t)P.slot_bytes;
-            const uint32_t wsm = xs + (uint32_t)P.box_bytes + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
+            warp_wait(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
+            const uint32_t xi = xinfo[wslot];
+            const int xslot = (int)(xi & 0xffu);
+            const uint32_t wsm = w_s + wslot * wblock + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
             float w[9];
             int clb;                                      // channel index inside the staged box
             if (MODE != 0) {
@@ -428,15 +482,22 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             } else {
                 clb = (int)lds32(wsm + (uint32_t)(K * K) * 4);
             }
+            warp_wait(bar_xfull + 8 * xslot, xi >> 8, &abort_flag, P.status, kStatusWaitOperand);
+            const uint32_t xs = x_s + xslot * (uint32_t)P.slot_bytes;
             if (k >= 1) warp_wait(bar_afree + 8 * g, (k - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
             if (MODE == 1) dw_rows_k3<S, PS>(P, xs, clb, w, il, run, live_i, a_stage);
             else if (MODE == 2) dw_quads_k3<S, PS>(P, xs, clb, w, il, run, live_i, a_stage);
             else dw_generic<K>(P, xs, clb, wsm, il, run, live_i, a_stage);
             fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
             warp_arrive(bar_afull + 8 * g);
-            warp_arrive(bar_xfree + 8 * slot);
+            if (MODE == 0) __syncwarp();                  // the generic path reads its filter during the compute
+            warp_arrive(bar_wfree + 8 * wslot);
+            if (flags & 1) warp_arrive(bar_xfree + 8 * xslot);
+            if (flags & 2) warp_arrive(bar_xfree + 8 * xslot);
             q += 2;
             while (q >= P.nchunks) q -= P.nchunks;
+            wslot += 2;
+            while (wslot >= P.nwslots) { wslot -= P.nwslots; wpar ^= 1; }
         }
     }
     tc_fence_before();
@@ -522,12 +583,12 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
     }
     P.y = (uint16_t *)y->ptr;
     P.dwpack = p->d_dwpack; P.pw_img = p->d_pw_img; P.bias = p->d_bias;
-    P.chunk_c0 = p->d_chunk_c0; P.status = p->d_status;
+    P.chunk_meta = reinterpret_cast<const int4 *>(p->d_chunk_meta); P.status = p->d_status;
     P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = y->h; P.Wo = y->w; P.D = p->D; P.Dpad = p->Dpad;
     P.G = p->G; P.nchunks = p->nchunks; P.stride = p->stride; P.pad = p->pad;
     P.relu = p->opt_relu;
     P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
-    P.IH = t.IH; P.IW = t.IW; P.ps = t.cbox * 2; P.nslots = t.nslots; P.nsb = t.nsb; P.wstride = p->wstride;
+    P.IH = t.IH; P.IW = t.IW; P.ps = t.cbox * 2; P.nslots = t.nslots; P.nwslots = t.nwslots; P.nboxes = p->nboxes; P.nsb = t.nsb; P.wstride = p->wstride;
     P.box_bytes = t.box_bytes; P.slot_bytes = t.slot_bytes;
     P.nhalf = p->Dpad > 256 ? 2 : 1;
     P.unit_bytes = (p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;

@@ -29,8 +29,9 @@ struct Tile {
     int IH = 0, IW = 0;              // input patch rows / columns per image (with halo)
     int cbox = 0;                    // channels per staged box (32, 64 or 128)
     int box_bytes = 0;               // TN*IH*IW*cbox*2: one TMA box
-    int slot_bytes = 0;              // box + the chunk's filters, rounded up to 128
-    int nslots = 0;                  // staged-input slots
+    int slot_bytes = 0;              // box rounded up to 128
+    int nslots = 0;                  // staged-input slots (boxes in flight)
+    int nwslots = 0;                 // filter blocks in flight (one per chunk)
     int nsb = 0;                     // pointwise-weight units in the ring
     int fast = 0;                    // 1: row-run depthwise path, 2: 4-wide-patch path, 0: generic
     size_t smem = 0;                 // dynamic shared memory of the fused kernel
@@ -45,8 +46,15 @@ struct gdws_plan_s {
     int wstride = 0;                 // 32-bit words per intermediate channel in d_dwpack (multiple of 4)
     std::vector<int32_t> g, off, chan;
     std::vector<int32_t> chunk_c0;   // first input channel read by K chunk q (intermediate channels 64q..64q+63)
+    std::vector<int32_t> chunk_c1;   // last input channel read by K chunk q
     int span_max = 0;                // widest channel range of one K chunk, counted from the chunk's first
-                                     // channel rounded down to a multiple of 8 (the staged box starts there)
+                                     // channel rounded down to a multiple of 8 (a staged box starts there)
+    // Input boxes of the fused kernel: consecutive chunks whose channels fit into one box of `cbox`
+    // channels share it.  chunk_meta[q] = {box index within the tile, flags, first channel of the box, 0};
+    // flags: 1 = this chunk releases the box when done (last or second-to-last chunk using it),
+    // 2 = it is the only chunk of its box (releases twice), 4 = first chunk of its box (the loader fetches it).
+    int cbox = 0, nboxes = 0;
+    std::vector<int32_t> chunk_meta; // 4 ints per chunk
 
     int opt_path = GDWS_PATH_AUTO;
     int opt_relu = 0;
@@ -60,7 +68,7 @@ struct gdws_plan_s {
     bool arch_ok = false;          // the plan's device was checked to be compute capability 10.x
     int32_t *d_off = nullptr;      // [C+1]
     int32_t *d_chan = nullptr;     // [Gpad], -1 for padding
-    int32_t *d_chunk_c0 = nullptr; // [nchunks]
+    int32_t *d_chunk_meta = nullptr; // [nchunks][4]
     float *d_dw = nullptr;         // [Gpad][k*k] fp32 depthwise filters, zero rows for padding
     uint32_t *d_dwpack = nullptr;  // [Gpad][wstride]: k*k fp32 filter taps, then the channel's index within its K chunk's slot
     uint16_t *d_pw_img = nullptr;  // [nchunks][Dpad*64] bf16, 128-byte-swizzled K-major operand images

@@ -57,7 +57,7 @@ static void free_device(gdws_plan_s *p)
     cudaDeviceSynchronize();
     cudaFree(p->d_off);
     cudaFree(p->d_chan);
-    cudaFree(p->d_chunk_c0);
+    cudaFree(p->d_chunk_meta);
     cudaFree(p->d_dw);
     cudaFree(p->d_dwpack);
     cudaFree(p->d_pw_img);
@@ -89,7 +89,7 @@ gdws_status_t ensure_device(gdws_plan_s *p)
     } while (0)
     GDWS_TRY_ALLOC(p->d_off, sizeof(int32_t) * (p->C + 1));
     GDWS_TRY_ALLOC(p->d_chan, sizeof(int32_t) * p->Gpad);
-    GDWS_TRY_ALLOC(p->d_chunk_c0, sizeof(int32_t) * p->nchunks);
+    GDWS_TRY_ALLOC(p->d_chunk_meta, sizeof(int32_t) * 4 * p->nchunks);
     GDWS_TRY_ALLOC(p->d_dw, sizeof(float) * p->Gpad * k2);
     GDWS_TRY_ALLOC(p->d_dwpack, sizeof(uint32_t) * p->Gpad * p->wstride);
     GDWS_TRY_ALLOC(p->d_pw_img, img);
@@ -100,7 +100,7 @@ gdws_status_t ensure_device(gdws_plan_s *p)
     e = cudaMemcpy(p->d_off, p->off.data(), sizeof(int32_t) * (p->C + 1), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_chan, p->chan.data(), sizeof(int32_t) * p->Gpad, cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
-        e = cudaMemcpy(p->d_chunk_c0, p->chunk_c0.data(), sizeof(int32_t) * p->nchunks, cudaMemcpyHostToDevice);
+        e = cudaMemcpy(p->d_chunk_meta, p->chunk_meta.data(), sizeof(int32_t) * 4 * p->nchunks, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_bias, 0, sizeof(float) * p->Dpad);
     if (e != cudaSuccess) {
@@ -122,7 +122,9 @@ static bool fit_smem(const gdws_plan_s *p, Tile &t)
     const int nhalf = p->Dpad > 256 ? 2 : 1;
     const size_t unit = (size_t)(p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
     const size_t slot = (size_t)t.slot_bytes;
-    const size_t fixed = a + 1024 /*alignment slack*/;
+    const size_t wblock = (size_t)kChunk * p->wstride * 4;                 // one chunk's filters
+    t.nwslots = (int)std::max<size_t>(3, std::min<size_t>(8, (20 * 1024) / wblock));
+    const size_t fixed = a + 1024 /*alignment slack*/ + t.nwslots * wblock + (size_t)p->nchunks * 16 /*chunk table*/;
     int best_score = -1;
     for (int ns = 2; ns <= 8; ++ns) {
         if (fixed + ns * slot + (size_t)(nhalf + 1) * unit > (size_t)kMaxSmem) break;
@@ -145,10 +147,8 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
     const int Ho = gdws_out_dim(h, p->k, p->stride, p->pad);
     const int Wo = gdws_out_dim(w, p->k, p->stride, p->pad);
     if (n < 1 || Ho < 1 || Wo < 1) return false;
-    // channels per staged box: the widest aligned channel range of a chunk, as 32, 64 or 128
-    int cbox = 32;
-    while (cbox < p->span_max) cbox *= 2;
-    if (cbox > 128) return false;
+    const int cbox = p->cbox;
+    if (cbox <= 0) return false;            // some chunk reads more than 128 channels: no fused kernel
     double best = 1e300;
     bool found = false;
     const int forced = p->opt_tile;
@@ -178,7 +178,7 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
                 if (t.IH > 256 || t.IW > 256 || TN > 256) continue;      // TMA box extents
                 t.cbox = cbox;
                 t.box_bytes = TN * t.IH * t.IW * cbox * 2;
-                t.slot_bytes = round_up(t.box_bytes + kChunk * p->wstride * 4, 128);
+                t.slot_bytes = round_up(t.box_bytes, 128);
                 if (!fit_smem(p, t)) continue;
                 const double tiles = (double)t.tiles();
                 const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IW) * (t.fast ? 1.0 : 4.0) - 1e-3 * PW;
@@ -249,11 +249,57 @@ gdws_status_t gdws_plan(int C, int D, int k, int stride, int pad, const int32_t 
         delete p;
         return fail(GDWS_ERR_ALLOC, "gdws_plan: out of host memory");
     }
+    try {
+        p->chunk_c1.assign(p->nchunks, 0);
+        p->chunk_meta.assign((size_t)p->nchunks * 4, 0);
+    } catch (...) {
+        delete p;
+        return fail(GDWS_ERR_ALLOC, "gdws_plan: out of host memory");
+    }
     for (int q = 0; q < p->nchunks; ++q) {   // channel range read by K chunk q
         const int lo = p->chan[q * kChunk];
         const int last = std::min(p->G, (q + 1) * kChunk) - 1;
         p->chunk_c0[q] = lo;
+        p->chunk_c1[q] = p->chan[last];
         p->span_max = std::max(p->span_max, p->chan[last] - (lo & ~7) + 1);
+    }
+    // Group consecutive chunks into input boxes of cbox channels (32, 64 or 128): take the size that
+    // moves the fewest channels per tile, but no more than 64 unless a single chunk needs it.
+    {
+        long best_cost = -1;
+        for (int cb = 32; cb <= 128; cb *= 2) {
+            if (cb < p->span_max) continue;
+            if (cb > 64 && best_cost >= 0) break;
+            if (cb > 32 && best_cost >= 0 && p->Dpad > 256) break;   // wide layers: shared memory goes to the weight ring
+            int nb = 0;
+            for (int q = 0; q < p->nchunks;) {
+                const int cbase = p->chunk_c0[q] & ~7;
+                int e = q;
+                while (e + 1 < p->nchunks && p->chunk_c1[e + 1] < cbase + cb) ++e;
+                q = e + 1;
+                ++nb;
+            }
+            const long cost = (long)nb * cb;
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; p->cbox = cb; p->nboxes = nb; }
+        }
+        if (p->cbox > 0) {
+            int b = 0;
+            for (int q = 0; q < p->nchunks; ++b) {
+                const int cbase = p->chunk_c0[q] & ~7;
+                int e = q;
+                while (e + 1 < p->nchunks && p->chunk_c1[e + 1] < cbase + p->cbox) ++e;
+                for (int c = q; c <= e; ++c) {
+                    int flags = 0;
+                    if (c == e || c == e - 1) flags |= 1;
+                    if (q == e) flags |= 2;
+                    if (c == q) flags |= 4;
+                    p->chunk_meta[4 * c + 0] = b;
+                    p->chunk_meta[4 * c + 1] = flags;
+                    p->chunk_meta[4 * c + 2] = cbase;
+                }
+                q = e + 1;
+            }
+        }
     }
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
