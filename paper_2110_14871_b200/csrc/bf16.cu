@@ -136,6 +136,10 @@ __global__ void gdw_bf16_kernel(DwShape s, const uint16_t *__restrict__ x, const
 
 gdws_status_t bf16_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cudaStream_t st)
 {
+    if (p->C % 8 == 0) {   // tiled pipeline first; shapes it cannot tile fall through to the simple kernel
+        const gdws_status_t rc = bf16_depthwise_tiled(p, x, z, st);
+        if (rc != GDWS_ERR_UNSUPPORTED) return rc;
+    }
     DwShape s;
     s.N = x->n; s.H = x->h; s.W = x->w; s.C = p->C; s.G = p->G; s.Gpad = p->Gpad; s.k = p->k; s.stride = p->stride; s.pad = p->pad;
     s.Ho = gdws_out_dim(x->h, p->k, p->stride, p->pad);

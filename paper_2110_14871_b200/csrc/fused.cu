@@ -42,7 +42,7 @@ struct alignas(64) FusedParams {
     int IH, IW, ps, nslots, nwslots, nboxes, nsb, wstride;
     int box_bytes, slot_bytes;
     int nhalf, unit_bytes, nacc, acc_cols;
-    int a_kmajor, dw_math;
+    int a_kmajor, dw_math, zout;
 };
 
 // Warp roles, in warpgroups of 4 so that registers can be moved between the roles (setmaxnreg):
@@ -106,23 +106,6 @@ __device__ __forceinline__ float lds_bf16(uint32_t addr)
     return __uint_as_float(v << 16);
 }
 
-// Packed fp32 arithmetic: one instruction does two independent fused multiply-adds (same rounding as two
-// scalar FMAs), which halves the issue slots of the depthwise stage.
-__device__ __forceinline__ uint64_t pack2(float lo, float hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ void ffma2(uint64_t &d, uint64_t a, uint64_t b)
-{
-    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
-}
-
 // Where the 8 bf16 results of pixel group `o` (rows 8o..8o+7 of the tile) and intermediate
 // channel column kk go in a pixel-contiguous (MN-major) stage: K group kk/8 and 64-row block
 // o/8 select a 1024-byte atom, kk%8 the 128-byte row, and the 16-byte piece is swizzled.
@@ -162,49 +145,36 @@ __device__ __forceinline__ void dw_rows_k3(const FusedParams &P, uint32_t xs, in
     const int seg = run % nseg;
     const int R0 = (run / nseg) * 4;               // first of the 4 rows (row index = tn*PH + ph)
     const int o0 = R0 * nseg + seg;
-    uint64_t acc2[4][4];                           // pairs of adjacent output columns
+    float acc[4][8];
 #pragma unroll
     for (int ro = 0; ro < 4; ++ro)
 #pragma unroll
-        for (int p = 0; p < 4; ++p) acc2[ro][p] = 0ull;
+        for (int e = 0; e < 8; ++e) acc[ro][e] = 0.f;
     if (live_i && R0 < P.TN * P.PH) {
         const int tn = R0 / P.PH, ph0 = R0 - tn * P.PH;
         const uint32_t rowb = (uint32_t)P.IW * PS;
         const uint32_t base = xs + (uint32_t)((tn * P.IH + ph0 * S) * P.IW + seg * 8 * S) * PS + (uint32_t)clb * 2;
-        constexpr int NR = 3 * S + 3;              // input rows feeding 4 output rows
-        constexpr int NX = 7 * S + 3;              // input columns feeding 8 output columns
-        uint64_t w2[9];
-#pragma unroll
-        for (int t = 0; t < 9; ++t) w2[t] = pack2(w[t], w[t]);
+        constexpr int NR = 3 * S + 3;
+        constexpr int NX = 7 * S + 3;
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
             float xr[NX];
 #pragma unroll
             for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * rowb + j * PS);
-            uint64_t xp[3][4];                     // inputs of output columns (2p, 2p+1) for tap column v
-#pragma unroll
-            for (int v = 0; v < 3; ++v)
-#pragma unroll
-                for (int p = 0; p < 4; ++p) xp[v][p] = pack2(xr[(2 * p) * S + v], xr[(2 * p + 1) * S + v]);
 #pragma unroll
             for (int ro = 0; ro < 4; ++ro) {
                 const int u = r - ro * S;
                 if (u >= 0 && u < 3) {
 #pragma unroll
-                    for (int p = 0; p < 4; ++p)
+                    for (int e = 0; e < 8; ++e)
 #pragma unroll
-                        for (int v = 0; v < 3; ++v) ffma2(acc2[ro][p], w2[u * 3 + v], xp[v][p]);
+                        for (int v = 0; v < 3; ++v) acc[ro][e] = fmaf(w[u * 3 + v], xr[e * S + v], acc[ro][e]);
                 }
             }
         }
     }
 #pragma unroll
-    for (int ro = 0; ro < 4; ++ro) {
-        float out[8];
-#pragma unroll
-        for (int p = 0; p < 4; ++p) unpack2(acc2[ro][p], out[2 * p], out[2 * p + 1]);
-        store_group(P, a_stage, o0 + ro * nseg, kk, out);
-    }
+    for (int ro = 0; ro < 4; ++ro) store_group(P, a_stage, o0 + ro * nseg, kk, acc[ro]);
 }
 
 // ---- depthwise, k = 3, 4-wide patches: a pixel group is 2 output rows x 4 columns of one image.
@@ -286,7 +256,11 @@ __device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, in
 
 // MODE: 0 generic, 1 row runs (k=3), 2 4-wide patches (k=3); S = stride and PS = bytes per staged
 // pixel for modes 1/2 (mode 0 reads both from the parameters).
-template <int K, int MODE, int S, int PS>
+// ZOUT = true turns the kernel into the unfused GDW stage: the depthwise warps write channel-contiguous
+// stages and the four "epilogue" warps copy each finished stage to z[pixel][Gpad] in global memory
+// (16-byte stores, 128 contiguous bytes per pixel and chunk); no weights are streamed, no MMA is issued
+// and no TMEM is used.  P.y then points to z and P.D holds Gpad.
+template <int K, int MODE, int S, int PS, bool ZOUT>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __grid_constant__ FusedParams P)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -315,7 +289,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         abort_flag = 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_afull + 8 * i, kDwGroupWarps);
-            mbar_init(bar_afree + 8 * i, 1);
+            mbar_init(bar_afree + 8 * i, ZOUT ? kEpiWarps : 1);
             mbar_init(bar_accfull + 8 * i, 1);
             mbar_init(bar_accfree + 8 * i, kEpiWarps);
         }
@@ -328,12 +302,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         }
         fence_mbar_init();
     }
-    if (warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
+    if (!ZOUT && warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
     for (int q = tid; q < P.nchunks; q += kFusedThreads) meta_tab[q] = __ldg(P.chunk_meta + q);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = tmem_slot;
+    const uint32_t tmem = ZOUT ? 0u : tmem_slot;
 
     const int my_tiles = (P.ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const int total_chunks = my_tiles * P.nchunks;
@@ -344,7 +318,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int units_per_tile = P.nchunks * P.nhalf;
         const int total_units = my_tiles * units_per_tile;
         const int rows0 = P.Dpad > 256 ? 256 : P.Dpad, rows1 = P.Dpad - rows0;
-        if (warp == kCtrlWarp && lane == 0) {
+        if (!ZOUT && warp == kCtrlWarp && lane == 0) {
             // ---------------- MMA issue (one thread) ----------------
             const bool a_mn = !P.a_kmajor;
             const uint64_t adesc0 = a_mn ? make_sdesc(a_s, 1024, 2048) : make_sdesc(a_s, 16, 1024);
@@ -380,7 +354,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 }
                 umma_commit(bar_accfull + 8 * buf);
             }
-        } else if (warp == kCtrlWarp + 1 && lane == 0) {
+        } else if (!ZOUT && warp == kCtrlWarp + 1 && lane == 0) {
             // ---------------- pointwise-weight loader (one thread): ring of nsb units ----------------
             uint32_t sb = 0, pb = 1;          // parity of the "slot free" phase awaited (first round: nothing to wait for)
             int q = 0, h = 0;
@@ -432,6 +406,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int tn = r / hw;
         const int rem = r - tn * hw;
         const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
+        uint32_t sa = 0, pa = 0;                          // ZOUT: stage and phase parity of the next finished chunk
         for (int tl = 0; tl < my_tiles; ++tl) {
             int tile = (int)blockIdx.x + tl * (int)gridDim.x;
             const int bn = tile / tiles_hw;
@@ -440,6 +415,25 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
             const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
             uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D;
+            if (ZOUT) {
+                // this thread's pixel row of every finished stage goes to z (row r of the stage: 128 bytes, swizzled)
+                for (int q = 0; q < P.nchunks; ++q) {
+                    warp_wait(bar_afull + 8 * sa, pa, &abort_flag, P.status, kStatusWaitOperand);
+                    const uint32_t row_s = a_s + sa * 16384 + (uint32_t)r * 128;
+                    uint4 v[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) v[c] = lds128(row_s + (uint32_t)((c ^ (r & 7)) << 4));
+                    warp_arrive(bar_afree + 8 * sa);
+                    if (live) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(yrow + (size_t)q * kChunk);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) dst[c] = v[c];
+                    }
+                    sa ^= 1;
+                    if (sa == 0) pa ^= 1;
+                }
+                continue;
+            }
             const int buf = tl % P.nacc;
             warp_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
             tc_fence_after();
@@ -503,7 +497,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     tc_fence_before();
     __syncthreads();
     __syncwarp();
-    if (warp == kCtrlWarp) tmem_dealloc(tmem, (uint32_t)(P.nacc * P.acc_cols));
+    if (!ZOUT && warp == kCtrlWarp) tmem_dealloc(tmem, (uint32_t)(P.nacc * P.acc_cols));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -527,19 +521,26 @@ static tensor_map_encode_fn encode_fn()
     return fn;
 }
 
-template <int K, int MODE, int S, int PS>
-static gdws_status_t launch_fused(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
+template <int K, int MODE, int S, int PS, bool ZOUT>
+static gdws_status_t launch_one(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
 {
     cudaError_t e = cudaSuccess;
     static bool attr_set[64] = {};
     if (!attr_set[device & 63]) {   // once per device: allow the full dynamic shared memory
-        e = cudaFuncSetAttribute(fused_bf16_kernel<K, MODE, S, PS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        e = cudaFuncSetAttribute(fused_bf16_kernel<K, MODE, S, PS, ZOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_bf16_kernel)");
         attr_set[device & 63] = true;
     }
-    fused_bf16_kernel<K, MODE, S, PS><<<grid, kFusedThreads, smem, st>>>(P);
+    fused_bf16_kernel<K, MODE, S, PS, ZOUT><<<grid, kFusedThreads, smem, st>>>(P);
     e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "fused_bf16_kernel launch");
+}
+
+template <int K, int MODE, int S, int PS>
+static gdws_status_t launch_fused(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
+{
+    return P.zout ? launch_one<K, MODE, S, PS, true>(P, device, grid, smem, st)
+                  : launch_one<K, MODE, S, PS, false>(P, device, grid, smem, st);
 }
 
 template <int MODE, int S>
@@ -553,9 +554,9 @@ static gdws_status_t launch_fast(const FusedParams &P, int device, int grid, siz
     }
 }
 
-gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t st)
+static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out, int Ho, int Wo, bool zout, cudaStream_t st)
 {
-    if (p->Dpad > 512) return fail(GDWS_ERR_UNSUPPORTED, "bf16 fused kernel supports D <= 512 (got %d)", p->D);
+    if (!zout && p->Dpad > 512) return fail(GDWS_ERR_UNSUPPORTED, "bf16 fused kernel supports D <= 512 (got %d)", p->D);
     if (p->D % 8 || p->C % 8)
         return fail(GDWS_ERR_UNSUPPORTED, "bf16 kernels need C %% 8 == 0 and D %% 8 == 0 (got C=%d, D=%d)", p->C, p->D);
     Tile t;
@@ -581,10 +582,10 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     }
-    P.y = (uint16_t *)y->ptr;
+    P.y = (uint16_t *)out;
     P.dwpack = p->d_dwpack; P.pw_img = p->d_pw_img; P.bias = p->d_bias;
     P.chunk_meta = reinterpret_cast<const int4 *>(p->d_chunk_meta); P.status = p->d_status;
-    P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = y->h; P.Wo = y->w; P.D = p->D; P.Dpad = p->Dpad;
+    P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = Ho; P.Wo = Wo; P.D = zout ? p->Gpad : p->D; P.Dpad = p->Dpad;
     P.G = p->G; P.nchunks = p->nchunks; P.stride = p->stride; P.pad = p->pad;
     P.relu = p->opt_relu;
     P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
@@ -594,8 +595,9 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
     P.unit_bytes = (p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
     P.acc_cols = tmem_cols_for(p->Dpad);
     P.nacc = P.acc_cols <= 256 ? 2 : 1;
-    P.a_kmajor = p->opt_a_layout;
+    P.a_kmajor = zout ? 1 : p->opt_a_layout;
     P.dw_math = p->opt_dw_math;
+    P.zout = zout ? 1 : 0;
     const size_t smem = t.smem;     // one block per SM (register file), so the TMEM columns are never oversubscribed
     const int grid = P.ntiles < p->sm_count ? P.ntiles : p->sm_count;
     const int dev = p->device;
@@ -618,6 +620,20 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
     }
     if (rc == GDWS_OK) p->launches++;
     return rc;
+}
+
+gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t st)
+{
+    return run_tiled(p, x, y->ptr, y->h, y->w, false, st);
+}
+
+// The unfused GDW stage with the tiled pipeline (TMA-staged input, register-blocked depthwise warps,
+// coalesced 16-byte stores of z).  GDWS_ERR_UNSUPPORTED if no tile fits; the caller then takes the
+// simple kernel.
+gdws_status_t bf16_depthwise_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cudaStream_t st)
+{
+    const int Ho = gdws_out_dim(x->h, p->k, p->stride, p->pad), Wo = gdws_out_dim(x->w, p->k, p->stride, p->pad);
+    return run_tiled(p, x, z, Ho, Wo, true, st);
 }
 
 }  // namespace gdws

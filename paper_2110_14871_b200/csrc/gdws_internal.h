@@ -109,5 +109,6 @@ gdws_status_t bf16_pack(gdws_plan_s *p, const void *dw_w, const void *pw_w, cons
 gdws_status_t bf16_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cudaStream_t s);
 gdws_status_t bf16_pointwise(gdws_plan_s *p, const void *z, gdws_tensor_t *y, cudaStream_t s);
 gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t s);
+gdws_status_t bf16_depthwise_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cudaStream_t s);
 
 }  // namespace gdws

@@ -43,29 +43,29 @@ __device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes
 {
     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// One attempt: the thread is suspended by the hardware until the phase completes or about `hint_ns`
-// nanoseconds have passed, so a waiting warp does not compete for issue slots with the working ones.
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t hint_ns = 10000u)
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
 // Bounded wait.  When the limit runs out (about a second) the thread records `code` in the
 // status word and raises the block's abort flag; from then on every wait in the block returns
 // at once, so that all threads still walk the same control flow, reach the common teardown
-// (barriers stay matched, TMEM is freed) and the kernel ends.
-constexpr uint32_t kSpinLimit = 1u << 20;
+// (barriers stay matched, TMEM is freed) and the kernel ends.  The first few thousand polls
+// are back to back (waits in the pipeline are short and a sleeping waiter wakes up late).
+constexpr uint32_t kSpinLimit = 1u << 22;
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
 {
     if (*abort_flag) return;
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-        if (*abort_flag) return;
+        if (it > 4096) __nanosleep(64);
+        if ((it & 1023) == 1023 && *abort_flag) return;
     }
     *abort_flag = 1;
     atomicOr(status, code);
