@@ -67,6 +67,23 @@ def layer_roofline_us(macs, nbytes, peaks, sustained=False):
     return max(t_tensor, t_hbm), t_tensor, t_hbm
 
 
+def slowest_rank(value: float, device=None) -> float:
+    """Max of `value` over all ranks of the default process group (the value itself when there is none).
+    Replicas share nothing on the data path; this reduction of the measured time is the only exchange."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(units_per_rank: float, world: int, seconds_slowest: float) -> float:
+    """Whole-job throughput of `world` independent replicas: all units over the slowest rank's time."""
+    return world * units_per_rank / seconds_slowest
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
@@ -306,12 +323,10 @@ def run_ours(args, spec):
     ms = ev0.elapsed_time(ev1)
     if world > 1:
         dist.barrier()
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+        ms = slowest_rank(ms, device="cuda")
     plan.status()
     sec_per_step = ms / 1e3 / args.steps
-    value = world * spec.N / sec_per_step
+    value = aggregate_value(spec.N, world, sec_per_step)
 
     # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
@@ -329,10 +344,8 @@ def run_ours(args, spec):
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / k_e2e
         if world > 1:
-            t = torch.tensor([dt], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
-        e2e = {"value": world * spec.N / dt, "unit": UNIT, "h2d_bytes_per_step": xh.numel() * xh.element_size(),
+            dt = slowest_rank(dt, device="cuda")
+        e2e = {"value": aggregate_value(spec.N, world, dt), "unit": UNIT, "h2d_bytes_per_step": xh.numel() * xh.element_size(),
                "d2h_bytes_per_step": yh.numel() * yh.element_size(), "steps": k_e2e}
 
     if rank != 0:
