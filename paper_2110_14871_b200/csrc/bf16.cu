@@ -155,85 +155,111 @@ gdws_status_t bf16_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cu
 
 // ------------------------------------------------------------------------------------------
 // Pointwise 1x1 convolution as a GEMM: y[pixel][d] = bias[d] + sum_i z[pixel][i] * P[d][i].
-// One block = 128 pixels x all D; K loop over 64-wide chunks with two shared-memory stages.
+// Persistent blocks walk over tiles of 128 pixels (all D).  One thread loads (TMA tiled loads of the
+// 128 x 64 piece of z with the 128-byte swizzle the tensor cores expect, bulk copies of the packed
+// weight chunk), one thread issues tcgen05.mma into TMEM (two accumulators when D <= 256), four
+// warps run the epilogue of the previous tile meanwhile.  A ring of `ns` stages (z piece + weights).
 // ------------------------------------------------------------------------------------------
-constexpr int kPwThreads = 128;
+struct alignas(64) PwParams {
+    CUtensorMap tmap;            // z as (Gpad, pixels) bf16, box (64, 128), SWIZZLE_128B
+    const uint16_t *pw_img;
+    const float *bias;
+    uint16_t *y;
+    int *status;
+    long long npix;
+    int ntiles, nchunks, D, Dpad, relu, ns, stage_bytes, nacc, acc_cols;
+};
 
-__global__ void __launch_bounds__(kPwThreads)
-pw_bf16_tc_kernel(const uint16_t *__restrict__ z, const uint16_t *__restrict__ pw_img, const float *__restrict__ bias,
-                  uint16_t *__restrict__ y, long long npix, int Gpad, int D, int Dpad, int relu, int tmem_cols,
-                  int *status)
+constexpr int kPwThreads = 6 * 32;      // warp 0 loader, warp 1 MMA issue, warps 2-5 epilogue
+constexpr int kPwMaxStages = 8;
+
+__global__ void __launch_bounds__(kPwThreads, 1) pw_bf16_tc_kernel(const __grid_constant__ PwParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[4];     // b_full[2], mma_done[2]
+    __shared__ __align__(8) uint64_t bars[2 * kPwMaxStages + 4];   // full[8] free[8] acc_full[2] acc_free[2]
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const uint32_t a_s = smem_u32(base);
-    const uint32_t b_bytes = (uint32_t)Dpad * kChunk * 2;
-    const uint32_t b_s = a_s + 2 * 16384;
-    const uint32_t bar_bfull = smem_u32(&bars[0]), bar_done = smem_u32(&bars[2]);
-    const int nchunks = Gpad / kChunk;
+    const uint32_t st_s = smem_u32(base);
+    const uint32_t bar_full = smem_u32(&bars[0]), bar_free = smem_u32(&bars[kPwMaxStages]);
+    const uint32_t bar_accfull = smem_u32(&bars[2 * kPwMaxStages]), bar_accfree = bar_accfull + 16;
+    const uint32_t b_bytes = (uint32_t)P.Dpad * kChunk * 2;
 
     if (tid == 0) {
         abort_flag = 0;
-        for (int i = 0; i < 2; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_done + 8 * i, 1); }
+        for (int i = 0; i < kPwMaxStages; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_free + 8 * i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4); }
         fence_mbar_init();
     }
     __syncwarp();
-    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)tmem_cols);
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    const long long p0 = (long long)blockIdx.x * kTileRows;
+    const int my_tiles = (P.ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
 
-    for (int q = 0; q < nchunks; ++q) {
-        const int s = q & 1;
-        if (q >= 2) mbar_wait(bar_done + 8 * s, ((q >> 1) - 1) & 1, &abort_flag, status, kStatusWaitStage);
-        if (tid == 0) {
-            mbar_expect_tx(bar_bfull + 8 * s, b_bytes);
-            bulk_g2s(b_s + s * b_bytes, pw_img + (size_t)q * Dpad * kChunk, b_bytes, bar_bfull + 8 * s);
+    if (warp == 0) {
+        if (lane == 0) {        // ---------------- loader ----------------
+            uint32_t s = 0, par = 1;
+            int it = 0;
+            for (int tl = 0; tl < my_tiles; ++tl) {
+                const int row0 = ((int)blockIdx.x + tl * (int)gridDim.x) * kTileRows;
+                for (int q = 0; q < P.nchunks; ++q, ++it) {
+                    if (it >= P.ns) mbar_wait(bar_free + 8 * s, par, &abort_flag, P.status, kStatusWaitStage);
+                    const uint32_t dst = st_s + s * (uint32_t)P.stage_bytes;
+                    mbar_expect_tx(bar_full + 8 * s, 16384u + b_bytes);
+                    tma_load_2d(dst, &P.tmap, q * kChunk, row0, bar_full + 8 * s);
+                    bulk_g2s(dst + 16384u, P.pw_img + (size_t)q * P.Dpad * kChunk, b_bytes, bar_full + 8 * s);
+                    if (++s == (uint32_t)P.ns) { s = 0; par ^= 1; }
+                }
+            }
         }
-        // A chunk: 128 rows x 128 bytes, 16-byte pieces into the swizzled K-major layout
-        for (int t = tid; t < kTileRows * 8; t += kPwThreads) {
-            const int row = t >> 3, ch = t & 7;
-            const long long p = p0 + row;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (p < npix) v = __ldg(reinterpret_cast<const uint4 *>(z + (size_t)p * Gpad + q * kChunk + ch * 8));
-            sts128(a_s + s * 16384 + row * 128 + ((ch ^ (row & 7)) << 4), v);
+    } else if (warp == 1) {
+        if (lane == 0) {        // ---------------- MMA issue ----------------
+            uint32_t s = 0, par = 0;
+            for (int tl = 0; tl < my_tiles; ++tl) {
+                const int buf = tl % P.nacc;
+                if (tl >= P.nacc)
+                    mbar_wait(bar_accfree + 8 * buf, ((tl / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                tc_fence_after();
+                for (int q = 0; q < P.nchunks; ++q) {
+                    mbar_wait(bar_full + 8 * s, par, &abort_flag, P.status, kStatusWaitOperand);
+                    tc_fence_after();
+                    const uint32_t a_addr = st_s + s * (uint32_t)P.stage_bytes;
+                    issue_chunk(tmem + (uint32_t)(buf * P.acc_cols), a_addr, a_addr + 16384u, P.Dpad, false, q == 0);
+                    umma_commit(bar_free + 8 * s);
+                    if (++s == (uint32_t)P.ns) { s = 0; par ^= 1; }
+                }
+                umma_commit(bar_accfull + 8 * buf);
+            }
         }
-        fence_proxy_async();
-        __syncthreads();
-        if (tid == 0) {
-            mbar_wait(bar_bfull + 8 * s, (q >> 1) & 1, &abort_flag, status, kStatusWaitOperand);
+    } else {
+        // ---------------- epilogue warps ----------------
+        const int lg = warp & 3;
+        for (int tl = 0; tl < my_tiles; ++tl) {
+            const long long p = ((long long)blockIdx.x + (long long)tl * gridDim.x) * kTileRows + lg * 32 + lane;
+            const int buf = tl % P.nacc;
+            if (lane == 0) mbar_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
+            __syncwarp();
             tc_fence_after();
-            issue_chunk(tmem, a_s + s * 16384, b_s + s * b_bytes, Dpad, false, q == 0);
-            umma_commit(bar_done + 8 * s);
-        }
-    }
-    {
-        const int ql = nchunks - 1;
-        mbar_wait(bar_done + 8 * (ql & 1), (ql >> 1) & 1, &abort_flag, status, kStatusWaitMma);
-        if (nchunks >= 2) {   // the other stage's last commit, so that no arrival is pending at exit
-            const int qo = nchunks - 2;
-            mbar_wait(bar_done + 8 * (qo & 1), (qo >> 1) & 1, &abort_flag, status, kStatusWaitMma);
-        }
-    }
-    tc_fence_after();
-    {
-        const long long p = p0 + warp * 32 + lane;
-        for (int d0 = 0; d0 < Dpad; d0 += 16) {
-            uint32_t acc[16];
-            tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)d0, acc);
-            tmem_ld_wait();
-            if (p < npix) store_row16(acc, bias, d0, D, relu, y + (size_t)p * D);
+            const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * P.acc_cols);
+            for (int d0 = 0; d0 < P.Dpad; d0 += 16) {
+                uint32_t acc[16];
+                tmem_ld16(t_base + (uint32_t)d0, acc);
+                tmem_ld_wait();
+                if (p < P.npix) store_row16(acc, P.bias, d0, P.D, P.relu, P.y + (size_t)p * P.D);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_accfree + 8 * buf);
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, (uint32_t)tmem_cols);
+    __syncwarp();
+    if (warp == 1) tmem_dealloc(tmem, (uint32_t)(P.nacc * P.acc_cols));
 }
 
 gdws_status_t bf16_pointwise(gdws_plan_s *p, const void *z, gdws_tensor_t *y, cudaStream_t st)
@@ -241,9 +267,36 @@ gdws_status_t bf16_pointwise(gdws_plan_s *p, const void *z, gdws_tensor_t *y, cu
     if (p->Dpad > 512) return fail(GDWS_ERR_UNSUPPORTED, "bf16 pointwise kernel supports D <= 512 (got %d)", p->D);
     if (p->D % 8) return fail(GDWS_ERR_UNSUPPORTED, "bf16 kernels need D %% 8 == 0 (got %d)", p->D);
     const long long npix = (long long)y->n * y->h * y->w;
-    const int cols = tmem_cols_for(p->Dpad);
-    size_t smem = 1024 + 2 * 16384 + 2 * (size_t)p->Dpad * kChunk * 2;
-    smem = smem_for_tmem(smem, cols);
+    const long long tiles = (npix + kTileRows - 1) / kTileRows;
+    if (tiles > 0x7fffffffLL / kTileRows) return fail(GDWS_ERR_UNSUPPORTED, "too many pixels for the bf16 pointwise kernel");
+    if (p->sm_count <= 0) {
+        cudaError_t e0 = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+        if (e0 != cudaSuccess) return cuda_fail(e0, "cudaDeviceGetAttribute(MultiProcessorCount)");
+    }
+    tensor_map_encode_fn encode = encode_fn();
+    if (!encode) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    PwParams P;
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)p->Gpad, (cuuint64_t)npix};
+        const cuuint64_t strides[1] = {(cuuint64_t)p->Gpad * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)kChunk, (cuuint32_t)kTileRows};
+        const cuuint32_t estr[2] = {1, 1};
+        const CUresult r = encode(&P.tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(z), dims, strides, box,
+                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    }
+    P.pw_img = p->d_pw_img; P.bias = p->d_bias; P.y = (uint16_t *)y->ptr; P.status = p->d_status;
+    P.npix = npix; P.ntiles = (int)tiles; P.nchunks = p->nchunks; P.D = p->D; P.Dpad = p->Dpad; P.relu = p->opt_relu;
+    P.stage_bytes = 16384 + p->Dpad * kChunk * 2;
+    P.ns = (kMaxSmem - 1024) / P.stage_bytes;
+    if (P.ns > kPwMaxStages) P.ns = kPwMaxStages;
+    if (P.ns < 2) return fail(GDWS_ERR_UNSUPPORTED, "no room for two stages");
+    P.acc_cols = tmem_cols_for(p->Dpad);
+    P.nacc = P.acc_cols <= 256 ? 2 : 1;
+    // one block per SM: ask for more than half of the shared memory even when fewer stages would do
+    size_t smem = 1024 + (size_t)P.ns * P.stage_bytes;
+    if (smem < (size_t)kMaxSmem / 2 + 2048) smem = (size_t)kMaxSmem / 2 + 2048;
     cudaError_t e = cudaSuccess;
     static bool attr_set[64] = {};
     if (!attr_set[p->device & 63]) {   // once per device: allow the full dynamic shared memory
@@ -251,10 +304,8 @@ gdws_status_t bf16_pointwise(gdws_plan_s *p, const void *z, gdws_tensor_t *y, cu
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(pw_bf16_tc_kernel)");
         attr_set[p->device & 63] = true;
     }
-    const long long blocks = (npix + kTileRows - 1) / kTileRows;
-    pw_bf16_tc_kernel<<<(int)blocks, kPwThreads, smem, st>>>((const uint16_t *)z, p->d_pw_img, p->d_bias,
-                                                             (uint16_t *)y->ptr, npix, p->Gpad, p->D, p->Dpad,
-                                                             p->opt_relu, cols, p->d_status);
+    const int grid = (int)(tiles < p->sm_count ? tiles : p->sm_count);
+    pw_bf16_tc_kernel<<<grid, kPwThreads, smem, st>>>(P);
     p->launches++;
     e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "pw_bf16_tc_kernel launch");

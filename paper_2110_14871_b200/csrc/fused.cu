@@ -23,8 +23,6 @@
 //     optional ReLU, round to bf16 and store y.
 // Every wait is bounded; a wait that runs out raises a block-wide abort flag that turns all later
 // waits into no-ops, so the block still reaches its teardown, frees TMEM and ends.
-#include <cuda.h>
-
 #include "sm100.cuh"
 
 namespace gdws {
@@ -75,16 +73,6 @@ __device__ __forceinline__ void warp_arrive(uint32_t bar)
 
 template <int N> __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-
-// TMA tiled load of a rank-4 box; coordinates innermost first.  The innermost coordinate times the
-// element size must be a multiple of 16 bytes (here: a multiple of 8 channels).
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tmap, int c0, int c1, int c2, int c3,
-                                            uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
-}
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr)
 {
@@ -532,24 +520,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
-typedef CUresult (*tensor_map_encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                         const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
-                                         CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                         CUtensorMapFloatOOBfill);
-
-static tensor_map_encode_fn encode_fn()
-{
-    static tensor_map_encode_fn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (tensor_map_encode_fn)p;
-    }
-    return fn;
-}
-
 template <int K, int MODE, int S, int PS, bool ZOUT>
 static gdws_status_t launch_one(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
 {

@@ -11,6 +11,7 @@
 //     64 M are `leading byte offset` apart, groups of 8 K rows `stride byte offset` apart.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "gdws_internal.h"
@@ -222,6 +223,44 @@ inline size_t smem_for_tmem(size_t need, int cols)
     const int max_ctas = 512 / cols;
     const size_t floor_bytes = (size_t)kMaxSmem / (max_ctas + 1) + 1024;
     return need > floor_bytes ? need : floor_bytes;
+}
+
+
+// TMA tiled load of a rank-4 box; coordinates innermost first.  The innermost coordinate times the
+// element size must be a multiple of 16 bytes (here: a multiple of 8 channels).
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tmap, int c0, int c1, int c2, int c3,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+
+// TMA tiled load of a rank-2 box (innermost coordinate first; it must start on a 16-byte boundary).
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+// cuTensorMapEncodeTiled, looked up through the runtime (no link against the driver library).
+typedef CUresult (*tensor_map_encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                         const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                         CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                         CUtensorMapFloatOOBfill);
+
+inline tensor_map_encode_fn encode_fn()
+{
+    static tensor_map_encode_fn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (tensor_map_encode_fn)p;
+    }
+    return fn;
 }
 
 
