@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_afull + 8 * i, kDwGroupWarps);
+            mbar_init(bar_afull + 8 * i, 1);
             mbar_init(bar_afree + 8 * i, ZOUT ? kEpiWarps : 1);
             mbar_init(bar_accfull + 8 * i, 1);
             mbar_init(bar_accfree + 8 * i, kEpiWarps);
@@ -284,9 +284,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         for (int i = 0; i < kMaxBUnits; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
         for (int i = 0; i < kMaxSlots; ++i) {
             mbar_init(bar_xfull + 8 * i, 1);
-            mbar_init(bar_xfree + 8 * i, 2 * kDwGroupWarps);   // the last two chunks that use a box release it
+            mbar_init(bar_xfree + 8 * i, 2);                   // the last two chunks that use a box release it
             mbar_init(bar_wfull + 8 * i, 1);
-            mbar_init(bar_wfree + 8 * i, kDwGroupWarps);
+            mbar_init(bar_wfree + 8 * i, 1);
         }
         fence_mbar_init();
     }
@@ -446,69 +446,50 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         int wslot = g;
         uint32_t wpar = 0;
         while (wslot >= P.nwslots) { wslot -= P.nwslots; wpar ^= 1; }
-        // What a chunk needs besides the input box: flags, the thread's filter (in registers for the k=3
-        // paths), the channel's index in the box, and where the box is.
-        struct ChunkRegs {
-            float w[9];
-            int clb, flags, wslot;
-            uint32_t xi;
-            bool live;
-        };
-        auto fetch = [&](ChunkRegs &c) {
-            c.flags = meta_tab[q].y;
-            c.live = q * kChunk + il < P.G;
-            c.wslot = wslot;
-            warp_wait(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
-            c.xi = xinfo[wslot];
+        // Only one thread of a group touches the shared-memory barriers; the group's 256 threads meet at a
+        // hardware named barrier (id 1 + g) before and after a chunk's arithmetic.  (Barrier operations of
+        // all 16 warps would queue behind the other group's shared-memory loads.)
+        const bool leader = (tid & (kDwGroupWarps * 32 - 1)) == 0;
+        for (int gq = g, k = 0; gq < total_chunks; gq += 2, ++k) {
+            const int flags = meta_tab[q].y;
+            const bool live_i = q * kChunk + il < P.G;
+            if (leader) {
+                mbar_wait(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
+                const uint32_t xi0 = xinfo[wslot];
+                mbar_wait(bar_xfull + 8 * (xi0 & 0xffu), xi0 >> 8, &abort_flag, P.status, kStatusWaitOperand);
+                if (k >= 1) mbar_wait(bar_afree + 8 * g, (k - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+            }
+            named_bar_sync(1 + g, kDwGroupWarps * 32);
+            const uint32_t xi = xinfo[wslot];
+            const int xslot = (int)(xi & 0xffu);
+            const uint32_t xs = x_s + xslot * (uint32_t)P.slot_bytes;
             const uint32_t wsm = w_s + wslot * wblock + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
+            float w[9];
+            int clb;                                      // channel index inside the staged box
             if (MODE != 0) {
                 const uint4 w0 = lds128(wsm), w1 = lds128(wsm + 16), w2 = lds128(wsm + 32);
-                c.w[0] = __uint_as_float(w0.x); c.w[1] = __uint_as_float(w0.y); c.w[2] = __uint_as_float(w0.z);
-                c.w[3] = __uint_as_float(w0.w); c.w[4] = __uint_as_float(w1.x); c.w[5] = __uint_as_float(w1.y);
-                c.w[6] = __uint_as_float(w1.z); c.w[7] = __uint_as_float(w1.w); c.w[8] = __uint_as_float(w2.x);
-                c.clb = (int)w2.y;
+                w[0] = __uint_as_float(w0.x); w[1] = __uint_as_float(w0.y); w[2] = __uint_as_float(w0.z);
+                w[3] = __uint_as_float(w0.w); w[4] = __uint_as_float(w1.x); w[5] = __uint_as_float(w1.y);
+                w[6] = __uint_as_float(w1.z); w[7] = __uint_as_float(w1.w); w[8] = __uint_as_float(w2.x);
+                clb = (int)w2.y;
             } else {
-                c.clb = (int)lds32(wsm + (uint32_t)(K * K) * 4);
+                clb = (int)lds32(wsm + (uint32_t)(K * K) * 4);
+            }
+            if (MODE == 1) dw_rows_k3<S, PS>(P, xs, clb, w, il, run, live_i, a_stage);
+            else if (MODE == 2) dw_quads_k3<S, PS>(P, xs, clb, w, il, run, live_i, a_stage);
+            else dw_generic<K>(P, xs, clb, wsm, il, run, live_i, a_stage);
+            fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
+            named_bar_sync(1 + g, kDwGroupWarps * 32);
+            if (leader) {
+                mbar_arrive(bar_afull + 8 * g);
+                mbar_arrive(bar_wfree + 8 * wslot);
+                if (flags & 1) mbar_arrive(bar_xfree + 8 * xslot);
+                if (flags & 2) mbar_arrive(bar_xfree + 8 * xslot);
             }
             q += 2;
             while (q >= P.nchunks) q -= P.nchunks;
             wslot += 2;
             while (wslot >= P.nwslots) { wslot -= P.nwslots; wpar ^= 1; }
-        };
-        ChunkRegs cur, nxt;
-        if (g < total_chunks) fetch(cur);
-        for (int gq = g, k = 0; gq < total_chunks; gq += 2, ++k) {
-            // the k=3 paths keep the filter in registers: fetch the next chunk's filter now, so that its
-            // shared-memory latency and barrier round trip overlap this chunk's arithmetic
-            const bool has_next = gq + 2 < total_chunks;
-            // (only if that filter has already arrived: waiting for it here could wait for an input slot
-            // that this very chunk still has to release)
-            bool fetched = false;
-            if (MODE != 0 && has_next) {
-                uint32_t ready = 0;
-                if (lane == 0) ready = mbar_try_wait(bar_wfull + 8 * wslot, wpar);
-                ready = __shfl_sync(0xffffffffu, ready, 0);
-                if (ready) { fetch(nxt); fetched = true; }
-            }
-            const int xslot = (int)(cur.xi & 0xffu);
-            warp_wait(bar_xfull + 8 * xslot, cur.xi >> 8, &abort_flag, P.status, kStatusWaitOperand);
-            const uint32_t xs = x_s + xslot * (uint32_t)P.slot_bytes;
-            if (k >= 1) warp_wait(bar_afree + 8 * g, (k - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
-            if (MODE == 1) dw_rows_k3<S, PS>(P, xs, cur.clb, cur.w, il, run, cur.live, a_stage);
-            else if (MODE == 2) dw_quads_k3<S, PS>(P, xs, cur.clb, cur.w, il, run, cur.live, a_stage);
-            else dw_generic<K>(P, xs, cur.clb, w_s + cur.wslot * wblock + (uint32_t)(il * P.wstride) * 4, il, run, cur.live, a_stage);
-            fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
-            warp_arrive(bar_afull + 8 * g);
-            // The filter block is free once every lane holds its filter in registers (k=3 paths: the shared
-            // loads of this chunk's arithmetic were issued after the filter loads and have returned) or has
-            // finished reading it (generic path).
-            warp_arrive(bar_wfree + 8 * cur.wslot);
-            if (cur.flags & 1) warp_arrive(bar_xfree + 8 * xslot);
-            if (cur.flags & 2) warp_arrive(bar_xfree + 8 * xslot);
-            if (has_next) {
-                if (fetched) cur = nxt;
-                else fetch(cur);
-            }
         }
     }
     tc_fence_before();
