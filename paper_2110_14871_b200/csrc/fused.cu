@@ -321,10 +321,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     mbar_wait(bar_accfree + 8 * buf, ((tl / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
                 tc_fence_after();
                 for (int q = 0; q < P.nchunks; ++q) {
+                    // the weights arrive long before the intermediate tile: take that wait off the critical path
+                    mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
                     mbar_wait(bar_afull + 8 * sa, pa, &abort_flag, P.status, kStatusWaitOperand);
                     const uint64_t adesc = adesc0 + (uint64_t)(sa * (16384u >> 4));
                     for (int h = 0; h < P.nhalf; ++h) {
-                        mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
+                        if (h > 0) mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
                         tc_fence_after();
                         const uint32_t d_tmem = tmem + (uint32_t)(buf * P.acc_cols + h * 256);
                         const uint64_t bdesc = bdesc0 + (uint64_t)(sb * ((uint32_t)P.unit_bytes >> 4));
@@ -455,8 +457,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             const bool live_i = q * kChunk + il < P.G;
             if (leader) {
                 mbar_wait(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
-                const uint32_t xi0 = xinfo[wslot];
-                mbar_wait(bar_xfull + 8 * (xi0 & 0xffu), xi0 >> 8, &abort_flag, P.status, kStatusWaitOperand);
+                if (flags & 8) {   // first or second chunk of its box: later ones follow one of these in the same group
+                    const uint32_t xi0 = xinfo[wslot];
+                    mbar_wait(bar_xfull + 8 * (xi0 & 0xffu), xi0 >> 8, &abort_flag, P.status, kStatusWaitOperand);
+                }
                 if (k >= 1) mbar_wait(bar_afree + 8 * g, (k - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
             }
             named_bar_sync(1 + g, kDwGroupWarps * 32);

@@ -52,7 +52,8 @@ struct gdws_plan_s {
     // Input boxes of the fused kernel: consecutive chunks whose channels fit into one box of `cbox`
     // channels share it.  chunk_meta[q] = {box index within the tile, flags, first channel of the box, 0};
     // flags: 1 = this chunk releases the box when done (last or second-to-last chunk using it),
-    // 2 = it is the only chunk of its box (releases twice), 4 = first chunk of its box (the loader fetches it).
+    // 2 = it is the only chunk of its box (releases twice), 4 = first chunk of its box (the loader fetches it),
+    // 8 = first or second chunk of its box (must wait for the box to land).
     int cbox = 0, nboxes = 0;
     std::vector<int32_t> chunk_meta; // 4 ints per chunk
 

@@ -293,6 +293,7 @@ gdws_status_t gdws_plan(int C, int D, int k, int stride, int pad, const int32_t 
                     if (c == e || c == e - 1) flags |= 1;
                     if (q == e) flags |= 2;
                     if (c == q) flags |= 4;
+                    if (c == q || c == q + 1) flags |= 8;
                     p->chunk_meta[4 * c + 0] = b;
                     p->chunk_meta[4 * c + 1] = flags;
                     p->chunk_meta[4 * c + 2] = cbase;
