@@ -13,11 +13,14 @@
 //   * 16 depthwise warps in two groups that take alternate chunks: thread t of a group owns
 //     intermediate channel 64q + (t & 63) and a quarter of the tile's pixels; it keeps its k x k
 //     filter in registers, slides down the patch reusing each input row for up to k output rows,
-//     and writes bf16 results as 16-byte pieces into the group's pixel-contiguous (MN-major),
-//     128-byte-swizzled tensor-core operand stage;
+//     and writes bf16 results as 16-byte pieces into one of the group's (one or two) pixel-contiguous
+//     (MN-major), 128-byte-swizzled tensor-core operand stages; a finished chunk is handed over through
+//     a hardware named barrier on which the depthwise threads only arrive, so that they go on to their
+//     next chunk at once;
 //   * weight loader (one thread): streams the pre-swizzled pointwise weights (bulk copies with
 //     mbarrier completion, a ring of units of at most 256 output channels x 64);
-//   * MMA issuer (one thread): tcgen05.mma into a TMEM accumulator (128 lanes x D fp32 columns;
+//   * MMA warp: waits on that named barrier chunk by chunk, releases the chunk's filter block and
+//     input box, and one lane issues tcgen05.mma into a TMEM accumulator (128 lanes x D fp32 columns;
 //     two accumulators when D <= 256, so that a tile's epilogue overlaps the next tile's main loop);
 //   * 4 epilogue warps: read the finished accumulator (tcgen05.ld), add the bias, apply the
 //     optional ReLU, round to bf16 and store y.
@@ -38,18 +41,21 @@ struct alignas(64) FusedParams {
     int N, H, W, C, Ho, Wo, D, Dpad, G, nchunks, stride, pad, relu;
     int TN, PH, PW, tiles_h, tiles_w, ntiles;
     int IH, IW, ps, nslots, nwslots, nboxes, nsb, wstride;
+    int spg_shift;                 // log2 of the operand stages per depthwise group (0 or 1)
     int box_bytes, slot_bytes;
     int nhalf, unit_bytes, nacc, acc_cols;
     int a_kmajor, dw_math, zout;
 };
 
 // Warp roles, in warpgroups of 4 so that registers can be moved between the roles (setmaxnreg):
-// warps 0-15 depthwise (two groups of 8), 16 MMA issue, 17 weight loader, 18 input loader
-// (19 idle), 20-23 epilogue.
+// warp 0 MMA issue, 1 weight loader, 2 input loader (3 idle), 4-19 depthwise (two groups of 8),
+// 20-23 epilogue.  The control warps come first: the schedulers favour a block's oldest warps, and a
+// control lane that has to queue behind the depthwise warps' instruction streams stalls the pipeline.
 constexpr int kDwWarps = 16, kDwGroupWarps = 8, kEpiWarps = 4;
 constexpr int kDwThreads = kDwWarps * 32;
-constexpr int kCtrlWarp = kDwWarps;
-constexpr int kEpiWarp0 = kCtrlWarp + 4;
+constexpr int kCtrlWarp = 0;
+constexpr int kDwWarp0 = kCtrlWarp + 4;
+constexpr int kEpiWarp0 = kDwWarp0 + kDwWarps;
 constexpr int kFusedThreads = (kEpiWarp0 + kEpiWarps) * 32;
 // Registers per thread after the split.  setmaxnreg.inc can only claim what other warpgroups of the
 // same block released, so the sum must stay within the block's allocation at launch
@@ -58,6 +64,8 @@ constexpr int kRegsLaunch = 80, kRegsDw = 96, kRegsCtrl = 40, kRegsEpi = 56;
 static_assert(kDwThreads * kRegsDw + 128 * kRegsCtrl + kEpiWarps * 32 * kRegsEpi <= kFusedThreads * kRegsLaunch,
               "register split exceeds the block's allocation: setmaxnreg.inc would wait forever");
 constexpr int kMaxSlots = 8, kMaxBUnits = 8;
+constexpr int kBarGate0 = 1;        // named barriers 1..4: a group's gate to its next chunk (two per group, alternating)
+constexpr int kBarChunk0 = 5;       // named barriers 5..8: hand-over of a finished chunk
 
 // Barrier traffic is per warp, not per thread: one lane waits or arrives for its warp.
 __device__ __forceinline__ void warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
@@ -252,7 +260,7 @@ template <int K, int MODE, int S, int PS, bool ZOUT>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __grid_constant__ FusedParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    // a_full[2] a_free[2] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2] | w_full[8] w_free[8]
+    // a_free[4] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2] | w_full[8] w_free[8]
     __shared__ __align__(8) uint64_t bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots + 4 + 2 * kMaxSlots];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -260,9 +268,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t a_s = smem_u32(base);
-    const uint32_t b_s = a_s + 2 * 16384;
+    const uint32_t b_s = a_s + (32768u << P.spg_shift);   // one or two operand stages per depthwise group
     const uint32_t x_s = b_s + (uint32_t)P.nsb * P.unit_bytes;
-    const uint32_t bar_afull = smem_u32(&bars[0]), bar_afree = smem_u32(&bars[2]);
+    const uint32_t bar_afree = smem_u32(&bars[0]);
     const uint32_t bar_bfull = smem_u32(&bars[4]), bar_bfree = smem_u32(&bars[4 + kMaxBUnits]);
     const uint32_t bar_xfull = smem_u32(&bars[4 + 2 * kMaxBUnits]);
     const uint32_t bar_xfree = smem_u32(&bars[4 + 2 * kMaxBUnits + kMaxSlots]);
@@ -275,9 +283,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
 
     if (tid == 0) {
         abort_flag = 0;
+        for (int i = 0; i < 4; ++i) mbar_init(bar_afree + 8 * i, ZOUT ? kEpiWarps : 1);
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_afull + 8 * i, 1);
-            mbar_init(bar_afree + 8 * i, ZOUT ? kEpiWarps : 1);
             mbar_init(bar_accfull + 8 * i, 1);
             mbar_init(bar_accfree + 8 * i, kEpiWarps);
         }
@@ -301,30 +308,42 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const int total_chunks = my_tiles * P.nchunks;
     const int tiles_hw = P.tiles_h * P.tiles_w;
 
-    if (warp >= kCtrlWarp && warp < kEpiWarp0) {
+    if (warp < kDwWarp0) {
         regs_dec<kRegsCtrl>();
         const int units_per_tile = P.nchunks * P.nhalf;
         const int total_units = my_tiles * units_per_tile;
         const int rows0 = P.Dpad > 256 ? 256 : P.Dpad, rows1 = P.Dpad - rows0;
-        if (!ZOUT && warp == kCtrlWarp && lane == 0) {
-            // ---------------- MMA issue (one thread) ----------------
+        if (!ZOUT && warp == kCtrlWarp) {
+            // ---------------- MMA warp ----------------
+            // All 32 lanes walk the loop in step (waits and barriers included); the single-thread instructions
+            // are predicated on lane 0.  The warp releases a chunk's filter block and input box as well: the
+            // hand-over barrier tells it that every depthwise thread is done reading them.
+            const bool one = lane == 0;
             const bool a_mn = !P.a_kmajor;
             const uint64_t adesc0 = a_mn ? make_sdesc(a_s, 1024, 2048) : make_sdesc(a_s, 16, 1024);
             const uint64_t bdesc0 = make_sdesc(b_s, 16, 1024);
             const uint32_t a_step = a_mn ? (4096u >> 4) : (32u >> 4);     // descriptor advance per K step of 16
             const uint32_t idesc0 = make_idesc(rows0, a_mn), idesc1 = make_idesc(rows1 > 0 ? rows1 : 16, a_mn);
-            uint32_t sa = 0, pa = 0;          // intermediate-tile stage and its phase parity
             uint32_t sb = 0, pb = 0;          // weight-ring slot and its phase parity
+            uint32_t wslot = 0;               // filter-ring slot of the chunk
+            uint32_t xs_cur = 0, xs_next = 0; // input slot of the chunk's box; slot the next box will take
+            int gq = 0;
             for (int tl = 0; tl < my_tiles; ++tl) {
                 const int buf = tl % P.nacc;
                 if (tl >= P.nacc)
                     mbar_wait(bar_accfree + 8 * buf, ((tl / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
-                tc_fence_after();
-                for (int q = 0; q < P.nchunks; ++q) {
-                    // the weights arrive long before the intermediate tile: take that wait off the critical path
-                    mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
-                    mbar_wait(bar_afull + 8 * sa, pa, &abort_flag, P.status, kStatusWaitOperand);
+                for (int q = 0; q < P.nchunks; ++q, ++gq) {
+                    const int flags = meta_tab[q].y;
+                    if (flags & 4) { xs_cur = xs_next; if (++xs_next == (uint32_t)P.nslots) xs_next = 0; }
+                    // chunk gq is the (gq >> 1)-th chunk of group gq & 1, which cycles through its own stages
+                    const uint32_t sa = ((uint32_t)(gq & 1) << P.spg_shift) + ((uint32_t)(gq >> 1) & ((1u << P.spg_shift) - 1u));
                     const uint64_t adesc = adesc0 + (uint64_t)(sa * (16384u >> 4));
+                    mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);   // long there
+                    named_bar_sync(kBarChunk0 + (gq & 3), kDwGroupWarps * 32 + 32);   // the group has written chunk gq
+                    mbar_arrive_if(one, bar_wfree + 8 * wslot);
+                    mbar_arrive_if(one && (flags & 1), bar_xfree + 8 * xs_cur);
+                    mbar_arrive_if(one && (flags & 2), bar_xfree + 8 * xs_cur);
+                    if (++wslot == (uint32_t)P.nwslots) wslot = 0;
                     for (int h = 0; h < P.nhalf; ++h) {
                         if (h > 0) mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
                         tc_fence_after();
@@ -333,16 +352,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                         const uint32_t idesc = h ? idesc1 : idesc0;
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
-                            umma_bf16(d_tmem, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * 2), idesc,
-                                      (q == 0 && ks == 0) ? 0u : 1u);
-                        umma_commit(bar_bfree + 8 * sb);
+                            umma_bf16_if(one, d_tmem, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * 2), idesc,
+                                         (q == 0 && ks == 0) ? 0u : 1u);
+                        umma_commit_if(one, bar_bfree + 8 * sb);
                         if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
                     }
-                    umma_commit(bar_afree + 8 * sa);
-                    sa ^= 1;
-                    if (sa == 0) pa ^= 1;
+                    umma_commit_if(one, bar_afree + 8 * sa);
+                    umma_commit_if(one && q == P.nchunks - 1, bar_accfull + 8 * buf);
                 }
-                umma_commit(bar_accfull + 8 * buf);
             }
         } else if (!ZOUT && warp == kCtrlWarp + 1 && lane == 0) {
             // ---------------- pointwise-weight loader (one thread): ring of nsb units ----------------
@@ -386,6 +403,35 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     if (++wslot == (uint32_t)P.nwslots) { wslot = 0; wpar ^= 1; }
                 }
             }
+        } else if (warp == kCtrlWarp + 3) {
+            // ---------------- gate warp ----------------
+            // Waits, chunk by chunk, until the chunk's filters and input box have landed and its operand stage
+            // is free again, then arrives at the group's gate barrier, where the depthwise threads wait: they
+            // never poll a shared-memory barrier themselves.  A gate barrier (two per group, alternating) is
+            // used again two chunks of the group later; by then the stage wait has shown that the group is
+            // past its earlier use.
+            uint32_t wslot = 0, wpar = 0;
+            uint32_t xs_cur = 0, xp_cur = 0, xs_next = 0, xp_next = 0;   // box slot and the parity of its "full" phase
+            int gq = 0;
+            for (int tl = 0; tl < my_tiles; ++tl) {
+                for (int q = 0; q < P.nchunks; ++q, ++gq) {
+                    const int flags = meta_tab[q].y;
+                    const int g = gq & 1, k = gq >> 1;
+                    mbar_wait(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
+                    if (flags & 4) {
+                        xs_cur = xs_next; xp_cur = xp_next;
+                        if (++xs_next == (uint32_t)P.nslots) { xs_next = 0; xp_next ^= 1; }
+                        mbar_wait(bar_xfull + 8 * xs_cur, xp_cur, &abort_flag, P.status, kStatusWaitOperand);
+                    }
+                    if ((k >> P.spg_shift) >= 1) {
+                        const uint32_t sa = ((uint32_t)g << P.spg_shift) + ((uint32_t)k & ((1u << P.spg_shift) - 1u));
+                        mbar_wait(bar_afree + 8 * sa, ((k >> P.spg_shift) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                    }
+                    __threadfence_block();
+                    named_bar_arrive(kBarGate0 + 2 * g + (k & 1), kDwGroupWarps * 32 + 32);
+                    if (++wslot == (uint32_t)P.nwslots) { wslot = 0; wpar ^= 1; }
+                }
+            }
         }
     } else if (warp >= kEpiWarp0) {
         // ---------------- epilogue warps: TMEM -> registers -> bias / ReLU -> bf16 -> global ----------------
@@ -396,7 +442,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int tn = r / hw;
         const int rem = r - tn * hw;
         const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
-        uint32_t sa = 0, pa = 0;                          // ZOUT: stage and phase parity of the next finished chunk
+        int wq = 0;                                       // ZOUT: running index of the next finished chunk
+        uint32_t zslot = 0;                               // ZOUT: its filter-ring slot
         for (int tl = 0; tl < my_tiles; ++tl) {
             int tile = (int)blockIdx.x + tl * (int)gridDim.x;
             const int bn = tile / tiles_hw;
@@ -407,8 +454,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D;
             if (ZOUT) {
                 // this thread's pixel row of every finished stage goes to z (row r of the stage: 128 bytes, swizzled)
-                for (int q = 0; q < P.nchunks; ++q) {
-                    warp_wait(bar_afull + 8 * sa, pa, &abort_flag, P.status, kStatusWaitOperand);
+                for (int q = 0; q < P.nchunks; ++q, ++wq) {
+                    named_bar_sync(kBarChunk0 + (wq & 3), kDwGroupWarps * 32 + kEpiWarps * 32);   // chunk wq is written
+                    if (warp == kEpiWarp0 && lane == 0) {
+                        const int flags = meta_tab[q].y;
+                        const uint32_t xslot = xinfo[zslot] & 0xffu;
+                        mbar_arrive(bar_wfree + 8 * zslot);
+                        if (flags & 1) mbar_arrive(bar_xfree + 8 * xslot);
+                        if (flags & 2) mbar_arrive(bar_xfree + 8 * xslot);
+                    }
+                    __syncwarp();
+                    if (++zslot == (uint32_t)P.nwslots) zslot = 0;
+                    const uint32_t sa = ((uint32_t)(wq & 1) << P.spg_shift) + ((uint32_t)(wq >> 1) & ((1u << P.spg_shift) - 1u));
                     const uint32_t row_s = a_s + sa * 16384 + (uint32_t)r * 128;
                     uint4 v[8];
 #pragma unroll
@@ -419,8 +476,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
 #pragma unroll
                         for (int c = 0; c < 8; ++c) dst[c] = v[c];
                     }
-                    sa ^= 1;
-                    if (sa == 0) pa ^= 1;
                 }
                 continue;
             }
@@ -440,33 +495,25 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     } else {
         // ---------------- depthwise warps: group g takes the chunks gq = g, g+2, ... ----------------
         regs_inc<kRegsDw>();
-        const int g = warp >> 3;
-        const int il = tid & 63, run = (tid >> 6) & 3;
-        const uint32_t a_stage = a_s + g * 16384;
+        const int dt = tid - kDwWarp0 * 32;               // index among the depthwise threads
+        const int g = dt >> 8;
+        const int il = dt & 63, run = (dt >> 6) & 3;
         int q = g;
         while (q >= P.nchunks) q -= P.nchunks;
         int wslot = g;
-        uint32_t wpar = 0;
-        while (wslot >= P.nwslots) { wslot -= P.nwslots; wpar ^= 1; }
-        // Only one thread of a group touches the shared-memory barriers; the group's 256 threads meet at a
-        // hardware named barrier (id 1 + g) before and after a chunk's arithmetic.  (Barrier operations of
-        // all 16 warps would queue behind the other group's shared-memory loads.)
-        const bool leader = (tid & (kDwGroupWarps * 32 - 1)) == 0;
+        while (wslot >= P.nwslots) wslot -= P.nwslots;
+        // The depthwise threads touch no shared-memory barrier: they wait at the group's gate barrier for the
+        // gate warp, and after a chunk's arithmetic they arrive, without waiting, at the chunk's hand-over
+        // barrier, where the consumer waits.  (Barrier operations of 16 warps would queue behind the other
+        // group's shared-memory loads.)  A hand-over barrier is used again four chunks later, by the same group
+        // and for the same stage (two chunks later with one stage per group); by then the gate warp has seen
+        // that stage released, hence the consumer past the barrier.
         for (int gq = g, k = 0; gq < total_chunks; gq += 2, ++k) {
-            const int flags = meta_tab[q].y;
             const bool live_i = q * kChunk + il < P.G;
-            if (leader) {
-                mbar_wait(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
-                if (flags & 8) {   // first or second chunk of its box: later ones follow one of these in the same group
-                    const uint32_t xi0 = xinfo[wslot];
-                    mbar_wait(bar_xfull + 8 * (xi0 & 0xffu), xi0 >> 8, &abort_flag, P.status, kStatusWaitOperand);
-                }
-                if (k >= 1) mbar_wait(bar_afree + 8 * g, (k - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
-            }
-            named_bar_sync(1 + g, kDwGroupWarps * 32);
-            const uint32_t xi = xinfo[wslot];
-            const int xslot = (int)(xi & 0xffu);
-            const uint32_t xs = x_s + xslot * (uint32_t)P.slot_bytes;
+            const uint32_t sa = ((uint32_t)g << P.spg_shift) + ((uint32_t)k & ((1u << P.spg_shift) - 1u));   // this chunk's stage
+            const uint32_t a_stage = a_s + sa * 16384;
+            named_bar_sync(kBarGate0 + 2 * g + (k & 1), kDwGroupWarps * 32 + 32);
+            const uint32_t xs = x_s + (xinfo[wslot] & 0xffu) * (uint32_t)P.slot_bytes;
             const uint32_t wsm = w_s + wslot * wblock + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
             float w[9];
             int clb;                                      // channel index inside the staged box
@@ -483,17 +530,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             else if (MODE == 2) dw_quads_k3<S, PS>(P, xs, clb, w, il, run, live_i, a_stage);
             else dw_generic<K>(P, xs, clb, wsm, il, run, live_i, a_stage);
             fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
-            named_bar_sync(1 + g, kDwGroupWarps * 32);
-            if (leader) {
-                mbar_arrive(bar_afull + 8 * g);
-                mbar_arrive(bar_wfree + 8 * wslot);
-                if (flags & 1) mbar_arrive(bar_xfree + 8 * xslot);
-                if (flags & 2) mbar_arrive(bar_xfree + 8 * xslot);
-            }
+            __threadfence_block();
+            named_bar_arrive(kBarChunk0 + (gq & 3), kDwGroupWarps * 32 + (ZOUT ? kEpiWarps * 32 : 32));
             q += 2;
             while (q >= P.nchunks) q -= P.nchunks;
             wslot += 2;
-            while (wslot >= P.nwslots) { wslot -= P.nwslots; wpar ^= 1; }
+            while (wslot >= P.nwslots) wslot -= P.nwslots;
         }
     }
     tc_fence_before();
@@ -574,6 +616,7 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     P.relu = p->opt_relu;
     P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
     P.IH = t.IH; P.IW = t.IW; P.ps = t.cbox * 2; P.nslots = t.nslots; P.nwslots = t.nwslots; P.nboxes = p->nboxes; P.nsb = t.nsb; P.wstride = p->wstride;
+    P.spg_shift = t.spg == 2 ? 1 : 0;
     P.box_bytes = t.box_bytes; P.slot_bytes = t.slot_bytes;
     P.nhalf = p->Dpad > 256 ? 2 : 1;
     P.unit_bytes = (p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;

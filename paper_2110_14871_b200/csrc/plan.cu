@@ -112,13 +112,13 @@ gdws_status_t ensure_device(gdws_plan_s *p)
 
 static int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-// Shared-memory layout of the fused bf16 kernel: two intermediate-tile stages, a ring of `nsb`
+// Shared-memory layout of the fused bf16 kernel: 2 * t.spg intermediate-tile stages, a ring of `nsb`
 // pointwise-weight units (a unit = one K chunk x up to 256 output channels, at most 32 KB) and
 // `nslots` staged-input slots (one TMA box plus the chunk's filters).  Fills t.nsb / t.nslots /
 // t.smem; false if it cannot fit.  Prefers at least 3 chunks of weights and 4 input slots in flight.
 static bool fit_smem(const gdws_plan_s *p, Tile &t)
 {
-    const size_t a = 2 * (size_t)kTileRows * kChunk * 2;
+    const size_t a = 2 * (size_t)t.spg * kTileRows * kChunk * 2;
     const int nhalf = p->Dpad > 256 ? 2 : 1;
     const size_t unit = (size_t)(p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
     const size_t slot = (size_t)t.slot_bytes;
@@ -179,10 +179,13 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
                 t.cbox = cbox;
                 t.box_bytes = TN * t.IH * t.IW * cbox * 2;
                 t.slot_bytes = round_up(t.box_bytes, 128);
-                if (!fit_smem(p, t)) continue;
-                const double tiles = (double)t.tiles();
-                const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IW) * (t.fast ? 1.0 : 4.0) - 1e-3 * PW;
-                if (cost < best) { best = cost; *out = t; found = true; }
+                for (int spg = 2; spg >= 1; --spg) {     // one operand stage per group costs some overlap
+                    t.spg = spg;
+                    if (!fit_smem(p, t)) continue;
+                    const double tiles = (double)t.tiles();
+                    const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IW) * (t.fast ? 1.0 : 4.0) * (spg == 1 ? 1.08 : 1.0) - 1e-3 * PW;
+                    if (cost < best) { best = cost; *out = t; found = true; }
+                }
             }
         }
     }
@@ -270,7 +273,7 @@ gdws_status_t gdws_plan(int C, int D, int k, int stride, int pad, const int32_t 
         for (int cb = 32; cb <= 128; cb *= 2) {
             if (cb < p->span_max) continue;
             if (cb > 64 && best_cost >= 0) break;
-            if (cb > 32 && best_cost >= 0 && p->Dpad > 256) break;   // wide layers: shared memory goes to the weight ring
+            if (cb > 32 && best_cost >= 0 && p->Dpad >= 256) break;   // wide layers: shared memory goes to the weight ring
             int nb = 0;
             for (int q = 0; q < p->nchunks;) {
                 const int cbase = p->chunk_c0[q] & ~7;
