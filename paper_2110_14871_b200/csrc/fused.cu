@@ -19,9 +19,11 @@
 //     next chunk at once;
 //   * weight loader (one thread): streams the pre-swizzled pointwise weights (bulk copies with
 //     mbarrier completion, a ring of units of at most 256 output channels x 64);
-//   * MMA warp: waits on that named barrier chunk by chunk, releases the chunk's filter block and
-//     input box, and one lane issues tcgen05.mma into a TMEM accumulator (128 lanes x D fp32 columns;
-//     two accumulators when D <= 256, so that a tile's epilogue overlaps the next tile's main loop);
+//   * gate warp: waits for a chunk's filters, input box and free operand stage and opens the group's
+//     gate barrier, so that no depthwise thread ever polls a shared-memory barrier;
+//   * MMA warp: waits on the hand-over barrier chunk by chunk, and one lane issues tcgen05.mma into a
+//     TMEM accumulator (128 lanes x D fp32 columns; two accumulators when D <= 256, so that a tile's
+//     epilogue overlaps the next tile's main loop);
 //   * 4 epilogue warps: read the finished accumulator (tcgen05.ld), add the bias, apply the
 //     optional ReLU, round to bf16 and store y.
 // Every wait is bounded; a wait that runs out raises a block-wide abort flag that turns all later
@@ -48,7 +50,7 @@ struct alignas(64) FusedParams {
 };
 
 // Warp roles, in warpgroups of 4 so that registers can be moved between the roles (setmaxnreg):
-// warp 0 MMA issue, 1 weight loader, 2 input loader (3 idle), 4-19 depthwise (two groups of 8),
+// warp 0 MMA issue, 1 weight loader, 2 input loader, 3 gate, 4-19 depthwise (two groups of 8),
 // 20-23 epilogue.  The control warps come first: the schedulers favour a block's oldest warps, and a
 // control lane that has to queue behind the depthwise warps' instruction streams stalls the pipeline.
 constexpr int kDwWarps = 16, kDwGroupWarps = 8, kEpiWarps = 4;
@@ -291,9 +293,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         for (int i = 0; i < kMaxBUnits; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
         for (int i = 0; i < kMaxSlots; ++i) {
             mbar_init(bar_xfull + 8 * i, 1);
-            mbar_init(bar_xfree + 8 * i, 2);                   // the last two chunks that use a box release it
+            mbar_init(bar_xfree + 8 * i, 2 * kDwGroupWarps);   // the last two chunks that use a box release it, warp by warp
             mbar_init(bar_wfull + 8 * i, 1);
-            mbar_init(bar_wfree + 8 * i, 1);
+            mbar_init(bar_wfree + 8 * i, kDwGroupWarps);
         }
         fence_mbar_init();
     }
@@ -315,50 +317,59 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int rows0 = P.Dpad > 256 ? 256 : P.Dpad, rows1 = P.Dpad - rows0;
         if (!ZOUT && warp == kCtrlWarp) {
             // ---------------- MMA warp ----------------
-            // All 32 lanes walk the loop in step (waits and barriers included); the single-thread instructions
-            // are predicated on lane 0.  The warp releases a chunk's filter block and input box as well: the
-            // hand-over barrier tells it that every depthwise thread is done reading them.
-            const bool one = lane == 0;
+            // All 32 lanes wait for the weights and at the chunk's hand-over barrier; lane 0 then issues the
+            // chunk's MMAs and commits.  Its per-chunk instruction stream is kept as short as possible (32-bit
+            // descriptor words, no table lookups): the pipeline cannot run faster than this one lane.
             const bool a_mn = !P.a_kmajor;
             const uint64_t adesc0 = a_mn ? make_sdesc(a_s, 1024, 2048) : make_sdesc(a_s, 16, 1024);
             const uint64_t bdesc0 = make_sdesc(b_s, 16, 1024);
+            const uint32_t a_lo0 = (uint32_t)adesc0, a_hi = (uint32_t)(adesc0 >> 32);
+            const uint32_t b_lo0 = (uint32_t)bdesc0, b_hi = (uint32_t)(bdesc0 >> 32);
             const uint32_t a_step = a_mn ? (4096u >> 4) : (32u >> 4);     // descriptor advance per K step of 16
+            const uint32_t b_unit = (uint32_t)P.unit_bytes >> 4;
             const uint32_t idesc0 = make_idesc(rows0, a_mn), idesc1 = make_idesc(rows1 > 0 ? rows1 : 16, a_mn);
+            const uint32_t spg_mask = (1u << P.spg_shift) - 1u;
             uint32_t sb = 0, pb = 0;          // weight-ring slot and its phase parity
-            uint32_t wslot = 0;               // filter-ring slot of the chunk
-            uint32_t xs_cur = 0, xs_next = 0; // input slot of the chunk's box; slot the next box will take
-            int gq = 0;
+            uint32_t gq = 0;
             for (int tl = 0; tl < my_tiles; ++tl) {
                 const int buf = tl % P.nacc;
+                const uint32_t d_tmem = tmem + (uint32_t)(buf * P.acc_cols);
                 if (tl >= P.nacc)
                     mbar_wait(bar_accfree + 8 * buf, ((tl / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
                 for (int q = 0; q < P.nchunks; ++q, ++gq) {
-                    const int flags = meta_tab[q].y;
-                    if (flags & 4) { xs_cur = xs_next; if (++xs_next == (uint32_t)P.nslots) xs_next = 0; }
                     // chunk gq is the (gq >> 1)-th chunk of group gq & 1, which cycles through its own stages
-                    const uint32_t sa = ((uint32_t)(gq & 1) << P.spg_shift) + ((uint32_t)(gq >> 1) & ((1u << P.spg_shift) - 1u));
-                    const uint64_t adesc = adesc0 + (uint64_t)(sa * (16384u >> 4));
+                    const uint32_t sa = ((gq & 1u) << P.spg_shift) + ((gq >> 1) & spg_mask);
+                    const uint32_t a_lo = a_lo0 + sa * (16384u >> 4);
                     mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);   // long there
-                    named_bar_sync(kBarChunk0 + (gq & 3), kDwGroupWarps * 32 + 32);   // the group has written chunk gq
-                    mbar_arrive_if(one, bar_wfree + 8 * wslot);
-                    mbar_arrive_if(one && (flags & 1), bar_xfree + 8 * xs_cur);
-                    mbar_arrive_if(one && (flags & 2), bar_xfree + 8 * xs_cur);
-                    if (++wslot == (uint32_t)P.nwslots) wslot = 0;
-                    for (int h = 0; h < P.nhalf; ++h) {
-                        if (h > 0) mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
+                    named_bar_sync(kBarChunk0 + (int)(gq & 3u), kDwGroupWarps * 32 + 32);   // the group has written chunk gq
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t b_lo = b_lo0 + sb * b_unit;
+                        umma_bf16_words(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc0, q != 0);
+                        umma_bf16_words(d_tmem, a_lo + a_step, a_hi, b_lo + 2, b_hi, idesc0, 1u);
+                        umma_bf16_words(d_tmem, a_lo + 2 * a_step, a_hi, b_lo + 4, b_hi, idesc0, 1u);
+                        umma_bf16_words(d_tmem, a_lo + 3 * a_step, a_hi, b_lo + 6, b_hi, idesc0, 1u);
+                        umma_commit(bar_bfree + 8 * sb);
+                    }
+                    if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
+                    if (P.nhalf == 2) {       // output channels 256 and up: a second weight unit, a second set of columns
+                        mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
                         tc_fence_after();
-                        const uint32_t d_tmem = tmem + (uint32_t)(buf * P.acc_cols + h * 256);
-                        const uint64_t bdesc = bdesc0 + (uint64_t)(sb * ((uint32_t)P.unit_bytes >> 4));
-                        const uint32_t idesc = h ? idesc1 : idesc0;
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            umma_bf16_if(one, d_tmem, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * 2), idesc,
-                                         (q == 0 && ks == 0) ? 0u : 1u);
-                        umma_commit_if(one, bar_bfree + 8 * sb);
+                        if (lane == 0) {
+                            const uint32_t b_lo = b_lo0 + sb * b_unit;
+                            umma_bf16_words(d_tmem + 256, a_lo, a_hi, b_lo, b_hi, idesc1, q != 0);
+                            umma_bf16_words(d_tmem + 256, a_lo + a_step, a_hi, b_lo + 2, b_hi, idesc1, 1u);
+                            umma_bf16_words(d_tmem + 256, a_lo + 2 * a_step, a_hi, b_lo + 4, b_hi, idesc1, 1u);
+                            umma_bf16_words(d_tmem + 256, a_lo + 3 * a_step, a_hi, b_lo + 6, b_hi, idesc1, 1u);
+                            umma_commit(bar_bfree + 8 * sb);
+                        }
                         if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
                     }
-                    umma_commit_if(one, bar_afree + 8 * sa);
-                    umma_commit_if(one && q == P.nchunks - 1, bar_accfull + 8 * buf);
+                    if (lane == 0) {
+                        umma_commit(bar_afree + 8 * sa);
+                        if (q == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
+                    }
+                    __syncwarp();
                 }
             }
         } else if (!ZOUT && warp == kCtrlWarp + 1 && lane == 0) {
@@ -443,7 +454,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int rem = r - tn * hw;
         const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
         int wq = 0;                                       // ZOUT: running index of the next finished chunk
-        uint32_t zslot = 0;                               // ZOUT: its filter-ring slot
         for (int tl = 0; tl < my_tiles; ++tl) {
             int tile = (int)blockIdx.x + tl * (int)gridDim.x;
             const int bn = tile / tiles_hw;
@@ -456,15 +466,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 // this thread's pixel row of every finished stage goes to z (row r of the stage: 128 bytes, swizzled)
                 for (int q = 0; q < P.nchunks; ++q, ++wq) {
                     named_bar_sync(kBarChunk0 + (wq & 3), kDwGroupWarps * 32 + kEpiWarps * 32);   // chunk wq is written
-                    if (warp == kEpiWarp0 && lane == 0) {
-                        const int flags = meta_tab[q].y;
-                        const uint32_t xslot = xinfo[zslot] & 0xffu;
-                        mbar_arrive(bar_wfree + 8 * zslot);
-                        if (flags & 1) mbar_arrive(bar_xfree + 8 * xslot);
-                        if (flags & 2) mbar_arrive(bar_xfree + 8 * xslot);
-                    }
-                    __syncwarp();
-                    if (++zslot == (uint32_t)P.nwslots) zslot = 0;
                     const uint32_t sa = ((uint32_t)(wq & 1) << P.spg_shift) + ((uint32_t)(wq >> 1) & ((1u << P.spg_shift) - 1u));
                     const uint32_t row_s = a_s + sa * 16384 + (uint32_t)r * 128;
                     uint4 v[8];
@@ -513,7 +514,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             const uint32_t sa = ((uint32_t)g << P.spg_shift) + ((uint32_t)k & ((1u << P.spg_shift) - 1u));   // this chunk's stage
             const uint32_t a_stage = a_s + sa * 16384;
             named_bar_sync(kBarGate0 + 2 * g + (k & 1), kDwGroupWarps * 32 + 32);
-            const uint32_t xs = x_s + (xinfo[wslot] & 0xffu) * (uint32_t)P.slot_bytes;
+            const uint32_t xslot = xinfo[wslot] & 0xffu;
+            const uint32_t xs = x_s + xslot * (uint32_t)P.slot_bytes;
             const uint32_t wsm = w_s + wslot * wblock + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
             float w[9];
             int clb;                                      // channel index inside the staged box
@@ -531,6 +533,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             else dw_generic<K>(P, xs, clb, wsm, il, run, live_i, a_stage);
             fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
             __threadfence_block();
+            __syncwarp();
+            if (lane == 0) {          // this warp is done with the chunk's filters and input box
+                const int flags = meta_tab[q].y;
+                mbar_arrive(bar_wfree + 8 * wslot);
+                if (flags & 1) mbar_arrive(bar_xfree + 8 * xslot);
+                if (flags & 2) mbar_arrive(bar_xfree + 8 * xslot);
+            }
+            __syncwarp();
             named_bar_arrive(kBarChunk0 + (gq & 3), kDwGroupWarps * 32 + (ZOUT ? kEpiWarps * 32 : 32));
             q += 2;
             while (q >= P.nchunks) q -= P.nchunks;
