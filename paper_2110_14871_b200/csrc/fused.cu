@@ -133,85 +133,150 @@ __device__ __forceinline__ void store_group(const FusedParams &P, uint32_t a_sta
 // pixel.  Lanes of a warp read different channels of the same pixel, i.e. one or two 32-byte
 // sectors: a single shared-memory wavefront per load.
 
-// ---- depthwise, k = 3, patches at least 8 wide: a thread computes 4 consecutive output rows of one
-// 8-pixel column group, reading each input row once and using it for up to 3 output rows.
-template <int S, int PS>
-__device__ __forceinline__ void dw_rows_k3(const FusedParams &P, uint32_t xs, int clb, const float (&w)[9], int kk,
-                                           int run, bool live_i, uint32_t a_stage)
+// What a depthwise thread needs to know about its share of a tile; none of it changes from chunk to
+// chunk, so it is worked out once per kernel.  The thread owns up to four pixel groups (8 pixels each):
+// `in_off[m]` is where group m's input window starts inside a staged box (bytes, channel 0), `st_off[m]`
+// where its results go inside an operand stage, and bit m of `live` says whether the group has pixels.
+// In a pixel-contiguous stage a group's 8 results are one 16-byte piece at st_off[m]; in a channel-contiguous
+// stage (KMAJOR, the unfused GDW kernel) they are 8 two-byte elements in 8 consecutive 128-byte rows, each
+// in the 16-byte piece (kk/8) ^ (row & 7), and st_off[m] is the address of the first row's unswizzled piece 0.
+struct DwShare {
+    uint32_t in_off[4];
+    uint32_t st_off[4];
+    uint32_t rowb;              // bytes per input row of the staged box
+    uint32_t live;
+    uint32_t kg4;               // KMAJOR: 16 * (kk / 8)
+};
+template <bool KMAJOR>
+__device__ __forceinline__ uint32_t dw_st_off(int o, int kk)
 {
+    return KMAJOR ? (uint32_t)(o * 1024 + (kk & 7) * 2) : a_off_mn(o, kk);
+}
+template <bool KMAJOR>
+__device__ __forceinline__ void store_group_at(uint32_t addr, uint32_t kg4, const float (&v)[8])
+{
+    if (!KMAJOR) {
+        uint4 q;
+        q.x = pack_bf16x2(v[0], v[1]); q.y = pack_bf16x2(v[2], v[3]);
+        q.z = pack_bf16x2(v[4], v[5]); q.w = pack_bf16x2(v[6], v[7]);
+        sts128(addr, q);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sts16(addr + (uint32_t)(e * 128) + (kg4 ^ (uint32_t)(e << 4)), float_to_bf16_bits(v[e]));
+    }
+}
+
+// ---- depthwise, k = 3, patches at least 8 wide: a thread computes 4 consecutive output rows of one
+// 8-pixel column group (its four pixel groups), reading each input row once and using it for up to 3
+// output rows.
+template <int S, int PS, bool KMAJOR>
+__device__ __forceinline__ DwShare dw_rows_share(const FusedParams &P, int kk, int run)
+{
+    DwShare sh;
     const int nseg = P.PW >> 3;
     const int seg = run % nseg;
     const int R0 = (run / nseg) * 4;               // first of the 4 rows (row index = tn*PH + ph)
     const int o0 = R0 * nseg + seg;
+    const int tn = R0 / P.PH, ph0 = R0 - tn * P.PH;
+    sh.rowb = (uint32_t)P.IW * PS;
+    sh.live = R0 < P.TN * P.PH ? 1u : 0u;
+    sh.in_off[0] = (uint32_t)((tn * P.IH + ph0 * S) * P.IW + seg * 8 * S) * PS;
+#pragma unroll
+    for (int ro = 0; ro < 4; ++ro) sh.st_off[ro] = dw_st_off<KMAJOR>(o0 + ro * nseg, kk);
+    sh.kg4 = (uint32_t)(kk >> 3) << 4;
+    return sh;
+}
+template <int S, int PS, bool KMAJOR>
+__device__ __forceinline__ void dw_rows_k3(const DwShare &sh, uint32_t xs, int clb, const float (&w)[9], bool live_i,
+                                           uint32_t a_stage)
+{
     float acc[4][8];
-#pragma unroll
-    for (int ro = 0; ro < 4; ++ro)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[ro][e] = 0.f;
-    if (live_i && R0 < P.TN * P.PH) {
-        const int tn = R0 / P.PH, ph0 = R0 - tn * P.PH;
-        const uint32_t rowb = (uint32_t)P.IW * PS;
-        const uint32_t base = xs + (uint32_t)((tn * P.IH + ph0 * S) * P.IW + seg * 8 * S) * PS + (uint32_t)clb * 2;
+    if (live_i && sh.live) {
+        const uint32_t base = xs + sh.in_off[0] + (uint32_t)clb * 2;
         constexpr int NR = 3 * S + 3;
         constexpr int NX = 7 * S + 3;
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
             float xr[NX];
 #pragma unroll
-            for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * rowb + j * PS);
+            for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * sh.rowb + j * PS);
 #pragma unroll
             for (int ro = 0; ro < 4; ++ro) {
                 const int u = r - ro * S;
                 if (u >= 0 && u < 3) {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e)
-#pragma unroll
-                        for (int v = 0; v < 3; ++v) acc[ro][e] = fmaf(w[u * 3 + v], xr[e * S + v], acc[ro][e]);
+                    for (int e = 0; e < 8; ++e) {
+                        // the first tap starts the sum
+                        float a = u == 0 ? w[0] * xr[e * S] : fmaf(w[u * 3], xr[e * S], acc[ro][e]);
+                        a = fmaf(w[u * 3 + 1], xr[e * S + 1], a);
+                        acc[ro][e] = fmaf(w[u * 3 + 2], xr[e * S + 2], a);
+                    }
                 }
             }
         }
+    } else {
+#pragma unroll
+        for (int ro = 0; ro < 4; ++ro)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[ro][e] = 0.f;
     }
 #pragma unroll
-    for (int ro = 0; ro < 4; ++ro) store_group(P, a_stage, o0 + ro * nseg, kk, acc[ro]);
+    for (int ro = 0; ro < 4; ++ro) store_group_at<KMAJOR>(a_stage + sh.st_off[ro], sh.kg4, acc[ro]);
 }
 
 // ---- depthwise, k = 3, 4-wide patches: a pixel group is 2 output rows x 4 columns of one image.
-template <int S, int PS>
-__device__ __forceinline__ void dw_quads_k3(const FusedParams &P, uint32_t xs, int clb, const float (&w)[9], int kk,
-                                            int run, bool live_i, uint32_t a_stage)
+template <int S, int PS, bool KMAJOR>
+__device__ __forceinline__ DwShare dw_quads_share(const FusedParams &P, int kk, int run)
 {
+    DwShare sh;
     const int gpi = P.PH >> 1;                      // pixel groups per image
-#pragma unroll 1
+    sh.rowb = (uint32_t)P.IW * PS;
+    sh.live = 0;
+#pragma unroll
     for (int m = 0; m < 4; ++m) {
         const int o = run * 4 + m;
-        float acc[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] = 0.f;
         const int tn = o / gpi, ph0 = (o - tn * gpi) * 2;
-        if (live_i && tn < P.TN) {
-            const uint32_t rowb = (uint32_t)P.IW * PS;
-            const uint32_t base = xs + (uint32_t)((tn * P.IH + ph0 * S) * P.IW) * PS + (uint32_t)clb * 2;
+        if (tn < P.TN) sh.live |= 1u << m;
+        sh.in_off[m] = (uint32_t)((tn * P.IH + ph0 * S) * P.IW) * PS;
+        sh.st_off[m] = dw_st_off<KMAJOR>(o, kk);
+    }
+    sh.kg4 = (uint32_t)(kk >> 3) << 4;
+    return sh;
+}
+template <int S, int PS, bool KMAJOR>
+__device__ __forceinline__ void dw_quads_k3(const DwShare &sh, uint32_t xs, int clb, const float (&w)[9], bool live_i,
+                                            uint32_t a_stage)
+{
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+        float acc[8];
+        if (live_i && ((sh.live >> m) & 1u)) {
+            const uint32_t base = xs + sh.in_off[m] + (uint32_t)clb * 2;
             constexpr int NR = S + 3;               // input rows feeding 2 output rows
             constexpr int NX = 3 * S + 3;           // input columns feeding 4 output columns
 #pragma unroll
             for (int r = 0; r < NR; ++r) {
                 float xr[NX];
 #pragma unroll
-                for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * rowb + j * PS);
+                for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * sh.rowb + j * PS);
 #pragma unroll
                 for (int ro = 0; ro < 2; ++ro) {
                     const int u = r - ro * S;
                     if (u >= 0 && u < 3) {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-#pragma unroll
-                            for (int v = 0; v < 3; ++v)
-                                acc[ro * 4 + e] = fmaf(w[u * 3 + v], xr[e * S + v], acc[ro * 4 + e]);
+                        for (int e = 0; e < 4; ++e) {
+                            float a = u == 0 ? w[0] * xr[e * S] : fmaf(w[u * 3], xr[e * S], acc[ro * 4 + e]);
+                            a = fmaf(w[u * 3 + 1], xr[e * S + 1], a);
+                            acc[ro * 4 + e] = fmaf(w[u * 3 + 2], xr[e * S + 2], a);
+                        }
                     }
                 }
             }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
         }
-        store_group(P, a_stage, o, kk, acc);
+        store_group_at<KMAJOR>(a_stage + sh.st_off[m], sh.kg4, acc);
     }
 }
 
@@ -317,7 +382,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int rows0 = P.Dpad > 256 ? 256 : P.Dpad, rows1 = P.Dpad - rows0;
         if (!ZOUT && warp == kCtrlWarp) {
             // ---------------- MMA warp ----------------
-            // All 32 lanes wait for the weights and at the chunk's hand-over barrier; lane 0 then issues the
+            // All 32 lanes wait for the weights and at the chunk's hand-over barrier; one elected lane then issues the
             // chunk's MMAs and commits.  Its per-chunk instruction stream is kept as short as possible (32-bit
             // descriptor words, no table lookups): the pipeline cannot run faster than this one lane.
             const bool a_mn = !P.a_kmajor;
@@ -343,7 +408,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);   // long there
                     named_bar_sync(kBarChunk0 + (int)(gq & 3u), kDwGroupWarps * 32 + 32);   // the group has written chunk gq
                     tc_fence_after();
-                    if (lane == 0) {
+                    if (elect_one()) {
                         const uint32_t b_lo = b_lo0 + sb * b_unit;
                         umma_bf16_words(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc0, q != 0);
                         umma_bf16_words(d_tmem, a_lo + a_step, a_hi, b_lo + 2, b_hi, idesc0, 1u);
@@ -355,7 +420,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     if (P.nhalf == 2) {       // output channels 256 and up: a second weight unit, a second set of columns
                         mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
                         tc_fence_after();
-                        if (lane == 0) {
+                        if (elect_one()) {
                             const uint32_t b_lo = b_lo0 + sb * b_unit;
                             umma_bf16_words(d_tmem + 256, a_lo, a_hi, b_lo, b_hi, idesc1, q != 0);
                             umma_bf16_words(d_tmem + 256, a_lo + a_step, a_hi, b_lo + 2, b_hi, idesc1, 1u);
@@ -365,7 +430,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                         }
                         if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
                     }
-                    if (lane == 0) {
+                    if (elect_one()) {
                         umma_commit(bar_afree + 8 * sa);
                         if (q == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
                     }
@@ -503,6 +568,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         while (q >= P.nchunks) q -= P.nchunks;
         int wslot = g;
         while (wslot >= P.nwslots) wslot -= P.nwslots;
+        DwShare share = {};
+        if (MODE == 1) share = dw_rows_share<S, PS, ZOUT>(P, il, run);
+        else if (MODE == 2) share = dw_quads_share<S, PS, ZOUT>(P, il, run);
         // The depthwise threads touch no shared-memory barrier: they wait at the group's gate barrier for the
         // gate warp, and after a chunk's arithmetic they arrive, without waiting, at the chunk's hand-over
         // barrier, where the consumer waits.  (Barrier operations of 16 warps would queue behind the other
@@ -528,8 +596,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             } else {
                 clb = (int)lds32(wsm + (uint32_t)(K * K) * 4);
             }
-            if (MODE == 1) dw_rows_k3<S, PS>(P, xs, clb, w, il, run, live_i, a_stage);
-            else if (MODE == 2) dw_quads_k3<S, PS>(P, xs, clb, w, il, run, live_i, a_stage);
+            if (MODE == 1) dw_rows_k3<S, PS, ZOUT>(share, xs, clb, w, live_i, a_stage);
+            else if (MODE == 2) dw_quads_k3<S, PS, ZOUT>(share, xs, clb, w, live_i, a_stage);
             else dw_generic<K>(P, xs, clb, wsm, il, run, live_i, a_stage);
             fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
             __threadfence_block();
