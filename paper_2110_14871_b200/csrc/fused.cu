@@ -66,13 +66,13 @@ constexpr int kRegsLaunch = 80, kRegsDw = 96, kRegsCtrl = 40, kRegsEpi = 56;
 static_assert(kDwThreads * kRegsDw + 128 * kRegsCtrl + kEpiWarps * 32 * kRegsEpi <= kFusedThreads * kRegsLaunch,
               "register split exceeds the block's allocation: setmaxnreg.inc would wait forever");
 constexpr int kMaxSlots = 8, kMaxBUnits = 8;
-constexpr int kBarGate0 = 1;        // named barriers 1..4: a group's gate to its next chunk (two per group, alternating)
+constexpr int kPollNs = 1000;        // longest suspension of one poll by a waiter that runs ahead of the pipeline
 constexpr int kBarChunk0 = 5;       // named barriers 5..8: hand-over of a finished chunk
 
 // Barrier traffic is per warp, not per thread: one lane waits or arrives for its warp.
 __device__ __forceinline__ void warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
 {
-    if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, abort_flag, status, code);
+    if ((threadIdx.x & 31) == 0) mbar_wait_relaxed<kPollNs>(bar, parity, abort_flag, status, code);
     __syncwarp();
 }
 __device__ __forceinline__ void warp_arrive(uint32_t bar)
@@ -327,8 +327,8 @@ template <int K, int MODE, int S, int PS, bool ZOUT>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __grid_constant__ FusedParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    // a_free[4] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2] | w_full[8] w_free[8]
-    __shared__ __align__(8) uint64_t bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots + 4 + 2 * kMaxSlots];
+    // a_free[4] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2] | w_full[8] w_free[8] | open[4]
+    __shared__ __align__(8) uint64_t bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots + 4 + 2 * kMaxSlots + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ uint32_t xinfo[kMaxSlots];      // per filter-ring slot: input slot (bits 0-7) and phase parity (bit 8) of the chunk's box
@@ -344,13 +344,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const uint32_t bar_accfull = smem_u32(&bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots]);
     const uint32_t bar_accfree = bar_accfull + 16;
     const uint32_t bar_wfull = bar_accfull + 32, bar_wfree = bar_wfull + 8 * kMaxSlots;
+    const uint32_t bar_open = bar_wfree + 8 * kMaxSlots;       // a group's next chunk may start (two per group, alternating)
     const uint32_t wblock = (uint32_t)kChunk * P.wstride * 4;             // one chunk's filters
     const uint32_t w_s = x_s + (uint32_t)P.nslots * P.slot_bytes;         // ring of nwslots filter blocks
     int4 *meta_tab = reinterpret_cast<int4 *>(base + (w_s - a_s) + (size_t)P.nwslots * wblock);
 
     if (tid == 0) {
         abort_flag = 0;
-        for (int i = 0; i < 4; ++i) mbar_init(bar_afree + 8 * i, ZOUT ? kEpiWarps : 1);
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(bar_afree + 8 * i, ZOUT ? kEpiWarps : 1);
+            mbar_init(bar_open + 8 * i, 1);
+        }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_accfull + 8 * i, 1);
             mbar_init(bar_accfree + 8 * i, kEpiWarps);
@@ -442,7 +446,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             uint32_t sb = 0, pb = 1;          // parity of the "slot free" phase awaited (first round: nothing to wait for)
             int q = 0, h = 0;
             for (int u = 0; u < total_units; ++u) {
-                if (u >= P.nsb) mbar_wait(bar_bfree + 8 * sb, pb, &abort_flag, P.status, kStatusWaitStage);
+                if (u >= P.nsb) mbar_wait_relaxed<kPollNs>(bar_bfree + 8 * sb, pb, &abort_flag, P.status, kStatusWaitStage);
                 const uint32_t bytes = (uint32_t)(h ? rows1 : rows0) * 128u;
                 mbar_expect_tx(bar_bfull + 8 * sb, bytes);
                 bulk_g2s(b_s + sb * P.unit_bytes, P.pw_img + ((size_t)q * P.Dpad + h * 256) * kChunk, bytes,
@@ -465,14 +469,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 for (int q = 0; q < P.nchunks; ++q, ++gq) {
                     const int4 meta = meta_tab[q];
                     if (meta.y & 4) {         // first chunk of a box: fetch the box
-                        if (gb >= P.nslots) mbar_wait(bar_xfree + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitStage);
+                        if (gb >= P.nslots) mbar_wait_relaxed<kPollNs>(bar_xfree + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitStage);
                         mbar_expect_tx(bar_xfull + 8 * xslot, (uint32_t)P.box_bytes);
                         tma_load_4d(x_s + xslot * (uint32_t)P.slot_bytes, &P.tmap, meta.z, wi0, hi0, n0, bar_xfull + 8 * xslot);
                         cur_x = xslot | ((xpar ^ 1u) << 8);   // "full" phase parity = the opposite of the "free" parity awaited
                         ++gb;
                         if (++xslot == (uint32_t)P.nslots) { xslot = 0; xpar ^= 1; }
                     }
-                    if (gq >= P.nwslots) mbar_wait(bar_wfree + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitStage);
+                    if (gq >= P.nwslots) mbar_wait_relaxed<kPollNs>(bar_wfree + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitStage);
                     xinfo[wslot] = cur_x;                     // published by the arrive below
                     mbar_expect_tx(bar_wfull + 8 * wslot, wblock);
                     bulk_g2s(w_s + wslot * wblock, P.dwpack + (size_t)q * kChunk * P.wstride, wblock, bar_wfull + 8 * wslot);
@@ -482,10 +486,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         } else if (warp == kCtrlWarp + 3) {
             // ---------------- gate warp ----------------
             // Waits, chunk by chunk, until the chunk's filters and input box have landed and its operand stage
-            // is free again, then arrives at the group's gate barrier, where the depthwise threads wait: they
-            // never poll a shared-memory barrier themselves.  A gate barrier (two per group, alternating) is
-            // used again two chunks of the group later; by then the stage wait has shown that the group is
-            // past its earlier use.
+            // is free again, then completes a phase of the group's "open" barrier (two per group, alternating).
+            // Each depthwise warp checks that one barrier before a chunk, on its own: the warps of a group do
+            // not wait for one another.  An "open" barrier is used again two chunks of the group later; by then
+            // the stage wait has shown that every warp of the group is past its earlier use.
             uint32_t wslot = 0, wpar = 0;
             uint32_t xs_cur = 0, xp_cur = 0, xs_next = 0, xp_next = 0;   // box slot and the parity of its "full" phase
             int gq = 0;
@@ -493,18 +497,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 for (int q = 0; q < P.nchunks; ++q, ++gq) {
                     const int flags = meta_tab[q].y;
                     const int g = gq & 1, k = gq >> 1;
-                    mbar_wait(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
+                    mbar_wait_relaxed<kPollNs>(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
                     if (flags & 4) {
                         xs_cur = xs_next; xp_cur = xp_next;
                         if (++xs_next == (uint32_t)P.nslots) { xs_next = 0; xp_next ^= 1; }
-                        mbar_wait(bar_xfull + 8 * xs_cur, xp_cur, &abort_flag, P.status, kStatusWaitOperand);
+                        mbar_wait_relaxed<kPollNs>(bar_xfull + 8 * xs_cur, xp_cur, &abort_flag, P.status, kStatusWaitOperand);
                     }
                     if ((k >> P.spg_shift) >= 1) {
                         const uint32_t sa = ((uint32_t)g << P.spg_shift) + ((uint32_t)k & ((1u << P.spg_shift) - 1u));
-                        mbar_wait(bar_afree + 8 * sa, ((k >> P.spg_shift) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                        mbar_wait_relaxed<kPollNs>(bar_afree + 8 * sa, ((k >> P.spg_shift) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
                     }
-                    __threadfence_block();
-                    named_bar_arrive(kBarGate0 + 2 * g + (k & 1), kDwGroupWarps * 32 + 32);
+                    if (lane == 0) mbar_arrive(bar_open + 8 * (2 * g + (k & 1)));
+                    __syncwarp();
                     if (++wslot == (uint32_t)P.nwslots) { wslot = 0; wpar ^= 1; }
                 }
             }
@@ -571,17 +575,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         DwShare share = {};
         if (MODE == 1) share = dw_rows_share<S, PS, ZOUT>(P, il, run);
         else if (MODE == 2) share = dw_quads_share<S, PS, ZOUT>(P, il, run);
-        // The depthwise threads touch no shared-memory barrier: they wait at the group's gate barrier for the
-        // gate warp, and after a chunk's arithmetic they arrive, without waiting, at the chunk's hand-over
-        // barrier, where the consumer waits.  (Barrier operations of 16 warps would queue behind the other
-        // group's shared-memory loads.)  A hand-over barrier is used again four chunks later, by the same group
+        // A depthwise warp checks one shared-memory barrier per chunk (the group's "open" barrier, kept by the
+        // gate warp), and after the chunk's arithmetic its threads arrive, without waiting, at the chunk's
+        // hand-over barrier, where the consumer waits.  A hand-over barrier is used again four chunks later, by the same group
         // and for the same stage (two chunks later with one stage per group); by then the gate warp has seen
         // that stage released, hence the consumer past the barrier.
         for (int gq = g, k = 0; gq < total_chunks; gq += 2, ++k) {
             const bool live_i = q * kChunk + il < P.G;
             const uint32_t sa = ((uint32_t)g << P.spg_shift) + ((uint32_t)k & ((1u << P.spg_shift) - 1u));   // this chunk's stage
             const uint32_t a_stage = a_s + sa * 16384;
-            named_bar_sync(kBarGate0 + 2 * g + (k & 1), kDwGroupWarps * 32 + 32);
+            if (lane == 0) mbar_wait(bar_open + 8 * (2 * g + (k & 1)), (k >> 1) & 1, &abort_flag, P.status, kStatusWaitOperand);
+            __syncwarp();
             const uint32_t xslot = xinfo[wslot] & 0xffu;
             const uint32_t xs = x_s + xslot * (uint32_t)P.slot_bytes;
             const uint32_t wsm = w_s + wslot * wblock + (uint32_t)(il * P.wstride) * 4;   // this thread's filter

@@ -72,6 +72,31 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     atomicOr(status, code);
 }
+// The same for waiters that run ahead of the pipeline (loaders, the gate warp, epilogue warps): each poll
+// lets the hardware suspend the thread for up to SUSPEND_NS or until the phase completes, so that polling
+// does not take issue slots from the arithmetic warps.
+__device__ __forceinline__ uint32_t mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+    return ok;
+}
+template <int SUSPEND_NS>
+__device__ __forceinline__ void mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+{
+    if (mbar_try_wait(bar, parity)) return;
+    if (*abort_flag) return;
+    for (uint32_t it = 0; it < (1u << 20); ++it) {     // bounded: about a second at a microsecond per poll
+        if (mbar_try_wait_suspend(bar, parity, SUSPEND_NS)) return;
+        if ((it & 63) == 63 && *abort_flag) return;
+    }
+    *abort_flag = 1;
+    atomicOr(status, code);
+}
 // Same, but ignores the abort flag (used in teardown to drain copies that are in flight).
 __device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity)
 {
