@@ -166,8 +166,8 @@ __device__ __forceinline__ void store_group_at(uint32_t addr, uint32_t kg4, cons
     }
 }
 
-// ---- depthwise, k = 3, patches at least 8 wide: a thread computes 4 consecutive output rows of one
-// 8-pixel column group (its four pixel groups), reading each input row once and using it for up to 3
+// ---- depthwise, k = 3 or 5, patches at least 8 wide: a thread computes 4 consecutive output rows of one
+// 8-pixel column group (its four pixel groups), reading each input row once and using it for up to K
 // output rows.
 template <int S, int PS, bool KMAJOR>
 __device__ __forceinline__ DwShare dw_rows_share(const FusedParams &P, int kk, int run)
@@ -186,15 +186,15 @@ __device__ __forceinline__ DwShare dw_rows_share(const FusedParams &P, int kk, i
     sh.kg4 = (uint32_t)(kk >> 3) << 4;
     return sh;
 }
-template <int S, int PS, bool KMAJOR>
-__device__ __forceinline__ void dw_rows_k3(const DwShare &sh, uint32_t xs, int clb, const float (&w)[9], bool live_i,
-                                           uint32_t a_stage)
+template <int K, int S, int PS, bool KMAJOR>
+__device__ __forceinline__ void dw_rows(const DwShare &sh, uint32_t xs, int clb, const float (&w)[K * K], bool live_i,
+                                        uint32_t a_stage)
 {
     float acc[4][8];
     if (live_i && sh.live) {
         const uint32_t base = xs + sh.in_off[0] + (uint32_t)clb * 2;
-        constexpr int NR = 3 * S + 3;
-        constexpr int NX = 7 * S + 3;
+        constexpr int NR = 3 * S + K;
+        constexpr int NX = 7 * S + K;
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
             float xr[NX];
@@ -203,13 +203,14 @@ __device__ __forceinline__ void dw_rows_k3(const DwShare &sh, uint32_t xs, int c
 #pragma unroll
             for (int ro = 0; ro < 4; ++ro) {
                 const int u = r - ro * S;
-                if (u >= 0 && u < 3) {
+                if (u >= 0 && u < K) {
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         // the first tap starts the sum
-                        float a = u == 0 ? w[0] * xr[e * S] : fmaf(w[u * 3], xr[e * S], acc[ro][e]);
-                        a = fmaf(w[u * 3 + 1], xr[e * S + 1], a);
-                        acc[ro][e] = fmaf(w[u * 3 + 2], xr[e * S + 2], a);
+                        float a = u == 0 ? w[0] * xr[e * S] : fmaf(w[u * K], xr[e * S], acc[ro][e]);
+#pragma unroll
+                        for (int v = 1; v < K; ++v) a = fmaf(w[u * K + v], xr[e * S + v], a);
+                        acc[ro][e] = a;
                     }
                 }
             }
@@ -589,19 +590,24 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             const uint32_t xslot = xinfo[wslot] & 0xffu;
             const uint32_t xs = x_s + xslot * (uint32_t)P.slot_bytes;
             const uint32_t wsm = w_s + wslot * wblock + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
-            float w[9];
+            float w[K * K];
             int clb;                                      // channel index inside the staged box
             if (MODE != 0) {
-                const uint4 w0 = lds128(wsm), w1 = lds128(wsm + 16), w2 = lds128(wsm + 32);
-                w[0] = __uint_as_float(w0.x); w[1] = __uint_as_float(w0.y); w[2] = __uint_as_float(w0.z);
-                w[3] = __uint_as_float(w0.w); w[4] = __uint_as_float(w1.x); w[5] = __uint_as_float(w1.y);
-                w[6] = __uint_as_float(w1.z); w[7] = __uint_as_float(w1.w); w[8] = __uint_as_float(w2.x);
-                clb = (int)w2.y;
+                constexpr int NV = (K * K + 4) / 4;       // 16-byte pieces holding the taps and the channel index
+                uint32_t wv[NV * 4];
+#pragma unroll
+                for (int j = 0; j < NV; ++j) {
+                    const uint4 t = lds128(wsm + 16 * j);
+                    wv[4 * j] = t.x; wv[4 * j + 1] = t.y; wv[4 * j + 2] = t.z; wv[4 * j + 3] = t.w;
+                }
+#pragma unroll
+                for (int j = 0; j < K * K; ++j) w[j] = __uint_as_float(wv[j]);
+                clb = (int)wv[K * K];
             } else {
                 clb = (int)lds32(wsm + (uint32_t)(K * K) * 4);
             }
-            if (MODE == 1) dw_rows_k3<S, PS, ZOUT>(share, xs, clb, w, live_i, a_stage);
-            else if (MODE == 2) dw_quads_k3<S, PS, ZOUT>(share, xs, clb, w, live_i, a_stage);
+            if (MODE == 1) dw_rows<K, S, PS, ZOUT>(share, xs, clb, w, live_i, a_stage);
+            else if (MODE == 2) dw_quads_k3<S, PS, ZOUT>(share, xs, clb, reinterpret_cast<const float (&)[9]>(w), live_i, a_stage);
             else dw_generic<K>(P, xs, clb, wsm, il, run, live_i, a_stage);
             fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
             __threadfence_block();
@@ -651,13 +657,13 @@ static gdws_status_t launch_fused(const FusedParams &P, int device, int grid, si
                   : launch_one<K, MODE, S, PS, false>(P, device, grid, smem, st);
 }
 
-template <int MODE, int S>
+template <int K, int MODE, int S>
 static gdws_status_t launch_fast(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
 {
     switch (P.ps) {
-    case 64: return launch_fused<3, MODE, S, 64>(P, device, grid, smem, st);
-    case 128: return launch_fused<3, MODE, S, 128>(P, device, grid, smem, st);
-    case 256: return launch_fused<3, MODE, S, 256>(P, device, grid, smem, st);
+    case 64: return launch_fused<K, MODE, S, 64>(P, device, grid, smem, st);
+    case 128: return launch_fused<K, MODE, S, 128>(P, device, grid, smem, st);
+    case 256: return launch_fused<K, MODE, S, 256>(P, device, grid, smem, st);
     default: return fail(GDWS_ERR_UNSUPPORTED, "staged pixel size %d", P.ps);
     }
 }
@@ -711,10 +717,12 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     const int grid = P.ntiles < p->sm_count ? P.ntiles : p->sm_count;
     const int dev = p->device;
     gdws_status_t rc;
-    if (t.fast == 1 && p->stride == 1) rc = launch_fast<1, 1>(P, dev, grid, smem, st);
-    else if (t.fast == 1 && p->stride == 2) rc = launch_fast<1, 2>(P, dev, grid, smem, st);
-    else if (t.fast == 2 && p->stride == 1) rc = launch_fast<2, 1>(P, dev, grid, smem, st);
-    else if (t.fast == 2 && p->stride == 2) rc = launch_fast<2, 2>(P, dev, grid, smem, st);
+    if (t.fast == 1 && p->k == 3 && p->stride == 1) rc = launch_fast<3, 1, 1>(P, dev, grid, smem, st);
+    else if (t.fast == 1 && p->k == 3 && p->stride == 2) rc = launch_fast<3, 1, 2>(P, dev, grid, smem, st);
+    else if (t.fast == 1 && p->k == 5 && p->stride == 1) rc = launch_fast<5, 1, 1>(P, dev, grid, smem, st);
+    else if (t.fast == 1 && p->k == 5 && p->stride == 2) rc = launch_fast<5, 1, 2>(P, dev, grid, smem, st);
+    else if (t.fast == 2 && p->stride == 1) rc = launch_fast<3, 2, 1>(P, dev, grid, smem, st);
+    else if (t.fast == 2 && p->stride == 2) rc = launch_fast<3, 2, 2>(P, dev, grid, smem, st);
     else {
         switch (p->k) {
         case 1: rc = launch_fused<1, 0, 1, 0>(P, dev, grid, smem, st); break;

@@ -152,7 +152,7 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
     double best = 1e300;
     bool found = false;
     const int forced = p->opt_tile;
-    const bool fast_shape = p->k == 3 && (p->stride == 1 || p->stride == 2) && p->opt_a_layout == 0;
+    const bool fast_shape = (p->k == 3 || p->k == 5) && (p->stride == 1 || p->stride == 2) && p->opt_a_layout == 0;
     static const int pws[4] = {32, 16, 8, 4};
     for (int pi = 0; pi < 4; ++pi) {
         const int PW = pws[pi];
@@ -164,11 +164,11 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
                 Tile t;
                 t.TN = TN; t.PH = PH; t.PW = PW;
                 if (fast_shape && PW >= 8 && PH % 4 == 0) t.fast = 1;
-                else if (fast_shape && PW == 4) t.fast = 2;
+                else if (fast_shape && p->k == 3 && PW == 4) t.fast = 2;
                 if (forced) {
                     if (TN != ((forced >> 16) & 0xff) || PH != ((forced >> 8) & 0xff) || PW != (forced & 0xff)) continue;
-                } else if (fast_shape && !t.fast) {
-                    continue;                    // a specialised depthwise path exists: only take tiles it covers
+                } else if (fast_shape && p->k == 3 && !t.fast) {
+                    continue;                    // k = 3: every shape has a tile that a specialised depthwise path covers
                 }
                 t.tiles_w = (Wo + PW - 1) / PW;
                 t.tiles_h = (Ho + PH - 1) / PH;

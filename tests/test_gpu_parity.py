@@ -87,6 +87,8 @@ BF16_SHAPES = [
     (9, 16, 64, 8, 8, 3, 2, 1, ("uniform", 1, 9)),       # stride 2 onto 4x4 outputs
     (3, 72, 48, 16, 16, 3, 1, 1, ("const", 1)),            # depthwise-separable special case (g = 1)
     (1, 8, 16, 40, 70, 3, 1, 1, ("uniform", 5, 9)),
+    (2, 16, 24, 19, 17, 5, 2, 2, ("uniform", 1, 25)),      # k = 5, stride 2: the row-run depthwise code for 5 x 5 filters
+    (1, 8, 32, 16, 24, 5, 1, 2, ("heavy",)),
 ]
 
 
