@@ -80,8 +80,8 @@ typedef enum {
     GDWS_OPT_A_LAYOUT = 3, /* bf16 fused path, shared-memory layout of the intermediate
                               tile handed to the tensor cores: 0 = pixel-contiguous
                               (default), 1 = channel-contiguous                            */
-    GDWS_OPT_DW_MATH = 4   /* bf16 paths, depthwise arithmetic: 0 = fp32 FMAs (default),
-                              1 = packed bf16x2 FMAs per filter row, rows summed in fp32   */
+    GDWS_OPT_DW_MATH = 4   /* reserved: 0 or 1 is accepted and changes nothing (the depthwise
+                              arithmetic is fp32 FMAs on bf16 inputs)                      */
 } gdws_option_t;
 
 typedef enum {

@@ -610,7 +610,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             else if (MODE == 2) dw_quads_k3<S, PS, ZOUT>(share, xs, clb, reinterpret_cast<const float (&)[9]>(w), live_i, a_stage);
             else dw_generic<K>(P, xs, clb, wsm, il, run, live_i, a_stage);
             fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
-            __threadfence_block();
             __syncwarp();
             if (lane == 0) {          // this warp is done with the chunk's filters and input box
                 const int flags = meta_tab[q].y;
