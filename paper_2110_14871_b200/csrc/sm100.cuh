@@ -226,23 +226,31 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 __device__ __forceinline__ void store_row16(const uint32_t (&acc)[16], const float *__restrict__ bias, int d0, int D,
                                             int relu, uint16_t *__restrict__ yrow)
 {
+    // The 16 bias values as two 32-byte loads (every lane reads the same address: one sector each).
+    float bv[16];
+    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(bv[0]), "=f"(bv[1]), "=f"(bv[2]), "=f"(bv[3]), "=f"(bv[4]), "=f"(bv[5]), "=f"(bv[6]), "=f"(bv[7])
+                 : "l"(bias + d0));
+    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(bv[8]), "=f"(bv[9]), "=f"(bv[10]), "=f"(bv[11]), "=f"(bv[12]), "=f"(bv[13]), "=f"(bv[14]), "=f"(bv[15])
+                 : "l"(bias + d0 + 8));
     float v[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        v[j] = __uint_as_float(acc[j]) + __ldg(bias + d0 + j);
+        v[j] = __uint_as_float(acc[j]) + bv[j];
         if (relu) v[j] = fmaxf(v[j], 0.f);
     }
-    if (d0 + 8 <= D) {
-        uint4 a;
-        a.x = pack_bf16x2(v[0], v[1]); a.y = pack_bf16x2(v[2], v[3]);
-        a.z = pack_bf16x2(v[4], v[5]); a.w = pack_bf16x2(v[6], v[7]);
-        *reinterpret_cast<uint4 *>(yrow + d0) = a;
-    }
-    if (d0 + 16 <= D) {
-        uint4 b;
-        b.x = pack_bf16x2(v[8], v[9]); b.y = pack_bf16x2(v[10], v[11]);
-        b.z = pack_bf16x2(v[12], v[13]); b.w = pack_bf16x2(v[14], v[15]);
-        *reinterpret_cast<uint4 *>(yrow + d0 + 8) = b;
+    uint32_t o[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) o[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
+    uint16_t *dst = yrow + d0;
+    if (d0 + 16 <= D && (reinterpret_cast<uintptr_t>(dst) & 31) == 0) {
+        // a lane's 16 outputs are one 32-byte sector: one store instead of two half-sector stores
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     ::"l"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+    } else {
+        if (d0 + 8 <= D) *reinterpret_cast<uint4 *>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+        if (d0 + 16 <= D) *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(o[4], o[5], o[6], o[7]);
     }
 }
 
