@@ -34,6 +34,7 @@ namespace gdws {
 
 struct alignas(64) FusedParams {
     CUtensorMap tmap;            // x as (C, W, H, N) bf16, box (cbox, IW, IH, TN)
+    CUtensorMap tmap_y;          // y as (D, Wo, Ho, N) bf16, box (64, PW, PH, TN), 128-byte swizzle (when ostage != 0)
     uint16_t *y;
     const uint32_t *dwpack;
     const uint16_t *pw_img;
@@ -44,6 +45,7 @@ struct alignas(64) FusedParams {
     int TN, PH, PW, tiles_h, tiles_w, ntiles;
     int IH, IW, ps, nslots, nwslots, nboxes, nsb, wstride;
     int spg_shift;                 // log2 of the operand stages per depthwise group (0 or 1)
+    int ostage;                    // bytes of output staging (0: the epilogue stores rows directly)
     int box_bytes, slot_bytes;
     int nhalf, unit_bytes, nacc, acc_cols;
     int a_kmajor, dw_math, zout;
@@ -68,6 +70,7 @@ static_assert(kDwThreads * kRegsDw + 128 * kRegsCtrl + kEpiWarps * 32 * kRegsEpi
 constexpr int kMaxSlots = 8, kMaxBUnits = 8;
 constexpr int kPollNs = 1000;        // longest suspension of one poll by a waiter that runs ahead of the pipeline
 constexpr int kBarChunk0 = 5;       // named barriers 5..8: hand-over of a finished chunk
+constexpr int kBarEpi = 9;          // named barrier 9: the epilogue warps around the output staging buffer
 
 // Barrier traffic is per warp, not per thread: one lane waits or arrives for its warp.
 __device__ __forceinline__ void warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
@@ -336,7 +339,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t a_s = smem_u32(base);
-    const uint32_t b_s = a_s + (32768u << P.spg_shift);   // one or two operand stages per depthwise group
+    const uint32_t o_s = a_s + (32768u << P.spg_shift);   // after the one or two operand stages per depthwise group: output staging
+    const uint32_t b_s = o_s + (uint32_t)P.ostage;
     const uint32_t x_s = b_s + (uint32_t)P.nsb * P.unit_bytes;
     const uint32_t bar_afree = smem_u32(&bars[0]);
     const uint32_t bar_bfull = smem_u32(&bars[4]), bar_bfree = smem_u32(&bars[4 + kMaxBUnits]);
@@ -554,6 +558,39 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             warp_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
             tc_fence_after();
             const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * P.acc_cols);
+            if (P.ostage) {
+                // 64 output channels at a time: every thread puts its row's 128 bytes into the staging buffer
+                // (rows in tile order = the order of a (64, PW, PH, TN) box of y; 16-byte pieces swizzled by
+                // row), then one thread stores the box by TMA, which also clips it to the tensor.  Row-wise
+                // stores from registers would touch 32 different lines per instruction.
+                const bool issuer = warp == kEpiWarp0 && lane == 0;
+                const uint32_t row_s = o_s + (uint32_t)r * 128;
+                const int nblk = P.Dpad >> 6;
+                for (int cb = 0; cb < nblk; ++cb) {
+                    if (issuer) bulk_wait_read_all();          // the last box has left the staging buffer
+                    named_bar_sync(kBarEpi, kEpiWarps * 32);
+#pragma unroll 1
+                    for (int h4 = 0; h4 < 4; ++h4) {
+                        uint32_t acc[16], o[8];
+                        tmem_ld16(t_base + (uint32_t)(cb * 64 + h4 * 16), acc);
+                        tmem_ld_wait();
+                        finish_row16(acc, P.bias, cb * 64 + h4 * 16, P.relu, o);
+                        sts128(row_s + (uint32_t)(((2 * h4) ^ (r & 7)) << 4), make_uint4(o[0], o[1], o[2], o[3]));
+                        sts128(row_s + (uint32_t)(((2 * h4 + 1) ^ (r & 7)) << 4), make_uint4(o[4], o[5], o[6], o[7]));
+                    }
+                    fence_proxy_async();
+                    if (cb == nblk - 1) {                      // the accumulator has been read: the next tile may use it
+                        tc_fence_before();
+                        warp_arrive(bar_accfree + 8 * buf);
+                    }
+                    named_bar_sync(kBarEpi, kEpiWarps * 32);
+                    if (issuer) {
+                        tma_store_4d(o_s, &P.tmap_y, cb * 64, bw * P.PW, bh * P.PH, bn * P.TN);
+                        bulk_commit();
+                    }
+                }
+                continue;
+            }
             for (int d0 = 0; d0 < P.Dpad; d0 += 16) {
                 uint32_t acc[16];
                 tmem_ld16(t_base + (uint32_t)d0, acc);
@@ -563,6 +600,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             tc_fence_before();
             warp_arrive(bar_accfree + 8 * buf);
         }
+        if (!ZOUT && P.ostage && warp == kEpiWarp0 && lane == 0) bulk_wait_all();   // the staging buffer must outlive its stores
     } else {
         // ---------------- depthwise warps: group g takes the chunks gq = g, g+2, ... ----------------
         regs_inc<kRegsDw>();
@@ -695,6 +733,22 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     }
+    // The staged epilogue pays when it overlaps the next tile's main loop; a block with a single tile would
+    // only wait for its one staging buffer between the column blocks.
+    const bool tma_out = !zout && t.ostage && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && t.tiles() > p->sm_count;
+    if (tma_out) {
+        // y as a rank-4 tensor, innermost first: channels, width, height, batch
+        const cuuint64_t dims[4] = {(cuuint64_t)p->D, (cuuint64_t)Wo, (cuuint64_t)Ho, (cuuint64_t)x->n};
+        const cuuint64_t strides[3] = {(cuuint64_t)p->D * 2, (cuuint64_t)Wo * p->D * 2, (cuuint64_t)Ho * Wo * p->D * 2};
+        const cuuint32_t box[4] = {64, (cuuint32_t)t.PW, (cuuint32_t)t.PH, (cuuint32_t)t.TN};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        const CUresult r = encode(&P.tmap_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, out, dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled (y) failed with code %d", (int)r);
+    } else {
+        P.tmap_y = P.tmap;
+    }
     P.y = (uint16_t *)out;
     P.dwpack = p->d_dwpack; P.pw_img = p->d_pw_img; P.bias = p->d_bias;
     P.chunk_meta = reinterpret_cast<const int4 *>(p->d_chunk_meta); P.status = p->d_status;
@@ -704,6 +758,7 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
     P.IH = t.IH; P.IW = t.IW; P.ps = t.cbox * 2; P.nslots = t.nslots; P.nwslots = t.nwslots; P.nboxes = p->nboxes; P.nsb = t.nsb; P.wstride = p->wstride;
     P.spg_shift = t.spg == 2 ? 1 : 0;
+    P.ostage = tma_out ? t.ostage : 0;
     P.box_bytes = t.box_bytes; P.slot_bytes = t.slot_bytes;
     P.nhalf = p->Dpad > 256 ? 2 : 1;
     P.unit_bytes = (p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;

@@ -34,6 +34,7 @@ struct Tile {
     int nwslots = 0;                 // filter blocks in flight (one per chunk)
     int nsb = 0;                     // pointwise-weight units in the ring
     int spg = 2;                     // operand stages per depthwise group (1 or 2)
+    int ostage = 0;                  // bytes of output staging for the TMA-store epilogue (0: direct stores)
     int fast = 0;                    // 1: row-run depthwise path, 2: 4-wide-patch path, 0: generic
     size_t smem = 0;                 // dynamic shared memory of the fused kernel
     int64_t tiles() const { return (int64_t)tiles_n * tiles_h * tiles_w; }

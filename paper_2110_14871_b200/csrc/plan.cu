@@ -114,17 +114,20 @@ static int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
 // Shared-memory layout of the fused bf16 kernel: 2 * t.spg intermediate-tile stages, a ring of `nsb`
 // pointwise-weight units (a unit = one K chunk x up to 256 output channels, at most 32 KB) and
-// `nslots` staged-input slots (one TMA box plus the chunk's filters).  Fills t.nsb / t.nslots /
-// t.smem; false if it cannot fit.  Prefers at least 3 chunks of weights and 4 input slots in flight.
-static bool fit_smem(const gdws_plan_s *p, Tile &t)
+// `nslots` staged-input slots (one TMA box), a ring of filter blocks and, where the epilogue stores by TMA,
+// one output staging buffer.  Fills t.nsb / t.nslots / t.nwslots / t.ostage / t.smem; false if it cannot fit.  Prefers at least 3 chunks of weights and 4 input slots in flight.
+static bool fit_smem(const gdws_plan_s *p, Tile &t, bool stage_out)
 {
     const size_t a = 2 * (size_t)t.spg * kTileRows * kChunk * 2;
     const int nhalf = p->Dpad > 256 ? 2 : 1;
     const size_t unit = (size_t)(p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
     const size_t slot = (size_t)t.slot_bytes;
     const size_t wblock = (size_t)kChunk * p->wstride * 4;                 // one chunk's filters
-    t.nwslots = (int)std::max<size_t>(3, std::min<size_t>(8, (20 * 1024) / wblock));
-    const size_t fixed = a + 1024 /*alignment slack*/ + t.nwslots * wblock + (size_t)p->nchunks * 16 /*chunk table*/;
+    t.nwslots = 3;                   // two groups at work and one block in flight; deeper rings measured no faster
+    // Output channels in whole 64-column blocks: the epilogue stages 128 rows x 64 columns and stores them by TMA.
+    // (Not beyond 256 channels: there the weight ring needs the shared memory more.)
+    t.ostage = stage_out && p->D % 64 == 0 && p->Dpad <= 256 ? kTileRows * 128 : 0;
+    const size_t fixed = a + t.ostage + 1024 /*alignment slack*/ + t.nwslots * wblock + (size_t)p->nchunks * 16 /*chunk table*/;
     int best_score = -1;
     for (int ns = 2; ns <= 8; ++ns) {
         if (fixed + ns * slot + (size_t)(nhalf + 1) * unit > (size_t)kMaxSmem) break;
@@ -179,11 +182,14 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
                 t.cbox = cbox;
                 t.box_bytes = TN * t.IH * t.IW * cbox * 2;
                 t.slot_bytes = round_up(t.box_bytes, 128);
-                for (int spg = 2; spg >= 1; --spg) {     // one operand stage per group costs some overlap
-                    t.spg = spg;
-                    if (!fit_smem(p, t)) continue;
+                for (int variant = 0; variant < 4; ++variant) {
+                    // one operand stage per group costs some overlap, an epilogue without staging costs store bandwidth
+                    t.spg = 2 - (variant & 1);
+                    const bool stage_out = variant < 2;
+                    if (!fit_smem(p, t, stage_out)) continue;
                     const double tiles = (double)t.tiles();
-                    const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IW) * (t.fast ? 1.0 : 4.0) * (spg == 1 ? 1.08 : 1.0) - 1e-3 * PW;
+                    const double cost = tiles * (128.0 + 0.3 * TN * t.IH * t.IW) * (t.fast ? 1.0 : 4.0) * (t.spg == 1 ? 1.08 : 1.0) *
+                                            (stage_out ? 1.0 : 1.07) - 1e-3 * PW;
                     if (cost < best) { best = cost; *out = t; found = true; }
                 }
             }

@@ -223,6 +223,24 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 // ------------------------------------------------------------------------------------------
 // Epilogue shared by both tensor-core kernels: 16 accumulator columns of one pixel row.
 // ------------------------------------------------------------------------------------------
+// 16 accumulator columns of one row -> bias, optional ReLU, bf16: eight packed words.
+__device__ __forceinline__ void finish_row16(const uint32_t (&acc)[16], const float *__restrict__ bias, int d0, int relu,
+                                             uint32_t (&o)[8])
+{
+    float bv[16];
+    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(bv[0]), "=f"(bv[1]), "=f"(bv[2]), "=f"(bv[3]), "=f"(bv[4]), "=f"(bv[5]), "=f"(bv[6]), "=f"(bv[7])
+                 : "l"(bias + d0));
+    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(bv[8]), "=f"(bv[9]), "=f"(bv[10]), "=f"(bv[11]), "=f"(bv[12]), "=f"(bv[13]), "=f"(bv[14]), "=f"(bv[15])
+                 : "l"(bias + d0 + 8));
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        float lo = __uint_as_float(acc[2 * j]) + bv[2 * j], hi = __uint_as_float(acc[2 * j + 1]) + bv[2 * j + 1];
+        if (relu) { lo = fmaxf(lo, 0.f); hi = fmaxf(hi, 0.f); }
+        o[j] = pack_bf16x2(lo, hi);
+    }
+}
 __device__ __forceinline__ void store_row16(const uint32_t (&acc)[16], const float *__restrict__ bias, int d0, int D,
                                             int relu, uint16_t *__restrict__ yrow)
 {
@@ -299,6 +317,20 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tma
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
         ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
 }
+
+// TMA tiled store of a rank-4 box from shared memory (bulk async-group completion).  Coordinates
+// innermost first and non-negative; elements outside the tensor are not written.
+__device__ __forceinline__ void tma_store_4d(uint32_t src, const CUtensorMap *tmap, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+        ::"l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Until the bulk stores this thread committed have read their shared-memory source.
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// Until they are complete.
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // TMA tiled load of a rank-2 box (innermost coordinate first; it must start on a 16-byte boundary).
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int c0, int c1, uint32_t bar)
