@@ -60,6 +60,11 @@ def layer_numbers(spec: gi.LayerSpec, G: int):
     return px, macs, nbytes
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
+# summarised under profiles/ (key: config, layer, path).  An entry is removed when its kernel changes.
+TRAFFIC_BYTES_PER_LAUNCH = {(1, 0, "fused"): 9169152}   # y (8.39 MB) stays in L2 within the captured launch
+
+
 def layer_roofline_us(macs, nbytes, peaks, sustained=False):
     tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
     t_tensor = 2.0 * macs / (tf * 1e12) * 1e6
@@ -356,16 +361,32 @@ def run_ours(args, spec):
     t_roof, t_tensor, t_hbm = layer_roofline_us(macs, nbytes, peaks)
     t_roof_s, _, _ = layer_roofline_us(macs, nbytes, peaks, sustained=True)
     us = sec_per_step * 1e6
-    bound = "tensor" if t_tensor >= t_hbm else "hbm"
+    # The GDW stage runs on the fp32 FMA lanes (its k*k MACs per intermediate value cannot use the tensor
+    # cores: each output depends on one input channel only).  Its bound: 128 FMA lanes per SM at the
+    # maximum SM clock.
+    clocks = clk.summary()
+    props = torch.cuda.get_device_properties(local)
+    sm_mhz = float(clocks.get("sm_max_mhz") or 1965)
+    alu_tflops = 2.0 * props.multi_processor_count * 128 * sm_mhz * 1e6 / 1e12
+    dw_macs = px * G * spec.k * spec.k
+    t_alu = 2.0 * dw_macs / (alu_tflops * 1e12) * 1e6
+    bound = max((t_tensor, "tensor"), (t_hbm, "hbm"), (t_alu, "alu"))[1]
     if bound == "tensor":
         achieved, peak, runit = 2.0 * macs / sec_per_step / 1e12, peaks["bf16_tflops"], "TFLOP/s"
-    else:
+        psrc = peaks["source"] + " burst"
+    elif bound == "hbm":
         achieved, peak, runit = nbytes / sec_per_step / 1e9, peaks["hbm_gbs"], "GB/s"
-    traffic = None
+        psrc = peaks["source"] + " copy"
+    else:
+        achieved, peak, runit = 2.0 * dw_macs / sec_per_step / 1e12, alu_tflops, "TFLOP/s"
+        psrc = "derived: SMs x 128 fp32 FMA lanes x max SM clock"
+    t_roof = max(t_roof, t_alu)
+    t_roof_s = max(t_roof_s, t_alu)
     roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
-            "traffic": traffic, "peak_source": peaks["source"] + (" burst" if bound == "tensor" else " copy"),
+            "traffic": TRAFFIC_BYTES_PER_LAUNCH.get((args.config, args.layer, args.path)) if not f32 else None,
+            "peak_source": psrc,
             "kernel": "fused_bf16_kernel" if (not f32 and path != gdws.PATH_UNFUSED) else "see config.path",
-            "layer_roofline_us": t_roof, "t_tensor_us": t_tensor, "t_hbm_us": t_hbm,
+            "layer_roofline_us": t_roof, "t_tensor_us": t_tensor, "t_hbm_us": t_hbm, "t_alu_us": t_alu,
             "frac_of_layer_roofline": t_roof / us, "frac_of_layer_roofline_sustained_peak": t_roof_s / us}
 
     cpu_v, cpu_n, cpu_reps, cpu_dt, cores = oracle_throughput(spec, target_s=args.cpu_seconds)
@@ -396,7 +417,7 @@ def run_ours(args, spec):
         "dtype": spec.dtype, "data": "synthetic", "config": cfg,
         "effective_tmacs": world * macs / sec_per_step / 1e12,
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-        "clocks": clk.summary(), "parity_max_rel_err": parity,
+        "clocks": clocks, "parity_max_rel_err": parity,
     }
     print(json.dumps(out), flush=True)
     plan.destroy()
