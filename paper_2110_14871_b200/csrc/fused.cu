@@ -375,6 +375,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     }
     if (!ZOUT && warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
     for (int q = tid; q < P.nchunks; q += kFusedThreads) meta_tab[q] = __ldg(P.chunk_meta + q);
+    // a copy of the bias next to the chunk table: the epilogue reads it per 16 columns, with the accumulator in hand
+    float *bias_sm = reinterpret_cast<float *>(meta_tab + P.nchunks);
+    const uint32_t bias_s = smem_u32(bias_sm);
+    if (!ZOUT)
+        for (int d = tid; d < P.Dpad; d += kFusedThreads) bias_sm[d] = __ldg(P.bias + d);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -574,7 +579,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                         uint32_t acc[16], o[8];
                         tmem_ld16(t_base + (uint32_t)(cb * 64 + h4 * 16), acc);
                         tmem_ld_wait();
-                        finish_row16(acc, P.bias, cb * 64 + h4 * 16, P.relu, o);
+                        float bv[16];
+                        bias16_shared(bias_s + (uint32_t)(cb * 64 + h4 * 16) * 4, bv);
+                        finish_row16(acc, bv, P.relu, o);
                         sts128(row_s + (uint32_t)(((2 * h4) ^ (r & 7)) << 4), make_uint4(o[0], o[1], o[2], o[3]));
                         sts128(row_s + (uint32_t)(((2 * h4 + 1) ^ (r & 7)) << 4), make_uint4(o[4], o[5], o[6], o[7]));
                     }
@@ -595,7 +602,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 uint32_t acc[16];
                 tmem_ld16(t_base + (uint32_t)d0, acc);
                 tmem_ld_wait();
-                if (live) store_row16(acc, P.bias, d0, P.D, P.relu, yrow);
+                if (live) {
+                    float bv[16];
+                    uint32_t o[8];
+                    bias16_shared(bias_s + (uint32_t)d0 * 4, bv);
+                    finish_row16(acc, bv, P.relu, o);
+                    store_packed16(o, d0, P.D, yrow);
+                }
             }
             tc_fence_before();
             warp_arrive(bar_accfree + 8 * buf);

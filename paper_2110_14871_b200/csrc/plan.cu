@@ -127,7 +127,7 @@ static bool fit_smem(const gdws_plan_s *p, Tile &t, bool stage_out)
     // Output channels in whole 64-column blocks: the epilogue stages 128 rows x 64 columns and stores them by TMA.
     // (Not beyond 256 channels: there the weight ring needs the shared memory more.)
     t.ostage = stage_out && p->D % 64 == 0 && p->Dpad <= 256 ? kTileRows * 128 : 0;
-    const size_t fixed = a + t.ostage + 1024 /*alignment slack*/ + t.nwslots * wblock + (size_t)p->nchunks * 16 /*chunk table*/;
+    const size_t fixed = a + t.ostage + 1024 /*alignment slack*/ + t.nwslots * wblock + (size_t)p->nchunks * 16 /*chunk table*/ + (size_t)p->Dpad * 4 /*bias*/;
     int best_score = -1;
     for (int ns = 2; ns <= 8; ++ns) {
         if (fixed + ns * slot + (size_t)(nhalf + 1) * unit > (size_t)kMaxSmem) break;

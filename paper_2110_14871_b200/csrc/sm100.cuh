@@ -223,17 +223,27 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 // ------------------------------------------------------------------------------------------
 // Epilogue shared by both tensor-core kernels: 16 accumulator columns of one pixel row.
 // ------------------------------------------------------------------------------------------
-// 16 accumulator columns of one row -> bias, optional ReLU, bf16: eight packed words.
-__device__ __forceinline__ void finish_row16(const uint32_t (&acc)[16], const float *__restrict__ bias, int d0, int relu,
-                                             uint32_t (&o)[8])
+// 16 bias values from global memory as two 32-byte loads (every lane reads the same address: one sector each).
+__device__ __forceinline__ void bias16_global(const float *__restrict__ bias, float (&bv)[16])
 {
-    float bv[16];
     asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                  : "=f"(bv[0]), "=f"(bv[1]), "=f"(bv[2]), "=f"(bv[3]), "=f"(bv[4]), "=f"(bv[5]), "=f"(bv[6]), "=f"(bv[7])
-                 : "l"(bias + d0));
+                 : "l"(bias));
     asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                  : "=f"(bv[8]), "=f"(bv[9]), "=f"(bv[10]), "=f"(bv[11]), "=f"(bv[12]), "=f"(bv[13]), "=f"(bv[14]), "=f"(bv[15])
-                 : "l"(bias + d0 + 8));
+                 : "l"(bias + 8));
+}
+// The same from a copy in shared memory (address of the first of the 16; 16-byte aligned).
+__device__ __forceinline__ void bias16_shared(uint32_t addr, float (&bv)[16])
+{
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(bv[4 * j]), "=f"(bv[4 * j + 1]), "=f"(bv[4 * j + 2]), "=f"(bv[4 * j + 3]) : "r"(addr + 16 * j));
+}
+// 16 accumulator columns of one row -> bias, optional ReLU, bf16: eight packed words.
+__device__ __forceinline__ void finish_row16(const uint32_t (&acc)[16], const float (&bv)[16], int relu, uint32_t (&o)[8])
+{
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         float lo = __uint_as_float(acc[2 * j]) + bv[2 * j], hi = __uint_as_float(acc[2 * j + 1]) + bv[2 * j + 1];
@@ -241,26 +251,9 @@ __device__ __forceinline__ void finish_row16(const uint32_t (&acc)[16], const fl
         o[j] = pack_bf16x2(lo, hi);
     }
 }
-__device__ __forceinline__ void store_row16(const uint32_t (&acc)[16], const float *__restrict__ bias, int d0, int D,
-                                            int relu, uint16_t *__restrict__ yrow)
+// Stores a row's 16 finished channels d0 .. d0+15 (those below D) to yrow.
+__device__ __forceinline__ void store_packed16(const uint32_t (&o)[8], int d0, int D, uint16_t *__restrict__ yrow)
 {
-    // The 16 bias values as two 32-byte loads (every lane reads the same address: one sector each).
-    float bv[16];
-    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=f"(bv[0]), "=f"(bv[1]), "=f"(bv[2]), "=f"(bv[3]), "=f"(bv[4]), "=f"(bv[5]), "=f"(bv[6]), "=f"(bv[7])
-                 : "l"(bias + d0));
-    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=f"(bv[8]), "=f"(bv[9]), "=f"(bv[10]), "=f"(bv[11]), "=f"(bv[12]), "=f"(bv[13]), "=f"(bv[14]), "=f"(bv[15])
-                 : "l"(bias + d0 + 8));
-    float v[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        v[j] = __uint_as_float(acc[j]) + bv[j];
-        if (relu) v[j] = fmaxf(v[j], 0.f);
-    }
-    uint32_t o[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) o[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
     uint16_t *dst = yrow + d0;
     if (d0 + 16 <= D && (reinterpret_cast<uintptr_t>(dst) & 31) == 0) {
         // a lane's 16 outputs are one 32-byte sector: one store instead of two half-sector stores
@@ -270,6 +263,15 @@ __device__ __forceinline__ void store_row16(const uint32_t (&acc)[16], const flo
         if (d0 + 8 <= D) *reinterpret_cast<uint4 *>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
         if (d0 + 16 <= D) *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(o[4], o[5], o[6], o[7]);
     }
+}
+__device__ __forceinline__ void store_row16(const uint32_t (&acc)[16], const float *__restrict__ bias, int d0, int D,
+                                            int relu, uint16_t *__restrict__ yrow)
+{
+    float bv[16];
+    uint32_t o[8];
+    bias16_global(bias + d0, bv);
+    finish_row16(acc, bv, relu, o);
+    store_packed16(o, d0, D, yrow);
 }
 
 // Issue the MMAs of one 64-wide K chunk (4 steps of K=16; output channels beyond 256 take a
