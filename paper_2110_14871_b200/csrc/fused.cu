@@ -68,6 +68,7 @@ constexpr int kRegsLaunch = 80, kRegsDw = 96, kRegsCtrl = 40, kRegsEpi = 56;
 static_assert(kDwThreads * kRegsDw + 128 * kRegsCtrl + kEpiWarps * 32 * kRegsEpi <= kFusedThreads * kRegsLaunch,
               "register split exceeds the block's allocation: setmaxnreg.inc would wait forever");
 constexpr int kMaxSlots = 8, kMaxBUnits = 8;
+constexpr int kTailShare = 1 + kDwWarps / 4;   // warps per TMEM lane quarter that share the last tile's epilogue
 constexpr int kPollNs = 1000;        // longest suspension of one poll by a waiter that runs ahead of the pipeline
 constexpr int kBarChunk0 = 5;       // named barriers 5..8: hand-over of a finished chunk
 constexpr int kBarEpi = 9;          // named barrier 9: the epilogue warps around the output staging buffer
@@ -318,6 +319,26 @@ __device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, in
             }
         }
         store_group(P, a_stage, o, kk, out);
+    }
+}
+
+// Epilogue of one thread's accumulator row with direct stores: the 16-column granules first, first + step, ...
+// go from TMEM through bias / ReLU / bf16 rounding to y.
+__device__ __forceinline__ void epilogue_row(const FusedParams &P, uint32_t t_base, uint32_t bias_s, uint16_t *yrow, bool live,
+                                             int first, int step)
+{
+    const int ngran = P.Dpad >> 4;
+    for (int j = first; j < ngran; j += step) {
+        uint32_t acc[16];
+        tmem_ld16(t_base + (uint32_t)(j * 16), acc);
+        tmem_ld_wait();
+        if (live) {
+            float bv[16];
+            uint32_t o[8];
+            bias16_shared(bias_s + (uint32_t)j * 64, bv);
+            finish_row16(acc, bv, P.relu, o);
+            store_packed16(o, j * 16, P.D, yrow);
+        }
     }
 }
 
@@ -598,18 +619,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 }
                 continue;
             }
-            for (int d0 = 0; d0 < P.Dpad; d0 += 16) {
-                uint32_t acc[16];
-                tmem_ld16(t_base + (uint32_t)d0, acc);
-                tmem_ld_wait();
-                if (live) {
-                    float bv[16];
-                    uint32_t o[8];
-                    bias16_shared(bias_s + (uint32_t)d0 * 4, bv);
-                    finish_row16(acc, bv, P.relu, o);
-                    store_packed16(o, d0, P.D, yrow);
-                }
-            }
+            // the block's last tile: the depthwise warps, idle by then, take four fifths of the columns
+            epilogue_row(P, t_base, bias_s, yrow, live, 0, tl == my_tiles - 1 ? kTailShare : 1);
             tc_fence_before();
             warp_arrive(bar_accfree + 8 * buf);
         }
@@ -675,6 +686,30 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             wslot += 2;
             while (wslot >= P.nwslots) wslot -= P.nwslots;
         }
+    }
+    if (!ZOUT && !P.ostage && warp >= kDwWarp0 && warp < kEpiWarp0) {
+        // ---------------- depthwise warps, done with their chunks: help with the last tile's epilogue ----------------
+        // A warp reads the TMEM lanes 32 * (warp % 4) ...; the four depthwise warps and the epilogue warp of a
+        // lane quarter share its columns in granules of 16.
+        const int tl = my_tiles - 1;
+        const int lg = warp & 3;
+        const int r = lg * 32 + lane;
+        const int hw = P.PH * P.PW;
+        const int tn = r / hw;
+        const int rem = r - tn * hw;
+        const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
+        int tile = (int)blockIdx.x + tl * (int)gridDim.x;
+        const int bn = tile / tiles_hw;
+        tile -= bn * tiles_hw;
+        const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+        const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
+        const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
+        uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D;
+        const int buf = tl % P.nacc;
+        warp_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
+        tc_fence_after();
+        const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * P.acc_cols);
+        epilogue_row(P, t_base, bias_s, yrow, live, 1 + ((warp - kDwWarp0) >> 2), kTailShare);
     }
     tc_fence_before();
     __syncthreads();
