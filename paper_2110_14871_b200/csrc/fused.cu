@@ -758,14 +758,14 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     if (!zout && p->Dpad > 512) return fail(GDWS_ERR_UNSUPPORTED, "bf16 fused kernel supports D <= 512 (got %d)", p->D);
     if (p->D % 8 || p->C % 8)
         return fail(GDWS_ERR_UNSUPPORTED, "bf16 kernels need C %% 8 == 0 and D %% 8 == 0 (got C=%d, D=%d)", p->C, p->D);
-    Tile t;
-    if (!choose_tile(p, x->n, x->h, x->w, &t))
-        return fail(GDWS_ERR_UNSUPPORTED, "no fused tile fits this shape in shared memory");
-    if (t.tiles() > 0x7fffffffLL) return fail(GDWS_ERR_UNSUPPORTED, "too many tiles");
     if (p->sm_count <= 0) {
         cudaError_t e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
         if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute(MultiProcessorCount)");
     }
+    Tile t;
+    if (!choose_tile(p, x->n, x->h, x->w, &t))
+        return fail(GDWS_ERR_UNSUPPORTED, "no fused tile fits this shape in shared memory");
+    if (t.tiles() > 0x7fffffffLL) return fail(GDWS_ERR_UNSUPPORTED, "too many tiles");
     tensor_map_encode_fn encode = encode_fn();
     if (!encode) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
     FusedParams P;
