@@ -46,6 +46,8 @@ struct alignas(64) FusedParams {
     int IH, IW, ps, nslots, nwslots, nboxes, nsb, wstride;
     int spg_shift;                 // log2 of the operand stages per depthwise group (0 or 1)
     int ostage;                    // bytes of output staging (0: the epilogue stores rows directly)
+    int nsplit;                    // blocks per tile: each takes Dpad of the Dtot output channels (D, Dpad: one block's share)
+    int Dtot, Dpad_tot;            // output channels of the layer (row pitch of y), rows per chunk of the packed pointwise matrix
     int box_bytes, slot_bytes;
     int nhalf, unit_bytes, nacc, acc_cols;
     int a_kmajor, dw_math, zout;
@@ -348,9 +350,11 @@ __device__ __forceinline__ void epilogue_row(const FusedParams &P, uint32_t t_ba
 // stages and the four "epilogue" warps copy each finished stage to z[pixel][Gpad] in global memory
 // (16-byte stores, 128 contiguous bytes per pixel and chunk); no weights are streamed, no MMA is issued
 // and no TMEM is used.  P.y then points to z and P.D holds Gpad.
-template <int K, int MODE, int S, int PS, bool ZOUT>
+// VAR: 0 the fused kernel, 1 ZOUT, 2 the fused kernel with several blocks per tile (P.nsplit > 1).
+template <int K, int MODE, int S, int PS, int VAR>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __grid_constant__ FusedParams P)
 {
+    constexpr bool ZOUT = VAR == 1, SPLIT = VAR == 2;
     extern __shared__ uint8_t smem_raw[];
     // a_free[4] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2] | w_full[8] w_free[8] | open[4]
     __shared__ __align__(8) uint64_t bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots + 4 + 2 * kMaxSlots + 4];
@@ -358,6 +362,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     __shared__ int abort_flag;
     __shared__ uint32_t xinfo[kMaxSlots];      // per filter-ring slot: input slot (bits 0-7) and phase parity (bit 8) of the chunk's box
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // With few tiles, nsplit blocks share a tile: each does the whole depthwise stage and its share of the output channels.
+    // (worked out where it is needed, not kept in registers through the depthwise loop)
+#define GDWS_BLOCK_SHARE                                                                                     \
+    const int part = SPLIT ? (int)blockIdx.x % P.nsplit : 0, bid = SPLIT ? (int)blockIdx.x / P.nsplit : (int)blockIdx.x, \
+              nblocks = SPLIT ? (int)gridDim.x / P.nsplit : (int)gridDim.x;                                 \
+    (void)part; (void)bid; (void)nblocks
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t a_s = smem_u32(base);
     const uint32_t o_s = a_s + (32768u << P.spg_shift);   // after the one or two operand stages per depthwise group: output staging
@@ -399,14 +409,20 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     // a copy of the bias next to the chunk table: the epilogue reads it per 16 columns, with the accumulator in hand
     float *bias_sm = reinterpret_cast<float *>(meta_tab + P.nchunks);
     const uint32_t bias_s = smem_u32(bias_sm);
-    if (!ZOUT)
-        for (int d = tid; d < P.Dpad; d += kFusedThreads) bias_sm[d] = __ldg(P.bias + d);
+    if (!ZOUT) {
+        GDWS_BLOCK_SHARE;
+        for (int d = tid; d < P.Dpad; d += kFusedThreads) bias_sm[d] = __ldg(P.bias + part * P.Dpad + d);
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = ZOUT ? 0u : tmem_slot;
 
-    const int my_tiles = (P.ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    int my_tiles;
+    {
+        GDWS_BLOCK_SHARE;
+        my_tiles = (P.ntiles - bid + nblocks - 1) / nblocks;
+    }
     const int total_chunks = my_tiles * P.nchunks;
     const int tiles_hw = P.tiles_h * P.tiles_w;
 
@@ -474,25 +490,27 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             }
         } else if (!ZOUT && warp == kCtrlWarp + 1 && lane == 0) {
             // ---------------- pointwise-weight loader (one thread): ring of nsb units ----------------
+            GDWS_BLOCK_SHARE;
             uint32_t sb = 0, pb = 1;          // parity of the "slot free" phase awaited (first round: nothing to wait for)
             int q = 0, h = 0;
             for (int u = 0; u < total_units; ++u) {
                 if (u >= P.nsb) mbar_wait_relaxed<kPollNs>(bar_bfree + 8 * sb, pb, &abort_flag, P.status, kStatusWaitStage);
                 const uint32_t bytes = (uint32_t)(h ? rows1 : rows0) * 128u;
                 mbar_expect_tx(bar_bfull + 8 * sb, bytes);
-                bulk_g2s(b_s + sb * P.unit_bytes, P.pw_img + ((size_t)q * P.Dpad + h * 256) * kChunk, bytes,
+                bulk_g2s(b_s + sb * P.unit_bytes, P.pw_img + ((size_t)q * P.Dpad_tot + part * P.Dpad + h * 256) * kChunk, bytes,
                          bar_bfull + 8 * sb);
                 if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
                 if (++h == P.nhalf) { h = 0; if (++q == P.nchunks) q = 0; }
             }
         } else if (warp == kCtrlWarp + 2 && lane == 0) {
             // ---------------- input loader (one thread): ring of boxes, ring of filter blocks ----------------
+            GDWS_BLOCK_SHARE;
             uint32_t xslot = 0, xpar = 1;     // next box slot; parity of the "slot free" phase awaited
             uint32_t wslot = 0, wpar = 1;
             uint32_t cur_x = 0;               // slot and "full" phase parity of the box the current chunks read
             int gq = 0, gb = 0;
             for (int tl = 0; tl < my_tiles; ++tl) {
-                int tile = (int)blockIdx.x + tl * (int)gridDim.x;
+                int tile = bid + tl * nblocks;
                 const int bn = tile / tiles_hw;
                 tile -= bn * tiles_hw;
                 const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
@@ -546,6 +564,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         }
     } else if (warp >= kEpiWarp0) {
         // ---------------- epilogue warps: TMEM -> registers -> bias / ReLU -> bf16 -> global ----------------
+        GDWS_BLOCK_SHARE;
         regs_dec<kRegsEpi>();
         const int lg = warp & 3;                          // TMEM lanes 32*lg .. 32*lg+31 belong to this warp
         const int r = lg * 32 + lane;
@@ -555,13 +574,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
         int wq = 0;                                       // ZOUT: running index of the next finished chunk
         for (int tl = 0; tl < my_tiles; ++tl) {
-            int tile = (int)blockIdx.x + tl * (int)gridDim.x;
+            int tile = bid + tl * nblocks;
             const int bn = tile / tiles_hw;
             tile -= bn * tiles_hw;
             const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
             const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
             const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
-            uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D;
+            uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.Dtot + part * P.Dpad;
             if (ZOUT) {
                 // this thread's pixel row of every finished stage goes to z (row r of the stage: 128 bytes, swizzled)
                 for (int q = 0; q < P.nchunks; ++q, ++wq) {
@@ -613,7 +632,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     }
                     named_bar_sync(kBarEpi, kEpiWarps * 32);
                     if (issuer) {
-                        tma_store_4d(o_s, &P.tmap_y, cb * 64, bw * P.PW, bh * P.PH, bn * P.TN);
+                        tma_store_4d(o_s, &P.tmap_y, part * P.Dpad + cb * 64, bw * P.PW, bh * P.PH, bn * P.TN);
                         bulk_commit();
                     }
                 }
@@ -689,6 +708,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     }
     if (!ZOUT && !P.ostage && warp >= kDwWarp0 && warp < kEpiWarp0) {
         // ---------------- depthwise warps, done with their chunks: help with the last tile's epilogue ----------------
+        GDWS_BLOCK_SHARE;
         // A warp reads the TMEM lanes 32 * (warp % 4) ...; the four depthwise warps and the epilogue warp of a
         // lane quarter share its columns in granules of 16.
         const int tl = my_tiles - 1;
@@ -698,13 +718,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int tn = r / hw;
         const int rem = r - tn * hw;
         const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
-        int tile = (int)blockIdx.x + tl * (int)gridDim.x;
+        int tile = bid + tl * nblocks;
         const int bn = tile / tiles_hw;
         tile -= bn * tiles_hw;
         const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
         const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
         const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
-        uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D;
+        uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.Dtot + part * P.Dpad;
         const int buf = tl % P.nacc;
         warp_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
         tc_fence_after();
@@ -720,17 +740,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
-template <int K, int MODE, int S, int PS, bool ZOUT>
+template <int K, int MODE, int S, int PS, int VAR>
 static gdws_status_t launch_one(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
 {
     cudaError_t e = cudaSuccess;
     static bool attr_set[64] = {};
     if (!attr_set[device & 63]) {   // once per device: allow the full dynamic shared memory
-        e = cudaFuncSetAttribute(fused_bf16_kernel<K, MODE, S, PS, ZOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        e = cudaFuncSetAttribute(fused_bf16_kernel<K, MODE, S, PS, VAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_bf16_kernel)");
         attr_set[device & 63] = true;
     }
-    fused_bf16_kernel<K, MODE, S, PS, ZOUT><<<grid, kFusedThreads, smem, st>>>(P);
+    fused_bf16_kernel<K, MODE, S, PS, VAR><<<grid, kFusedThreads, smem, st>>>(P);
     e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "fused_bf16_kernel launch");
 }
@@ -738,8 +758,12 @@ static gdws_status_t launch_one(const FusedParams &P, int device, int grid, size
 template <int K, int MODE, int S, int PS>
 static gdws_status_t launch_fused(const FusedParams &P, int device, int grid, size_t smem, cudaStream_t st)
 {
-    return P.zout ? launch_one<K, MODE, S, PS, true>(P, device, grid, smem, st)
-                  : launch_one<K, MODE, S, PS, false>(P, device, grid, smem, st);
+    if (P.zout) return launch_one<K, MODE, S, PS, 1>(P, device, grid, smem, st);
+    if (P.nsplit > 1) {
+        if constexpr (K == 3 && MODE != 0) return launch_one<K, MODE, S, PS, 2>(P, device, grid, smem, st);
+        else return fail(GDWS_ERR_UNSUPPORTED, "several blocks per tile: no such kernel for k=%d", K);
+    }
+    return launch_one<K, MODE, S, PS, 0>(P, device, grid, smem, st);
 }
 
 template <int K, int MODE, int S>
@@ -800,7 +824,11 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     P.y = (uint16_t *)out;
     P.dwpack = p->d_dwpack; P.pw_img = p->d_pw_img; P.bias = p->d_bias;
     P.chunk_meta = reinterpret_cast<const int4 *>(p->d_chunk_meta); P.status = p->d_status;
-    P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = Ho; P.Wo = Wo; P.D = zout ? p->Gpad : p->D; P.Dpad = p->Dpad;
+    // Few tiles and many output channels: two blocks per tile, each with half of the channels (and of the weight stream).
+    const int nsplit = (!zout && t.fast && p->k == 3 && p->Dpad == p->D && p->D >= 256 && p->D % 32 == 0 && 2 * t.tiles() <= p->sm_count) ? 2 : 1;
+    const int Dloc = p->Dpad / nsplit;
+    P.nsplit = nsplit; P.Dtot = zout ? p->Gpad : p->D; P.Dpad_tot = p->Dpad;
+    P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = Ho; P.Wo = Wo; P.D = zout ? p->Gpad : (nsplit > 1 ? Dloc : p->D); P.Dpad = Dloc;
     P.G = p->G; P.nchunks = p->nchunks; P.stride = p->stride; P.pad = p->pad;
     P.relu = p->opt_relu;
     P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
@@ -808,15 +836,15 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     P.spg_shift = t.spg == 2 ? 1 : 0;
     P.ostage = tma_out ? t.ostage : 0;
     P.box_bytes = t.box_bytes; P.slot_bytes = t.slot_bytes;
-    P.nhalf = p->Dpad > 256 ? 2 : 1;
-    P.unit_bytes = (p->Dpad > 256 ? 256 : p->Dpad) * kChunk * 2;
-    P.acc_cols = tmem_cols_for(p->Dpad);
+    P.nhalf = Dloc > 256 ? 2 : 1;
+    P.unit_bytes = (Dloc > 256 ? 256 : Dloc) * kChunk * 2;
+    P.acc_cols = tmem_cols_for(Dloc);
     P.nacc = P.acc_cols <= 256 ? 2 : 1;
     P.a_kmajor = zout ? 1 : p->opt_a_layout;
     P.dw_math = p->opt_dw_math;
     P.zout = zout ? 1 : 0;
     const size_t smem = t.smem;     // one block per SM (register file), so the TMEM columns are never oversubscribed
-    const int grid = P.ntiles < p->sm_count ? P.ntiles : p->sm_count;
+    const int grid = nsplit > 1 ? P.ntiles * nsplit : (P.ntiles < p->sm_count ? P.ntiles : p->sm_count);
     const int dev = p->device;
     gdws_status_t rc;
     if (t.fast == 1 && p->k == 3 && p->stride == 1) rc = launch_fast<3, 1, 1>(P, dev, grid, smem, st);
