@@ -62,7 +62,7 @@ def layer_numbers(spec: gi.LayerSpec, G: int):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (key: config, layer, path).  An entry is removed when its kernel changes.
-TRAFFIC_BYTES_PER_LAUNCH = {(1, 0, "fused"): 9169152}   # y (8.39 MB) stays in L2 within the captured launch
+TRAFFIC_BYTES_PER_LAUNCH = {(1, 0, "fused"): 9181696}   # y (8.39 MB) stays in L2 within the captured launch
 
 
 def layer_roofline_us(macs, nbytes, peaks, sustained=False):
