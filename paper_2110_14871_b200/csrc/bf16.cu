@@ -77,6 +77,7 @@ gdws_status_t bf16_pack(gdws_plan_s *p, const void *dw_w, const void *pw_w, cons
                                             p->d_dw, p->d_dwpack);
     pack_bias_kernel<<<(p->Dpad + 255) / 256, 256, 0, st>>>(bias, p->D, p->Dpad, p->d_bias);
     p->launches += 3;
+    tc_pack(p, dw_w, pw_w, is_bf16, st);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "weight pack launch");
     p->packed = true;

@@ -1,0 +1,686 @@
+// Fused GDWS forward for bf16 NHWC tensors on sm_100a with BOTH stages on the tensor cores.
+//
+// GDW stage as a sum of k*k small GEMMs (Section 3.1, Definition of the (C,K,g) GDW convolution).  For filter
+// tap (u,v) the GDW output of a tile of 128 pixels and a window of 16 input channels is
+//     z[pixel, i] += x[pixel shifted by (u,v), c] * B_uv[c, i],   B_uv[c, i] = K[i,u,v] if c = c(i), else 0,
+// i.e. a [128 x 16] x [16 x n] product per tap whose B operand has one non-zero per column.  The A operand is
+// not copied per tap: the staged input box lies in shared memory as [8-channel group][row][column][8 channels],
+// which for every tap is a valid K-major tensor-core operand (8 consecutive pixels of an output row are 8
+// consecutive 16-byte entries) that differs from the next tap's only in its start address.  The fp32 result
+// z (128 lanes x n columns of TMEM) is read back by four converter warps, rounded to bf16 and written as the
+// K-major A operand of the pointwise stage (Property 1: W_P is M x G), whose products accumulate in a second
+// TMEM region over all windows of the tile.  The ALUs only round z, scatter the filter taps into the B
+// operands and run the epilogue; they execute no multiply of the GDW stage.
+//
+// One persistent block of 16 warps per SM walks over work items (tile of 128 output pixels x block of up to
+// 256 output channels).  Roles, coupled by mbarriers only:
+//   warp 0 (one lane)  issues every tcgen05.mma: for chunk u the k*k GDW products, then the PW products of
+//                      chunk u-1 (whose z is being converted meanwhile);
+//   warp 1 (one lane)  fetches the input boxes by TMA (rank-5 view of x: 8 channels, W, H, N, C/8);
+//   warp 2 (one lane)  streams the packed pointwise weights (bulk copies into a ring of 16-channel slabs);
+//   warps 4-7          converter: TMEM z -> bf16 -> ring of 16-channel operand slabs;
+//   warps 8-11         epilogue: TMEM y -> bias, ReLU, bf16 -> global memory (TMA store or direct);
+//   warps 12-15        builder: one thread per intermediate channel of the chunk scatters its k taps of a filter
+//                      row into a B operand buffer that is otherwise zero, and clears what it wrote when the
+//                      buffer comes back.
+// All operands use the un-swizzled K-major canonical layout: core matrices of 8 rows x 16 bytes stored
+// contiguously, `leading byte offset` between the two core matrices along K, `stride byte offset` between
+// 8-row groups.  Every wait is bounded (see mbar_wait).
+#include <string.h>
+
+#include <algorithm>
+
+#include "sm100.cuh"
+
+namespace gdws {
+
+static_assert(sizeof(TcChunk) == 32, "chunk table entries are copied as two 16-byte words");
+
+constexpr int kTcThreads = 512;
+constexpr int kTcNU = 4;              // chunks in flight per ring (barriers per ring)
+constexpr int kTcMaxNB = 4;           // B operand buffers of the GDW stage
+constexpr int kTcMaxNX = 4;           // input box slots
+constexpr int kTcMaxTaps = 25;
+constexpr int kTcZCol = 256;          // TMEM columns 256..511: two GDW accumulators of up to 128 columns
+constexpr int kTcSlab = 4096;         // bytes of one z slab: 128 pixels x 16 channels of bf16
+constexpr int kTcMaxChunks = 256;
+
+struct alignas(64) TcParams {
+    CUtensorMap tmap_x;          // x as (8, W, H, N, C/8) bf16
+    CUtensorMap tmap_y;          // y as (D, Wo, Ho, N) bf16, box (64, PW, PH, TN), 128-byte swizzle (when ostage != 0)
+    uint16_t *y;
+    const uint16_t *filt;
+    const uint16_t *pw;
+    const float *bias;
+    const TcChunk *chunks;
+    int *status;
+    int N, Ho, Wo, D, Dloc, Dpad_tot, nparts, nchunks, pad, relu;
+    int TN, PH, PW, tiles_h, tiles_w, nitems;
+    int nloads, xbox_bytes;
+    int load_dw[kTcMaxTaps], load_dh[kTcMaxTaps];
+    uint32_t load_off[kTcMaxTaps];
+    uint32_t tap_off[kTcMaxTaps];
+    uint32_t a_lbo, a_sbo;       // GDW A operand: bytes between the two 8-channel planes, between 8-pixel groups
+    int nb, nx, nz, nw, nacc;
+    uint32_t bbuf_bytes, bplane, b_lbo, xslot_bytes, wslab_bytes;
+    uint32_t off_b, off_z, off_w, off_x, off_tab;    // from the 1024-aligned base; the output staging comes first
+    int ostage, rec_hw, nslabs_total, bias_len;
+};
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *tmap, int c0, int c1, int c2, int c3, int c4,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor without swizzle (descriptor version 1): K-major canonical layout.
+__device__ __forceinline__ uint64_t make_sdesc_plain(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;
+    return d;
+}
+
+__device__ __forceinline__ void tc_warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+{
+    if ((threadIdx.x & 31) == 0) mbar_wait_relaxed<500>(bar, parity, abort_flag, status, code);
+    __syncwarp();
+}
+__device__ __forceinline__ void tc_warp_arrive(uint32_t bar)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
+
+// Producer-side bookkeeping of a ring of slabs whose consumer frees whole chunks (in order, one barrier
+// per chunk, kTcNU barriers in rotation).
+struct SlabRing {
+    int head = 0, free_slabs = 0, oldest = 0;
+};
+
+template <int K>
+__global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_constant__ TcParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    // xfull[4] xfree[4] | bfull[4] bfree[4] | zfull[2] zfree[2] | zsfull[4] pwdone[4] wfull[4] | accfull[2] accfree[2]
+    __shared__ __align__(8) uint64_t bars[2 * kTcMaxNX + 2 * kTcMaxNB + 4 + 3 * kTcNU + 4];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t base_s = smem_u32(base);
+    const uint32_t o_s = base_s, b_s = base_s + P.off_b, z_s = base_s + P.off_z, w_s = base_s + P.off_w, x_s = base_s + P.off_x;
+    const uint32_t bar_xfull = smem_u32(&bars[0]), bar_xfree = bar_xfull + 8 * kTcMaxNX;
+    const uint32_t bar_bfull = bar_xfree + 8 * kTcMaxNX, bar_bfree = bar_bfull + 8 * kTcMaxNB;
+    const uint32_t bar_zfull = bar_bfree + 8 * kTcMaxNB, bar_zfree = bar_zfull + 16;
+    const uint32_t bar_zsfull = bar_zfree + 16, bar_pwdone = bar_zsfull + 8 * kTcNU, bar_wfull = bar_pwdone + 8 * kTcNU;
+    const uint32_t bar_accfull = bar_wfull + 8 * kTcNU, bar_accfree = bar_accfull + 16;
+    TcChunk *tab = reinterpret_cast<TcChunk *>(base + P.off_tab);
+    float *bias_sm = reinterpret_cast<float *>(tab + P.nchunks);
+    uint16_t *bold = reinterpret_cast<uint16_t *>(bias_sm + P.Dpad_tot);     // [nb][128]: what each builder thread wrote last
+    const uint32_t bias_s = smem_u32(bias_sm);
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int i = 0; i < kTcMaxNX; ++i) { mbar_init(bar_xfull + 8 * i, 1); mbar_init(bar_xfree + 8 * i, 1); }
+        for (int i = 0; i < kTcMaxNB; ++i) { mbar_init(bar_bfull + 8 * i, 4); mbar_init(bar_bfree + 8 * i, 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_zfull + 8 * i, 1); mbar_init(bar_zfree + 8 * i, 4);
+            mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4);
+        }
+        for (int i = 0; i < kTcNU; ++i) {
+            mbar_init(bar_zsfull + 8 * i, 4); mbar_init(bar_pwdone + 8 * i, 1); mbar_init(bar_wfull + 8 * i, 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512u);
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(P.chunks);
+        uint4 *dst = reinterpret_cast<uint4 *>(tab);
+        for (int i = tid; i < P.nchunks * 2; i += kTcThreads) dst[i] = __ldg(src + i);
+        for (int d = tid; d < P.Dpad_tot; d += kTcThreads) bias_sm[d] = d < P.bias_len ? __ldg(P.bias + d) : 0.f;
+        for (int i = tid; i < P.nb * 128; i += kTcThreads) bold[i] = 0xFFFFu;
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        const uint32_t nb16 = (uint32_t)P.nb * P.bbuf_bytes / 16u;
+        for (uint32_t i = tid; i < nb16; i += kTcThreads) sts128(b_s + i * 16u, zero);
+        fence_proxy_async();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+
+    const int my_items = ((int)P.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int total = my_items * P.nchunks;
+    const int tiles_hw = P.tiles_h * P.tiles_w;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------- MMA issue ----------------
+            const uint32_t idesc_pw = make_idesc(P.Dloc, false);
+            uint32_t xslot = 0, xpar = 0, bslot = 0, bpar = 0, zhead = 0, whead = 0;
+            int q = 0;                  // chunk index of unit u within its work item
+            int qp = 0, itp = 0;        // the same for unit u - 1, and its work item
+            for (int u = 0; u <= total; ++u) {
+                if (u < total) {
+                    const TcChunk ch = tab[q];
+                    if (ch.flags & 1) mbar_wait(bar_xfull + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitOperand);
+                    if (u >= 2) mbar_wait(bar_zfree + 8 * (u & 1), ((u >> 1) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                    tc_fence_after();
+                    const uint32_t idesc = make_idesc(ch.npad, false);
+                    const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
+                    const uint32_t abase = x_s + xslot * P.xslot_bytes;
+#pragma unroll 1
+                    for (int ur = 0; ur < K; ++ur) {
+                        mbar_wait(bar_bfull + 8 * bslot, bpar, &abort_flag, P.status, kStatusWaitOperand);
+                        tc_fence_after();
+                        const uint32_t bb = b_s + bslot * P.bbuf_bytes;
+#pragma unroll
+                        for (int v = 0; v < K; ++v)
+                            umma_bf16(d_z, make_sdesc_plain(abase + P.tap_off[ur * K + v], P.a_lbo, P.a_sbo),
+                                      make_sdesc_plain(bb + (uint32_t)v * P.bplane, P.b_lbo, 128u), idesc, (ur | v) != 0);
+                        umma_commit(bar_bfree + 8 * bslot);
+                        if (++bslot == (uint32_t)P.nb) { bslot = 0; bpar ^= 1; }
+                    }
+                    umma_commit(bar_zfull + 8 * (u & 1));
+                    if (ch.flags & 2) {
+                        umma_commit(bar_xfree + 8 * xslot);
+                        if (++xslot == (uint32_t)P.nx) { xslot = 0; xpar ^= 1; }
+                    }
+                    if (++q == P.nchunks) q = 0;
+                }
+                if (u > 0) {
+                    const int v = u - 1;
+                    const int buf = itp % P.nacc;
+                    if (qp == 0 && itp >= P.nacc)
+                        mbar_wait(bar_accfree + 8 * buf, ((itp / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                    const uint32_t up = (uint32_t)(v & (kTcNU - 1)), par = (uint32_t)(v / kTcNU) & 1u;
+                    mbar_wait(bar_wfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
+                    mbar_wait(bar_zsfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
+                    tc_fence_after();
+                    const int ns = tab[qp].npad >> 4;
+                    const uint32_t d_y = tmem + (uint32_t)(buf * 128);
+#pragma unroll 1
+                    for (int s = 0; s < ns; ++s) {
+                        umma_bf16(d_y, make_sdesc_plain(z_s + zhead * kTcSlab, 2048u, 128u),
+                                  make_sdesc_plain(w_s + whead * P.wslab_bytes, (uint32_t)P.Dloc * 16u, 128u), idesc_pw,
+                                  (qp | s) != 0);
+                        if (++zhead == (uint32_t)P.nz) zhead = 0;
+                        if (++whead == (uint32_t)P.nw) whead = 0;
+                    }
+                    umma_commit(bar_pwdone + 8 * up);
+                    if (qp == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
+                    if (++qp == P.nchunks) { qp = 0; ++itp; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------- input loader ----------------
+            int box = 0;
+            uint32_t xslot = 0;
+            for (int it = 0; it < my_items; ++it) {
+                const int item = (int)blockIdx.x + it * (int)gridDim.x;
+                int tile = item / P.nparts;
+                const int bn = tile / tiles_hw;
+                tile -= bn * tiles_hw;
+                const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+                const int n0 = bn * P.TN, hi0 = bh * P.PH - P.pad, wi0 = bw * P.PW - P.pad;
+                for (int q = 0; q < P.nchunks; ++q) {
+                    const TcChunk ch = tab[q];
+                    if (!(ch.flags & 1)) continue;
+                    if (box >= P.nx)
+                        mbar_wait_relaxed<500>(bar_xfree + 8 * xslot, (uint32_t)((box / P.nx) - 1) & 1u, &abort_flag, P.status,
+                                               kStatusWaitStage);
+                    mbar_expect_tx(bar_xfull + 8 * xslot, (uint32_t)P.xbox_bytes);
+                    const uint32_t dst = x_s + xslot * P.xslot_bytes;
+                    for (int l = 0; l < P.nloads; ++l)
+                        tma_load_5d(dst + P.load_off[l], &P.tmap_x, 0, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, ch.cbase >> 3,
+                                    bar_xfull + 8 * xslot);
+                    ++box;
+                    if (++xslot == (uint32_t)P.nx) xslot = 0;
+                }
+            }
+        }
+    } else if (warp == 2) {
+        if (lane == 0) {
+            // ---------------- pointwise-weight loader ----------------
+            SlabRing ring;
+            ring.free_slabs = P.nw;
+            int q = 0, it = 0;
+            for (int v = 0; v < total; ++v) {
+                const TcChunk ch = tab[q];
+                const int ns = ch.npad >> 4;
+                while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
+                    const int o = ring.oldest;
+                    mbar_wait_relaxed<500>(bar_pwdone + 8 * (o & (kTcNU - 1)), (uint32_t)(o / kTcNU) & 1u, &abort_flag, P.status,
+                                           kStatusWaitStage);
+                    ring.free_slabs += tab[o % P.nchunks].npad >> 4;
+                    ++ring.oldest;
+                }
+                const int part = ((int)blockIdx.x + it * (int)gridDim.x) % P.nparts;
+                const uint32_t bar = bar_wfull + 8 * (v & (kTcNU - 1));
+                mbar_expect_tx(bar, (uint32_t)ns * P.wslab_bytes);
+                const uint16_t *src = P.pw + ((size_t)part * P.nslabs_total + ch.slab0) * 16 * P.Dloc;
+                const int first = ns < P.nw - ring.head ? ns : P.nw - ring.head;
+                bulk_g2s(w_s + (uint32_t)ring.head * P.wslab_bytes, src, (uint32_t)first * P.wslab_bytes, bar);
+                if (first < ns) bulk_g2s(w_s, src + (size_t)first * 16 * P.Dloc, (uint32_t)(ns - first) * P.wslab_bytes, bar);
+                ring.head = (ring.head + ns) % P.nw;
+                ring.free_slabs -= ns;
+                if (++q == P.nchunks) { q = 0; ++it; }
+            }
+        }
+    } else if (warp >= 4 && warp < 8) {
+        // ---------------- converter: z (fp32, TMEM) -> bf16 operand slabs ----------------
+        const int lg = warp & 3;
+        const uint32_t r = (uint32_t)(lg * 32 + lane);
+        SlabRing ring;
+        ring.free_slabs = P.nz;
+        int q = 0;
+        for (int v = 0; v < total; ++v) {
+            const int ns = tab[q].npad >> 4;
+            while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
+                const int o = ring.oldest;
+                tc_warp_wait(bar_pwdone + 8 * (o & (kTcNU - 1)), (uint32_t)(o / kTcNU) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                ring.free_slabs += tab[o % P.nchunks].npad >> 4;
+                ++ring.oldest;
+            }
+            tc_warp_wait(bar_zfull + 8 * (v & 1), (uint32_t)(v >> 1) & 1u, &abort_flag, P.status, kStatusWaitMma);
+            tc_fence_after();
+            const uint32_t taddr = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(kTcZCol + 128 * (v & 1));
+            int slab = ring.head;
+#pragma unroll 1
+            for (int g = 0; g < ns; ++g) {
+                uint32_t acc[16];
+                tmem_ld16(taddr + (uint32_t)(g * 16), acc);
+                tmem_ld_wait();
+                uint4 lo, hi;
+                lo.x = pack_bf16x2(__uint_as_float(acc[0]), __uint_as_float(acc[1]));
+                lo.y = pack_bf16x2(__uint_as_float(acc[2]), __uint_as_float(acc[3]));
+                lo.z = pack_bf16x2(__uint_as_float(acc[4]), __uint_as_float(acc[5]));
+                lo.w = pack_bf16x2(__uint_as_float(acc[6]), __uint_as_float(acc[7]));
+                hi.x = pack_bf16x2(__uint_as_float(acc[8]), __uint_as_float(acc[9]));
+                hi.y = pack_bf16x2(__uint_as_float(acc[10]), __uint_as_float(acc[11]));
+                hi.z = pack_bf16x2(__uint_as_float(acc[12]), __uint_as_float(acc[13]));
+                hi.w = pack_bf16x2(__uint_as_float(acc[14]), __uint_as_float(acc[15]));
+                const uint32_t addr = z_s + (uint32_t)slab * kTcSlab + r * 16u;
+                sts128(addr, lo);              // channels 16g .. 16g+7 of this pixel: first core-matrix plane
+                sts128(addr + 2048u, hi);      // channels 16g+8 .. 16g+15: second plane
+                if (++slab == P.nz) slab = 0;
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            tc_warp_arrive(bar_zsfull + 8 * (v & (kTcNU - 1)));
+            tc_warp_arrive(bar_zfree + 8 * (v & 1));
+            ring.head = (ring.head + ns) % P.nz;
+            ring.free_slabs -= ns;
+            if (++q == P.nchunks) q = 0;
+        }
+    } else if (warp >= 8 && warp < 12) {
+        // ---------------- epilogue: TMEM -> bias / ReLU -> bf16 -> global ----------------
+        const int lg = warp & 3;
+        const int r = lg * 32 + lane;
+        const int hw = P.PH * P.PW;
+        const int tn = r / hw;
+        const int rem = r - tn * hw;
+        const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
+        const bool issuer = warp == 8 && lane == 0;
+        for (int it = 0; it < my_items; ++it) {
+            const int item = (int)blockIdx.x + it * (int)gridDim.x;
+            int tile = item / P.nparts;
+            const int part = item - tile * P.nparts;
+            const int bn = tile / tiles_hw;
+            tile -= bn * tiles_hw;
+            const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+            const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
+            const bool live = n < P.N && ho < P.Ho && wo < P.Wo;
+            uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D + part * P.Dloc;
+            const int dvalid = P.D - part * P.Dloc < P.Dloc ? P.D - part * P.Dloc : P.Dloc;
+            const int buf = it % P.nacc;
+            tc_warp_wait(bar_accfull + 8 * buf, (uint32_t)(it / P.nacc) & 1u, &abort_flag, P.status, kStatusWaitMma);
+            tc_fence_after();
+            const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * 128);
+            const uint32_t bias_part = bias_s + (uint32_t)(part * P.Dloc) * 4u;
+            if (P.ostage) {
+                // 64 output channels at a time through a staging buffer (rows in tile order = the order of a
+                // (64, PW, PH, TN) box of y; 16-byte pieces swizzled by row), stored by TMA, which clips the box.
+                const uint32_t row_s = o_s + (uint32_t)r * 128;
+                const int nblk = P.Dloc >> 6;
+                for (int cb = 0; cb < nblk; ++cb) {
+                    if (issuer) bulk_wait_read_all();
+                    named_bar_sync(1, 128);
+#pragma unroll 1
+                    for (int h4 = 0; h4 < 4; ++h4) {
+                        uint32_t acc[16], o[8];
+                        tmem_ld16(t_base + (uint32_t)(cb * 64 + h4 * 16), acc);
+                        tmem_ld_wait();
+                        float bv[16];
+                        bias16_shared(bias_part + (uint32_t)(cb * 64 + h4 * 16) * 4, bv);
+                        finish_row16(acc, bv, P.relu, o);
+                        sts128(row_s + (uint32_t)(((2 * h4) ^ (r & 7)) << 4), make_uint4(o[0], o[1], o[2], o[3]));
+                        sts128(row_s + (uint32_t)(((2 * h4 + 1) ^ (r & 7)) << 4), make_uint4(o[4], o[5], o[6], o[7]));
+                    }
+                    fence_proxy_async();
+                    if (cb == nblk - 1) {
+                        tc_fence_before();
+                        tc_warp_arrive(bar_accfree + 8 * buf);
+                    }
+                    named_bar_sync(1, 128);
+                    if (issuer) {
+                        tma_store_4d(o_s, &P.tmap_y, part * P.Dloc + cb * 64, bw * P.PW, bh * P.PH, bn * P.TN);
+                        bulk_commit();
+                    }
+                }
+            } else {
+                const int ngran = P.Dloc >> 4;
+                for (int j = 0; j < ngran; ++j) {
+                    uint32_t acc[16];
+                    tmem_ld16(t_base + (uint32_t)(j * 16), acc);
+                    tmem_ld_wait();
+                    if (live && j * 16 < dvalid) {
+                        float bv[16];
+                        uint32_t o[8];
+                        bias16_shared(bias_part + (uint32_t)j * 64, bv);
+                        finish_row16(acc, bv, P.relu, o);
+                        store_packed16(o, j * 16, dvalid, yrow);
+                    }
+                }
+                tc_fence_before();
+                tc_warp_arrive(bar_accfree + 8 * buf);
+            }
+        }
+        if (P.ostage && issuer) bulk_wait_all();
+    } else if (warp >= 12) {
+        // ---------------- builder: filter taps -> B operands of the GDW products ----------------
+        // Thread t owns intermediate slot t of the current chunk.  The B operand of tap (ur, v) is a [n x 16]
+        // K-major matrix whose row t has the tap's value in column `channel of slot t inside the window`.
+        const int t = tid - 384;
+        constexpr int RW = (1 + K * K + 7) / 8 * 4;         // 32-bit words of a filter record
+        const uint32_t rowoff = (uint32_t)((t >> 3) * 128 + (t & 7) * 16);
+        uint32_t rec[RW], nxt[RW];
+        auto load_rec = [&](const TcChunk &ch, uint32_t (&dst)[RW]) {
+            if (t < ch.npad) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(P.filt + ((size_t)ch.slab0 * 16 + t) * (RW * 2));
+#pragma unroll
+                for (int j = 0; j < RW / 4; ++j) {
+                    const uint4 w4 = __ldg(src + j);
+                    dst[4 * j] = w4.x; dst[4 * j + 1] = w4.y; dst[4 * j + 2] = w4.z; dst[4 * j + 3] = w4.w;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < RW; ++j) dst[j] = 0xFFFFu;
+            }
+        };
+        if (total > 0) load_rec(tab[0], nxt);
+        uint32_t bslot = 0;
+        int ub = 0, q = 0;
+        for (int v = 0; v < total; ++v) {
+#pragma unroll
+            for (int j = 0; j < RW; ++j) rec[j] = nxt[j];
+            if (++q == P.nchunks) q = 0;
+            if (v + 1 < total) load_rec(tab[q], nxt);
+            const uint32_t cw = rec[0] & 0xFFFFu;
+            const bool valid = cw != 0xFFFFu;
+            const uint32_t off = (cw >> 3) * P.b_lbo + rowoff + (cw & 7u) * 2u;
+#pragma unroll
+            for (int ur = 0; ur < K; ++ur) {
+                if (ub >= P.nb) tc_warp_wait(bar_bfree + 8 * bslot, (uint32_t)((ub / P.nb) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                const uint32_t bb = b_s + bslot * P.bbuf_bytes;
+                const uint32_t old = bold[bslot * 128 + t];
+                if (old != 0xFFFFu) {
+#pragma unroll
+                    for (int vv = 0; vv < K; ++vv) sts16(bb + (uint32_t)vv * P.bplane + old, (uint16_t)0);
+                }
+                if (valid) {
+#pragma unroll
+                    for (int vv = 0; vv < K; ++vv) {
+                        const int h = 1 + ur * K + vv;          // 16-bit word of the record holding tap (ur, vv)
+                        sts16(bb + (uint32_t)vv * P.bplane + off, (uint16_t)(rec[h >> 1] >> (16 * (h & 1))));
+                    }
+                }
+                bold[bslot * 128 + t] = (uint16_t)(valid ? off : 0xFFFFu);
+                fence_proxy_async();
+                tc_warp_arrive(bar_bfull + 8 * bslot);
+                ++ub;
+                if (++bslot == (uint32_t)P.nb) bslot = 0;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    __syncwarp();
+    if (warp == 0) tmem_dealloc(tmem, 512u);
+}
+
+// ------------------------------------------------------------------------------------------
+// Weight packing
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float tc_load_weight(const void *w, size_t idx, int is_bf16)
+{
+    return is_bf16 ? bf16_bits_to_float(((const uint16_t *)w)[idx]) : ((const float *)w)[idx];
+}
+
+// dw_w[G][k][k] -> one record per intermediate slot: the slot's channel inside its 16-channel window
+// (0xFFFF for the padding slots of a chunk), then the k*k taps as bf16.
+__global__ void tc_pack_filt_kernel(const void *__restrict__ dw, int is_bf16, int k2, int rec_hw, const TcChunk *__restrict__ chunks,
+                                    const int32_t *__restrict__ chan, uint16_t *__restrict__ out)
+{
+    const TcChunk ch = chunks[blockIdx.x];
+    for (int e = threadIdx.x; e < ch.npad * rec_hw; e += blockDim.x) {
+        const int t = e / rec_hw, h = e - t * rec_hw;
+        uint16_t val = 0;
+        if (h == 0) val = t < ch.n ? (uint16_t)(chan[ch.i0 + t] - ch.cbase) : (uint16_t)0xFFFFu;
+        else if (h <= k2 && t < ch.n) val = float_to_bf16_bits(tc_load_weight(dw, (size_t)(ch.i0 + t) * k2 + (h - 1), is_bf16));
+        out[((size_t)ch.slab0 * 16 + t) * rec_hw + h] = val;
+    }
+}
+
+// pw_w[D][G] -> [part][slab][8-channel plane][output channel][8] bf16: per 16 intermediate slots one K-major
+// operand slab of the pointwise product, core matrices of 8 output channels x 8 slots stored contiguously.
+__global__ void tc_pack_pw_kernel(const void *__restrict__ pw, int is_bf16, int D, int G, int Dloc, int nslabs,
+                                  const TcChunk *__restrict__ chunks, uint16_t *__restrict__ out)
+{
+    const TcChunk ch = chunks[blockIdx.x];
+    const int part = blockIdx.y;
+    const int per_slab = 16 * Dloc;
+    for (int e = threadIdx.x; e < (ch.npad >> 4) * per_slab; e += blockDim.x) {
+        const int s = e / per_slab;
+        int rem = e - s * per_slab;
+        const int kg = rem / (8 * Dloc);
+        rem -= kg * 8 * Dloc;
+        const int dl = rem >> 3, el = rem & 7;
+        const int t = s * 16 + kg * 8 + el, d = part * Dloc + dl;
+        float val = 0.f;
+        if (t < ch.n && d < D) val = tc_load_weight(pw, (size_t)d * G + ch.i0 + t, is_bf16);
+        out[((size_t)part * nslabs + ch.slab0 + s) * per_slab + (size_t)kg * 8 * Dloc + dl * 8 + el] = float_to_bf16_bits(val);
+    }
+}
+
+void tc_pack(gdws_plan_s *p, const void *dw_w, const void *pw_w, int is_bf16, cudaStream_t st)
+{
+    if (!p->tc_ok) return;
+    const int nch = (int)p->tc_chunks.size();
+    tc_pack_filt_kernel<<<nch, 256, 0, st>>>(dw_w, is_bf16, p->k * p->k, p->tc_rec_hw, p->d_tc_chunks, p->d_chan, p->d_tc_filt);
+    tc_pack_pw_kernel<<<dim3(nch, p->tc_nparts), 256, 0, st>>>(pw_w, is_bf16, p->D, p->G, p->tc_dloc, p->tc_nslabs, p->d_tc_chunks,
+                                                            p->d_tc_pw);
+    p->launches += 2;
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+namespace {
+
+struct TcGeom {
+    int layout = 0;              // 1: one box with halo rows (one image per tile), 2: one copy per filter row,
+                                 // 3: one copy per tap (maps at most 4 wide)
+    int TN = 0, PH = 0, PW = 0, IW = 0;
+    int tiles_n = 0, tiles_h = 0, tiles_w = 0;
+    int nloads = 0, xbox = 0;
+    int64_t tiles() const { return (int64_t)tiles_n * tiles_h * tiles_w; }
+};
+
+bool tc_geometry(const gdws_plan_s *p, int n, int Ho, int Wo, TcGeom *out)
+{
+    const int k = p->k;
+    double best = 1e300;
+    bool found = false;
+    auto consider = [&](int layout, int TN, int PH, int PW) {
+        TcGeom g;
+        g.layout = layout; g.TN = TN; g.PH = PH; g.PW = PW;
+        g.tiles_n = (n + TN - 1) / TN; g.tiles_h = (Ho + PH - 1) / PH; g.tiles_w = (Wo + PW - 1) / PW;
+        g.IW = layout == 3 ? 4 : PW + k - 1;
+        g.nloads = layout == 1 ? 1 : (layout == 2 ? k : k * k);
+        g.xbox = layout == 1 ? 2 * (PH + k - 1) * g.IW * 16 : (layout == 2 ? k * 2 * 16 * g.IW * 16 : k * k * 4096);
+        const double cost = (double)g.tiles() * (1.0 + 0.02 * (g.nloads - 1));
+        if (cost < best) { best = cost; *out = g; found = true; }
+    };
+    if (Wo > 4) {
+        consider(1, 1, 16, 8);
+        for (int PH = 8; PH >= 1; PH >>= 1) consider(2, 16 / PH, PH, 8);
+    } else {
+        for (int PH = 32; PH >= 2; PH >>= 1) consider(3, 32 / PH, PH, 4);
+    }
+    return found;
+}
+
+}  // namespace
+
+gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t st)
+{
+    if (!p->tc_ok) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: layer not covered (stride 1, k <= 5, C and D multiples of 8)");
+    const int nchunks = (int)p->tc_chunks.size();
+    if (nchunks > kTcMaxChunks) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: %d chunks (at most %d)", nchunks, kTcMaxChunks);
+    if (p->sm_count <= 0) {
+        cudaError_t e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute(MultiProcessorCount)");
+    }
+    const int Ho = y->h, Wo = y->w, k = p->k;
+    TcGeom g;
+    if (!tc_geometry(p, x->n, Ho, Wo, &g)) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: no tile");
+    const int64_t nitems = g.tiles() * p->tc_nparts;
+    if (nitems > 0x7fffffffLL) return fail(GDWS_ERR_UNSUPPORTED, "too many tiles");
+    tensor_map_encode_fn encode = encode_fn();
+    if (!encode) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+
+    TcParams P;
+    memset(&P, 0, sizeof(P));
+    const int Dloc = p->tc_dloc, m = p->tc_maxslabs;
+    const uint32_t nmax = Dloc > 128 ? 96u : 128u;
+    P.bplane = nmax * 32u; P.b_lbo = nmax * 16u; P.bbuf_bytes = (uint32_t)k * P.bplane;
+    P.wslab_bytes = (uint32_t)Dloc * 32u;
+    P.xslot_bytes = (uint32_t)((g.xbox + 127) / 128 * 128);
+    // Shared memory: output staging (optional) | B operand buffers | z slabs | weight slabs | input boxes | tables
+    const bool can_stage = p->D % 64 == 0 && Dloc % 64 == 0 && ((uintptr_t)y->ptr & 15) == 0 && nitems > p->sm_count;
+    const size_t tables = (size_t)nchunks * sizeof(TcChunk) + (size_t)p->tc_nparts * Dloc * 4 + kTcMaxNB * 256 + 256;
+    double best_score = -1;
+    int b_ost = 0, b_nx = 0, b_nb = 0, b_nz = 0, b_nw = 0;
+    for (int ost = can_stage ? 1 : 0; ost >= 0; --ost)
+        for (int nx = 3; nx >= 2; --nx)
+            for (int nb = 4; nb >= 2; --nb)
+                for (int nz = 2 * m; nz >= m; --nz) {
+                    const size_t fixed = 1024 + (ost ? 16384 : 0) + (size_t)nb * P.bbuf_bytes + (size_t)nz * kTcSlab +
+                                         (size_t)nx * P.xslot_bytes + tables;
+                    if (fixed + (size_t)m * P.wslab_bytes > (size_t)kMaxSmem) continue;
+                    int nw = (int)(((size_t)kMaxSmem - fixed) / P.wslab_bytes);
+                    if (nw > 3 * m) nw = 3 * m;
+                    const double score = 2.0 * std::min(nw, 2 * m) / m + 0.3 * std::min(nw, 3 * m) / m + 1.5 * nz / m + 0.4 * ost +
+                                         0.25 * nx + 0.15 * nb;
+                    if (score > best_score) { best_score = score; b_ost = ost; b_nx = nx; b_nb = nb; b_nz = nz; b_nw = nw; }
+                }
+    if (best_score < 0) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: shared memory does not fit this layer");
+    P.ostage = b_ost ? 16384 : 0; P.nx = b_nx; P.nb = b_nb; P.nz = b_nz; P.nw = b_nw;
+    P.off_b = (uint32_t)P.ostage;
+    P.off_z = P.off_b + (uint32_t)P.nb * P.bbuf_bytes;
+    P.off_w = P.off_z + (uint32_t)P.nz * kTcSlab;
+    P.off_x = P.off_w + (uint32_t)P.nw * P.wslab_bytes;
+    P.off_tab = P.off_x + (uint32_t)P.nx * P.xslot_bytes;
+    size_t smem = 1024 + (size_t)P.off_tab + tables;
+    if (smem < (size_t)kMaxSmem / 2 + 4096) smem = (size_t)kMaxSmem / 2 + 4096;   // one block per SM: it owns all of TMEM
+    if (smem > (size_t)kMaxSmem) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: shared memory plan exceeds the limit");
+
+    {   // x as a rank-5 tensor, innermost first: 8 channels, width, height, batch, 8-channel group
+        const cuuint64_t dims[5] = {8, (cuuint64_t)x->w, (cuuint64_t)x->h, (cuuint64_t)x->n, (cuuint64_t)(p->C / 8)};
+        const cuuint64_t strides[4] = {(cuuint64_t)p->C * 2, (cuuint64_t)x->w * p->C * 2, (cuuint64_t)x->h * x->w * p->C * 2, 16};
+        cuuint32_t box[5] = {8, (cuuint32_t)g.IW, 0, (cuuint32_t)g.TN, 2};
+        box[2] = (cuuint32_t)(g.layout == 1 ? g.PH + k - 1 : g.PH);
+        const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        const CUresult r = encode(&P.tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x->ptr, dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled (x, rank 5) failed with code %d", (int)r);
+    }
+    if (P.ostage) {
+        const cuuint64_t dims[4] = {(cuuint64_t)p->D, (cuuint64_t)Wo, (cuuint64_t)Ho, (cuuint64_t)x->n};
+        const cuuint64_t strides[3] = {(cuuint64_t)p->D * 2, (cuuint64_t)Wo * p->D * 2, (cuuint64_t)Ho * Wo * p->D * 2};
+        const cuuint32_t box[4] = {64, (cuuint32_t)g.PW, (cuuint32_t)g.PH, (cuuint32_t)g.TN};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        const CUresult r = encode(&P.tmap_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, y->ptr, dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled (y) failed with code %d", (int)r);
+    } else {
+        P.tmap_y = P.tmap_x;
+    }
+    // Where each copy of the box goes, and where the A operand of tap (u, v) starts.
+    const uint32_t px = 16;      // bytes of one staged pixel within a plane (8 channels)
+    if (g.layout == 1) {
+        P.nloads = 1; P.load_dw[0] = 0; P.load_dh[0] = 0; P.load_off[0] = 0;
+        P.a_lbo = (uint32_t)((g.PH + k - 1) * g.IW) * px; P.a_sbo = (uint32_t)g.IW * px;
+        for (int u = 0; u < k; ++u) for (int v = 0; v < k; ++v) P.tap_off[u * k + v] = (uint32_t)(u * g.IW + v) * px;
+    } else if (g.layout == 2) {
+        const uint32_t copy = 2u * 16u * (uint32_t)g.IW * px;
+        P.nloads = k;
+        for (int u = 0; u < k; ++u) { P.load_dw[u] = 0; P.load_dh[u] = u; P.load_off[u] = (uint32_t)u * copy; }
+        P.a_lbo = 16u * (uint32_t)g.IW * px; P.a_sbo = (uint32_t)g.IW * px;
+        for (int u = 0; u < k; ++u) for (int v = 0; v < k; ++v) P.tap_off[u * k + v] = (uint32_t)u * copy + (uint32_t)v * px;
+    } else {
+        P.nloads = k * k;
+        for (int u = 0; u < k; ++u) for (int v = 0; v < k; ++v) {
+            P.load_dw[u * k + v] = v; P.load_dh[u * k + v] = u; P.load_off[u * k + v] = (uint32_t)(u * k + v) * 4096u;
+            P.tap_off[u * k + v] = (uint32_t)(u * k + v) * 4096u;
+        }
+        P.a_lbo = 2048u; P.a_sbo = 128u;
+    }
+    P.xbox_bytes = g.xbox;
+    P.y = (uint16_t *)y->ptr; P.filt = p->d_tc_filt; P.pw = p->d_tc_pw; P.bias = p->d_bias; P.chunks = p->d_tc_chunks;
+    P.status = p->d_status;
+    P.N = x->n; P.Ho = Ho; P.Wo = Wo; P.D = p->D; P.Dloc = Dloc; P.Dpad_tot = p->tc_nparts * Dloc; P.nparts = p->tc_nparts;
+    P.nchunks = nchunks; P.pad = p->pad; P.relu = p->opt_relu;
+    P.TN = g.TN; P.PH = g.PH; P.PW = g.PW; P.tiles_h = g.tiles_h; P.tiles_w = g.tiles_w; P.nitems = (int)nitems;
+    P.nacc = Dloc <= 128 ? 2 : 1;
+    P.rec_hw = p->tc_rec_hw; P.nslabs_total = p->tc_nslabs;
+    P.bias_len = p->Dpad;
+
+    const int grid = (int)(nitems < p->sm_count ? nitems : p->sm_count);
+    cudaError_t e = cudaSuccess;
+#define GDWS_TC_LAUNCH(KK)                                                                                              \
+    do {                                                                                                                \
+        static bool attr_set[64] = {};                                                                                  \
+        if (!attr_set[p->device & 63]) {                                                                                \
+            e = cudaFuncSetAttribute(fused_tc_kernel<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);       \
+            if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_tc_kernel)");                         \
+            attr_set[p->device & 63] = true;                                                                            \
+        }                                                                                                               \
+        fused_tc_kernel<KK><<<grid, kTcThreads, smem, st>>>(P);                                                         \
+    } while (0)
+    switch (k) {
+    case 1: GDWS_TC_LAUNCH(1); break;
+    case 2: GDWS_TC_LAUNCH(2); break;
+    case 3: GDWS_TC_LAUNCH(3); break;
+    case 4: GDWS_TC_LAUNCH(4); break;
+    case 5: GDWS_TC_LAUNCH(5); break;
+    default: return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: k=%d", k);
+    }
+#undef GDWS_TC_LAUNCH
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "fused_tc_kernel launch");
+    p->launches++;
+    return GDWS_OK;
+}
+
+}  // namespace gdws

@@ -23,6 +23,19 @@ enum : int {
     kStatusWaitMma = 4,     // wait for the tensor-core commit ran out
 };
 
+// One unit of work of the tensor-core GDW path: the intermediate channels i0 .. i0+n-1, all fed by the
+// 16 input channels cbase .. cbase+15 (a "window"; cbase is a multiple of 16).  Windows whose channels
+// produce more than the path's limit of intermediate channels are cut into several chunks.
+struct TcChunk {
+    int32_t cbase;       // first input channel of the window
+    int32_t i0;          // first intermediate channel (canonical order, Property 2)
+    int32_t n;           // intermediate channels of the chunk
+    int32_t npad;        // n rounded up to a multiple of 16 (columns of the GDW product, K of the PW product)
+    int32_t slab0;       // index of the chunk's first 16-channel slab in the packed arrays
+    int32_t flags;       // 1: first chunk of its window (its input box is fetched), 2: last chunk of its window
+    int32_t reserved0, reserved1;
+};
+
 struct Tile {
     int TN = 0, PH = 0, PW = 0;      // images x rows x columns of output pixels per 128-row tile
     int tiles_n = 0, tiles_h = 0, tiles_w = 0;
@@ -59,6 +72,14 @@ struct gdws_plan_s {
     int cbox = 0, nboxes = 0;
     std::vector<int32_t> chunk_meta; // 4 ints per chunk
 
+    // Tensor-core GDW path (fused_tc.cu): chunk list, output-channel split, packed sizes.
+    bool tc_ok = false;              // the layer is one the path covers (stride 1, k <= 5, ...)
+    std::vector<gdws::TcChunk> tc_chunks;
+    int tc_nslabs = 0;               // sum of npad / 16 over the chunks
+    int tc_maxslabs = 0;             // largest npad / 16 of one chunk
+    int tc_nparts = 1, tc_dloc = 0;  // blocks per tile along D, output channels per block (multiple of 16, <= 256)
+    int tc_rec_hw = 0;               // 16-bit words per filter record (channel slot, then k*k taps; multiple of 8)
+
     int opt_path = GDWS_PATH_AUTO;
     int opt_relu = 0;
     int opt_tile = 0;
@@ -76,6 +97,9 @@ struct gdws_plan_s {
     uint32_t *d_dwpack = nullptr;  // [Gpad][wstride]: k*k fp32 filter taps, then the channel's index within its K chunk's slot
     uint16_t *d_pw_img = nullptr;  // [nchunks][Dpad*64] bf16, 128-byte-swizzled K-major operand images
     float *d_bias = nullptr;       // [Dpad]
+    gdws::TcChunk *d_tc_chunks = nullptr;
+    uint16_t *d_tc_filt = nullptr; // [tc_nslabs * 16][tc_rec_hw]: per intermediate slot, channel index inside the window and the taps (bf16)
+    uint16_t *d_tc_pw = nullptr;   // [tc_nparts][tc_nslabs][2][tc_dloc][8] bf16: pointwise weights, one K = 16 operand slab per 16 slots
     int *d_status = nullptr;       // device status word
     bool packed = false;
 
@@ -113,5 +137,9 @@ gdws_status_t bf16_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cu
 gdws_status_t bf16_pointwise(gdws_plan_s *p, const void *z, gdws_tensor_t *y, cudaStream_t s);
 gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t s);
 gdws_status_t bf16_depthwise_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cudaStream_t s);
+
+// fused_tc.cu
+void tc_pack(gdws_plan_s *p, const void *dw_w, const void *pw_w, int is_bf16, cudaStream_t s);
+gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t s);
 
 }  // namespace gdws

@@ -63,6 +63,10 @@ static void free_device(gdws_plan_s *p)
     cudaFree(p->d_pw_img);
     cudaFree(p->d_bias);
     cudaFree(p->d_status);
+    cudaFree(p->d_tc_chunks);
+    cudaFree(p->d_tc_filt);
+    cudaFree(p->d_tc_pw);
+    p->d_tc_chunks = nullptr; p->d_tc_filt = nullptr; p->d_tc_pw = nullptr;
     cudaFree(p->stage_x);
     cudaFree(p->stage_y);
     cudaSetDevice(cur);
@@ -95,12 +99,19 @@ gdws_status_t ensure_device(gdws_plan_s *p)
     GDWS_TRY_ALLOC(p->d_pw_img, img);
     GDWS_TRY_ALLOC(p->d_bias, sizeof(float) * p->Dpad);
     GDWS_TRY_ALLOC(p->d_status, sizeof(int));
+    if (p->tc_ok) {
+        GDWS_TRY_ALLOC(p->d_tc_chunks, sizeof(TcChunk) * p->tc_chunks.size());
+        GDWS_TRY_ALLOC(p->d_tc_filt, sizeof(uint16_t) * (size_t)p->tc_nslabs * 16 * p->tc_rec_hw);
+        GDWS_TRY_ALLOC(p->d_tc_pw, sizeof(uint16_t) * (size_t)p->tc_nparts * p->tc_nslabs * 16 * p->tc_dloc);
+    }
 #undef GDWS_TRY_ALLOC
     p->device = dev;
     e = cudaMemcpy(p->d_off, p->off.data(), sizeof(int32_t) * (p->C + 1), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_chan, p->chan.data(), sizeof(int32_t) * p->Gpad, cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
         e = cudaMemcpy(p->d_chunk_meta, p->chunk_meta.data(), sizeof(int32_t) * 4 * p->nchunks, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && p->tc_ok)
+        e = cudaMemcpy(p->d_tc_chunks, p->tc_chunks.data(), sizeof(TcChunk) * p->tc_chunks.size(), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_bias, 0, sizeof(float) * p->Dpad);
     if (e != cudaSuccess) {
@@ -111,6 +122,41 @@ gdws_status_t ensure_device(gdws_plan_s *p)
 }
 
 static int round_up(int a, int b) { return (a + b - 1) / b * b; }
+
+// Chunk list of the tensor-core GDW path.  The input channels are taken in windows of 16 (what one tensor-core
+// instruction contracts over); a window's intermediate channels (Property 2: contiguous, in channel order) form
+// one chunk, or several of equal size when there are more than the path handles at once.
+static void build_tc_chunks(gdws_plan_s *p)
+{
+    p->tc_ok = false;
+    if (p->stride != 1 || p->k > 5 || p->C % 8 || p->D % 8 || p->Dpad > 1024) return;
+    p->tc_nparts = (p->Dpad + 255) / 256;
+    p->tc_dloc = round_up((p->Dpad + p->tc_nparts - 1) / p->tc_nparts, 16);
+    const int nmax = p->tc_dloc > 128 ? 96 : 128;
+    p->tc_rec_hw = round_up(1 + p->k * p->k, 8);
+    int slab = 0;
+    for (int c0 = 0; c0 < p->C; c0 += 16) {
+        const int c1 = std::min(p->C, c0 + 16);
+        const int i0 = p->off[c0], n = p->off[c1] - i0;
+        if (n == 0) continue;
+        const int pieces = (n + nmax - 1) / nmax;
+        const int size = round_up((n + pieces - 1) / pieces, 16);
+        for (int done = 0, piece = 0; done < n; done += size, ++piece) {
+            TcChunk ch = {};
+            ch.cbase = c0;
+            ch.i0 = i0 + done;
+            ch.n = std::min(size, n - done);
+            ch.npad = round_up(ch.n, 16);
+            ch.slab0 = slab;
+            ch.flags = (done == 0 ? 1 : 0) | (done + size >= n ? 2 : 0);
+            slab += ch.npad / 16;
+            p->tc_maxslabs = std::max(p->tc_maxslabs, ch.npad / 16);
+            p->tc_chunks.push_back(ch);
+        }
+    }
+    p->tc_nslabs = slab;
+    p->tc_ok = !p->tc_chunks.empty();
+}
 
 // Shared-memory layout of the fused bf16 kernel: 2 * t.spg intermediate-tile stages, a ring of `nsb`
 // pointwise-weight units (a unit = one K chunk x up to 256 output channels, at most 32 KB) and
@@ -318,6 +364,12 @@ gdws_status_t gdws_plan(int C, int D, int k, int stride, int pad, const int32_t 
             }
         }
     }
+    try {
+        build_tc_chunks(p);
+    } catch (...) {
+        delete p;
+        return fail(GDWS_ERR_ALLOC, "gdws_plan: out of host memory");
+    }
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
         gdws_status_t st = ensure_device(p);
@@ -352,7 +404,7 @@ gdws_status_t gdws_plan_set_option(gdws_plan_t *p, int key, int value)
         if (value != 0 && value != 1) return fail(GDWS_ERR_INVALID_ARG, "a_layout must be 0 or 1");
         p->opt_a_layout = value; return GDWS_OK;
     case GDWS_OPT_DW_MATH:
-        if (value != 0 && value != 1) return fail(GDWS_ERR_INVALID_ARG, "dw_math must be 0 or 1");
+        if (value < 0 || value > 2) return fail(GDWS_ERR_INVALID_ARG, "dw_math must be 0, 1 or 2");
         p->opt_dw_math = value; return GDWS_OK;
     default:
         return fail(GDWS_ERR_INVALID_ARG, "unknown option %d", key);

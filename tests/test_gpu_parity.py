@@ -92,13 +92,15 @@ BF16_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("path,a_layout", [(gdws.PATH_UNFUSED, 0), (gdws.PATH_FUSED, 0), (gdws.PATH_FUSED, 1)])
+# dw_math: 0 = GDW stage on the tensor cores where that kernel covers the layer, 1 = on the ALUs
+@pytest.mark.parametrize("path,a_layout,dw_math", [(gdws.PATH_UNFUSED, 0, 0), (gdws.PATH_FUSED, 0, 1), (gdws.PATH_FUSED, 1, 1),
+                                                   (gdws.PATH_FUSED, 0, 0)])
 @pytest.mark.parametrize("shape", BF16_SHAPES)
-def test_bf16_forward_matches_reference(shape, path, a_layout):
+def test_bf16_forward_matches_reference(shape, path, a_layout, dw_math):
     N, C, D, H, W, k, s, p, gd = shape
     spec = small_spec("t", N, C, D, H, W, k, s, p, gd, "bf16", "NHWC", relu=(C == 24), seed=sum(shape[:8]))
     data = gi.make_layer(spec)
-    y = run_gpu(data, path=path, a_layout=a_layout)
+    y = run_gpu(data, path=path, a_layout=a_layout, dw_math=dw_math)
     ref, _ = run_oracle(data)
     err = rel_err(y, ref)
     assert err <= TOL["bf16"], err
@@ -112,7 +114,51 @@ def test_bf16_fused_generic_depthwise_path_with_forced_tiles(tile):
     spec = small_spec("t", 3, 16, 24, 13, 19, 3, 1, 1, ("uniform", 1, 9), seed=33)
     data = gi.make_layer(spec)
     ref, _ = run_oracle(data)
-    assert rel_err(run_gpu(data, path=gdws.PATH_FUSED, tile=tile), ref) <= 1e-2
+    assert rel_err(run_gpu(data, path=gdws.PATH_FUSED, tile=tile, dw_math=1), ref) <= 1e-2
+
+
+# Shapes for the kernel that runs the GDW stage on the tensor cores: every tile family (one image with halo rows,
+# several images per tile, maps at most 4 wide), ragged tails, windows of 8 and 16 input channels, chunks that a
+# window is cut into (many intermediate channels), D beyond 256 (two blocks per tile), k = 1, 2, 3, 5.
+TC_SHAPES = [
+    (2, 16, 16, 16, 8, 3, 1, 1, ("uniform", 1, 9)),
+    (3, 32, 64, 8, 8, 3, 1, 1, ("uniform", 1, 9)),
+    (5, 24, 40, 9, 11, 3, 1, 1, ("uniform", 0, 9)),
+    (9, 16, 64, 4, 4, 3, 1, 1, ("uniform", 1, 9)),
+    (3, 48, 272, 14, 14, 3, 1, 1, ("heavy",)),
+    (1, 32, 512, 28, 28, 3, 1, 1, ("uniform", 7, 9)),
+    (2, 8, 16, 14, 14, 5, 1, 2, ("uniform", 1, 25)),
+    (1, 16, 8, 12, 10, 2, 1, 0, ("uniform", 1, 4)),
+    (2, 40, 24, 7, 7, 1, 1, 0, ("uniform", 1, 1)),
+    (1, 64, 64, 40, 33, 3, 1, 1, ("heavy",)),
+    (4, 16, 128, 3, 3, 3, 1, 1, ("uniform", 1, 9)),
+    (2, 16, 32, 6, 20, 3, 1, 0, ("uniform", 1, 9)),
+    (1, 16, 16, 9, 9, 3, 1, 1, ("const", 12)),              # g_c > k*k is legal (Lemma 1 caps the rank, not the count)
+]
+
+
+@pytest.mark.parametrize("shape", TC_SHAPES)
+def test_bf16_tensor_core_gdw_matches_reference(shape):
+    N, C, D, H, W, k, s, p, gd = shape
+    spec = small_spec("t", N, C, D, H, W, k, s, p, gd, "bf16", "NHWC", relu=(C == 24), seed=7 + sum(shape[:8]))
+    data = gi.make_layer(spec)
+    y = run_gpu(data, path=gdws.PATH_FUSED, dw_math=2)
+    ref, _ = run_oracle(data)
+    err = rel_err(y, ref)
+    assert err <= 1e-2, err
+
+
+def test_tensor_core_gdw_agrees_with_alu_gdw_and_refuses_stride_2():
+    spec = small_spec("t", 6, 32, 48, 16, 16, seed=77)
+    data = gi.make_layer(spec)
+    a = run_gpu(data, path=gdws.PATH_FUSED, dw_math=2)
+    b = run_gpu(data, path=gdws.PATH_FUSED, dw_math=1)
+    # both round z to bf16 once and accumulate in fp32; only the summation order differs
+    assert rel_err(a, b) <= 4e-3
+    data2 = gi.make_layer(small_spec("t", 2, 16, 16, 8, 8, 3, 2, 1, seed=78))
+    with pytest.raises(gdws.GdwsError) as e:
+        run_gpu(data2, path=gdws.PATH_FUSED, dw_math=2)
+    assert e.value.status == gdws.ERR_UNSUPPORTED
 
 
 def test_bf16_depthwise_and_pointwise_stages():
