@@ -87,7 +87,7 @@ __device__ __forceinline__ uint64_t make_sdesc_plain(uint32_t saddr, uint32_t lb
 
 __device__ __forceinline__ void tc_warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
 {
-    if ((threadIdx.x & 31) == 0) mbar_wait_relaxed<500>(bar, parity, abort_flag, status, code);
+    if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, abort_flag, status, code);
     __syncwarp();
 }
 __device__ __forceinline__ void tc_warp_arrive(uint32_t bar)
