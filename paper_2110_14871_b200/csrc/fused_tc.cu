@@ -38,7 +38,7 @@ static_assert(sizeof(TcChunk) == 32, "chunk table entries are copied as two 16-b
 
 constexpr int kTcThreads = 512;
 constexpr int kTcNU = 4;              // chunks in flight per ring (barriers per ring)
-constexpr int kTcMaxNB = 4;           // B operand buffers of the GDW stage
+constexpr int kTcMaxNB = 4;           // B operand buffers of the GDW stage (one chunk each: k*k planes)
 constexpr int kTcMaxNX = 4;           // input box slots
 constexpr int kTcMaxTaps = 25;
 constexpr int kTcZCol = 256;          // TMEM columns 256..511: two GDW accumulators of up to 128 columns
@@ -59,7 +59,7 @@ struct alignas(64) TcParams {
     int nloads, xbox_bytes;
     int load_dw[kTcMaxTaps], load_dh[kTcMaxTaps];
     uint32_t load_off[kTcMaxTaps];
-    uint32_t tap_off[kTcMaxTaps];
+    uint32_t tap_row_step, tap_col_step;   // the A operand of tap (u, v) starts u * row_step + v * col_step bytes into the box
     uint32_t a_lbo, a_sbo;       // GDW A operand: bytes between the two 8-channel planes, between 8-pixel groups
     int nb, nx, nz, nw, nacc;
     uint32_t bbuf_bytes, bplane, b_lbo, xslot_bytes, wslab_bytes;
@@ -106,8 +106,8 @@ template <int K>
 __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_constant__ TcParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    // xfull[4] xfree[4] | bfull[4] bfree[4] | zfull[2] zfree[2] | zsfull[4] pwdone[4] wfull[4] | accfull[2] accfree[2]
-    __shared__ __align__(8) uint64_t bars[2 * kTcMaxNX + 2 * kTcMaxNB + 4 + 3 * kTcNU + 4];
+    // xfull[4] xfree[4] | bfull[4] bfree[4] | zfull[2] | zsfull[4] pwdone[4] wfull[4] | accfull[2] accfree[2]
+    __shared__ __align__(8) uint64_t bars[2 * kTcMaxNX + 2 * kTcMaxNB + 2 + 3 * kTcNU + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -116,8 +116,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const uint32_t o_s = base_s, b_s = base_s + P.off_b, z_s = base_s + P.off_z, w_s = base_s + P.off_w, x_s = base_s + P.off_x;
     const uint32_t bar_xfull = smem_u32(&bars[0]), bar_xfree = bar_xfull + 8 * kTcMaxNX;
     const uint32_t bar_bfull = bar_xfree + 8 * kTcMaxNX, bar_bfree = bar_bfull + 8 * kTcMaxNB;
-    const uint32_t bar_zfull = bar_bfree + 8 * kTcMaxNB, bar_zfree = bar_zfull + 16;
-    const uint32_t bar_zsfull = bar_zfree + 16, bar_pwdone = bar_zsfull + 8 * kTcNU, bar_wfull = bar_pwdone + 8 * kTcNU;
+    const uint32_t bar_zfull = bar_bfree + 8 * kTcMaxNB;
+    const uint32_t bar_zsfull = bar_zfull + 16, bar_pwdone = bar_zsfull + 8 * kTcNU, bar_wfull = bar_pwdone + 8 * kTcNU;
     const uint32_t bar_accfull = bar_wfull + 8 * kTcNU, bar_accfree = bar_accfull + 16;
     TcChunk *tab = reinterpret_cast<TcChunk *>(base + P.off_tab);
     float *bias_sm = reinterpret_cast<float *>(tab + P.nchunks);
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         for (int i = 0; i < kTcMaxNX; ++i) { mbar_init(bar_xfull + 8 * i, 1); mbar_init(bar_xfree + 8 * i, 1); }
         for (int i = 0; i < kTcMaxNB; ++i) { mbar_init(bar_bfull + 8 * i, 4); mbar_init(bar_bfree + 8 * i, 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_zfull + 8 * i, 1); mbar_init(bar_zfree + 8 * i, 4);
+            mbar_init(bar_zfull + 8 * i, 1);
             mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4);
         }
         for (int i = 0; i < kTcNU; ++i) {
@@ -159,63 +159,75 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const int tiles_hw = P.tiles_h * P.tiles_w;
 
     if (warp == 0) {
-        if (lane == 0) {
-            // ---------------- MMA issue ----------------
-            const uint32_t idesc_pw = make_idesc(P.Dloc, false);
-            uint32_t xslot = 0, xpar = 0, bslot = 0, bpar = 0, zhead = 0, whead = 0;
-            int q = 0;                  // chunk index of unit u within its work item
-            int qp = 0, itp = 0;        // the same for unit u - 1, and its work item
-            for (int u = 0; u <= total; ++u) {
-                if (u < total) {
-                    const TcChunk ch = tab[q];
-                    if (ch.flags & 1) mbar_wait(bar_xfull + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitOperand);
-                    if (u >= 2) mbar_wait(bar_zfree + 8 * (u & 1), ((u >> 1) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
-                    tc_fence_after();
-                    const uint32_t idesc = make_idesc(ch.npad, false);
+        // ---------------- MMA issue ----------------
+        // The whole warp walks the loop and waits; one elected lane issues.  This lane's instruction stream bounds
+        // the pipeline (a chunk is a few hundred tensor-core cycles), so descriptors are advanced as 32-bit words.
+        // Unit u: the k*k GDW products of chunk u, then the PW products of chunk u-1, whose z the converter
+        // rounds meanwhile.  The GDW accumulator u&1 is free again once the converter has announced the slabs of
+        // chunk u-2 (it reads TMEM before that), which this warp has waited for before the PW products of u-2.
+        const uint32_t idesc_pw = make_idesc(P.Dloc, false);
+        const uint32_t a_hi = ((P.a_sbo >> 4) & 0x3FFFu) | (1u << 14);
+        const uint32_t p_hi = (128u >> 4) | (1u << 14);               // 8-row groups 128 bytes apart: every other operand
+        const uint32_t a_lo0 = ((x_s & 0x3FFFFu) >> 4) | (((P.a_lbo >> 4) & 0x3FFFu) << 16);
+        const uint32_t b_lo0 = ((b_s & 0x3FFFFu) >> 4) | (((P.b_lbo >> 4) & 0x3FFFu) << 16);
+        const uint32_t z_lo0 = ((z_s & 0x3FFFFu) >> 4) | ((2048u >> 4) << 16);
+        const uint32_t w_lo0 = ((w_s & 0x3FFFFu) >> 4) | ((((uint32_t)P.Dloc * 16u) >> 4) << 16);
+        const uint32_t xstep = P.xslot_bytes >> 4, bstep = P.bbuf_bytes >> 4, pstep = P.bplane >> 4;
+        const uint32_t rstep = P.tap_row_step >> 4, cstep = P.tap_col_step >> 4, wstep = P.wslab_bytes >> 4;
+        uint32_t xslot = 0, xpar = 0, bslot = 0, bpar = 0, zhead = 0, whead = 0;
+        int q = 0;                  // chunk index of unit u within its work item
+        int qp = 0, itp = 0;        // the same for unit u - 1, and its work item
+        for (int u = 0; u <= total; ++u) {
+            if (u < total) {
+                const int npad = tab[q].npad, flags = tab[q].flags;
+                if (flags & 1) mbar_wait(bar_xfull + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitOperand);
+                mbar_wait(bar_bfull + 8 * bslot, bpar, &abort_flag, P.status, kStatusWaitOperand);
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint32_t idesc = make_idesc(npad, false);
                     const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
-                    const uint32_t abase = x_s + xslot * P.xslot_bytes;
-#pragma unroll 1
-                    for (int ur = 0; ur < K; ++ur) {
-                        mbar_wait(bar_bfull + 8 * bslot, bpar, &abort_flag, P.status, kStatusWaitOperand);
-                        tc_fence_after();
-                        const uint32_t bb = b_s + bslot * P.bbuf_bytes;
+                    const uint32_t a_lo = a_lo0 + xslot * xstep, b_lo = b_lo0 + bslot * bstep;
+#pragma unroll
+                    for (int ur = 0; ur < K; ++ur)
 #pragma unroll
                         for (int v = 0; v < K; ++v)
-                            umma_bf16(d_z, make_sdesc_plain(abase + P.tap_off[ur * K + v], P.a_lbo, P.a_sbo),
-                                      make_sdesc_plain(bb + (uint32_t)v * P.bplane, P.b_lbo, 128u), idesc, (ur | v) != 0);
-                        umma_commit(bar_bfree + 8 * bslot);
-                        if (++bslot == (uint32_t)P.nb) { bslot = 0; bpar ^= 1; }
-                    }
+                            umma_bf16_words(d_z, a_lo + (uint32_t)ur * rstep + (uint32_t)v * cstep, a_hi,
+                                            b_lo + (uint32_t)(ur * K + v) * pstep, p_hi, idesc, (ur | v) != 0);
+                    umma_commit(bar_bfree + 8 * bslot);
                     umma_commit(bar_zfull + 8 * (u & 1));
-                    if (ch.flags & 2) {
-                        umma_commit(bar_xfree + 8 * xslot);
-                        if (++xslot == (uint32_t)P.nx) { xslot = 0; xpar ^= 1; }
-                    }
-                    if (++q == P.nchunks) q = 0;
+                    if (flags & 2) umma_commit(bar_xfree + 8 * xslot);
                 }
-                if (u > 0) {
-                    const int v = u - 1;
-                    const int buf = itp % P.nacc;
-                    if (qp == 0 && itp >= P.nacc)
-                        mbar_wait(bar_accfree + 8 * buf, ((itp / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
-                    const uint32_t up = (uint32_t)(v & (kTcNU - 1)), par = (uint32_t)(v / kTcNU) & 1u;
-                    mbar_wait(bar_wfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
-                    mbar_wait(bar_zsfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
-                    tc_fence_after();
-                    const int ns = tab[qp].npad >> 4;
+                __syncwarp();
+                if (++bslot == (uint32_t)P.nb) { bslot = 0; bpar ^= 1; }
+                if (flags & 2) { if (++xslot == (uint32_t)P.nx) { xslot = 0; xpar ^= 1; } }
+                if (++q == P.nchunks) q = 0;
+            }
+            if (u > 0) {
+                const int v = u - 1;
+                const int buf = itp % P.nacc;
+                if (qp == 0 && itp >= P.nacc)
+                    mbar_wait(bar_accfree + 8 * buf, ((itp / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                const uint32_t up = (uint32_t)(v & (kTcNU - 1)), par = (uint32_t)(v / kTcNU) & 1u;
+                mbar_wait(bar_wfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
+                mbar_wait(bar_zsfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
+                tc_fence_after();
+                const int ns = tab[qp].npad >> 4;
+                if (elect_one()) {
                     const uint32_t d_y = tmem + (uint32_t)(buf * 128);
+                    uint32_t zh = zhead, wh = whead;
 #pragma unroll 1
                     for (int s = 0; s < ns; ++s) {
-                        umma_bf16(d_y, make_sdesc_plain(z_s + zhead * kTcSlab, 2048u, 128u),
-                                  make_sdesc_plain(w_s + whead * P.wslab_bytes, (uint32_t)P.Dloc * 16u, 128u), idesc_pw,
-                                  (qp | s) != 0);
-                        if (++zhead == (uint32_t)P.nz) zhead = 0;
-                        if (++whead == (uint32_t)P.nw) whead = 0;
+                        umma_bf16_words(d_y, z_lo0 + zh * (kTcSlab >> 4), p_hi, w_lo0 + wh * wstep, p_hi, idesc_pw, (qp | s) != 0);
+                        if (++zh == (uint32_t)P.nz) zh = 0;
+                        if (++wh == (uint32_t)P.nw) wh = 0;
                     }
                     umma_commit(bar_pwdone + 8 * up);
                     if (qp == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
-                    if (++qp == P.nchunks) { qp = 0; ++itp; }
                 }
+                __syncwarp();
+                zhead = (zhead + (uint32_t)ns) % (uint32_t)P.nz;
+                whead = (whead + (uint32_t)ns) % (uint32_t)P.nw;
+                if (++qp == P.nchunks) { qp = 0; ++itp; }
             }
         }
     } else if (warp == 1) {
@@ -293,11 +305,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             tc_fence_after();
             const uint32_t taddr = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(kTcZCol + 128 * (v & 1));
             int slab = ring.head;
-#pragma unroll 1
-            for (int g = 0; g < ns; ++g) {
-                uint32_t acc[16];
-                tmem_ld16(taddr + (uint32_t)(g * 16), acc);
-                tmem_ld_wait();
+            auto put = [&](const uint32_t (&acc)[16]) {
                 uint4 lo, hi;
                 lo.x = pack_bf16x2(__uint_as_float(acc[0]), __uint_as_float(acc[1]));
                 lo.y = pack_bf16x2(__uint_as_float(acc[2]), __uint_as_float(acc[3]));
@@ -308,14 +316,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 hi.z = pack_bf16x2(__uint_as_float(acc[12]), __uint_as_float(acc[13]));
                 hi.w = pack_bf16x2(__uint_as_float(acc[14]), __uint_as_float(acc[15]));
                 const uint32_t addr = z_s + (uint32_t)slab * kTcSlab + r * 16u;
-                sts128(addr, lo);              // channels 16g .. 16g+7 of this pixel: first core-matrix plane
-                sts128(addr + 2048u, hi);      // channels 16g+8 .. 16g+15: second plane
+                sts128(addr, lo);              // channels 0 .. 7 of the slab for this pixel: first core-matrix plane
+                sts128(addr + 2048u, hi);      // channels 8 .. 15: second plane
                 if (++slab == P.nz) slab = 0;
+            };
+#pragma unroll 1
+            for (int g = 0; g < ns; g += 2) {
+                uint32_t acc0[16], acc1[16];
+                tmem_ld16(taddr + (uint32_t)(g * 16), acc0);
+                if (g + 1 < ns) tmem_ld16(taddr + (uint32_t)(g * 16 + 16), acc1);
+                tmem_ld_wait();
+                put(acc0);
+                if (g + 1 < ns) put(acc1);
             }
             fence_proxy_async();
             tc_fence_before();
             tc_warp_arrive(bar_zsfull + 8 * (v & (kTcNU - 1)));
-            tc_warp_arrive(bar_zfree + 8 * (v & 1));
             ring.head = (ring.head + ns) % P.nz;
             ring.free_slabs -= ns;
             if (++q == P.nchunks) q = 0;
@@ -417,7 +433,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         };
         if (total > 0) load_rec(tab[0], nxt);
         uint32_t bslot = 0;
-        int ub = 0, q = 0;
+        int q = 0;
         for (int v = 0; v < total; ++v) {
 #pragma unroll
             for (int j = 0; j < RW; ++j) rec[j] = nxt[j];
@@ -426,28 +442,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             const uint32_t cw = rec[0] & 0xFFFFu;
             const bool valid = cw != 0xFFFFu;
             const uint32_t off = (cw >> 3) * P.b_lbo + rowoff + (cw & 7u) * 2u;
+            if (v >= P.nb) tc_warp_wait(bar_bfree + 8 * bslot, (uint32_t)((v / P.nb) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+            const uint32_t bb = b_s + bslot * P.bbuf_bytes;
+            const uint32_t old = bold[bslot * 128 + t];
+            if (old != 0xFFFFu) {
 #pragma unroll
-            for (int ur = 0; ur < K; ++ur) {
-                if (ub >= P.nb) tc_warp_wait(bar_bfree + 8 * bslot, (uint32_t)((ub / P.nb) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
-                const uint32_t bb = b_s + bslot * P.bbuf_bytes;
-                const uint32_t old = bold[bslot * 128 + t];
-                if (old != 0xFFFFu) {
-#pragma unroll
-                    for (int vv = 0; vv < K; ++vv) sts16(bb + (uint32_t)vv * P.bplane + old, (uint16_t)0);
-                }
-                if (valid) {
-#pragma unroll
-                    for (int vv = 0; vv < K; ++vv) {
-                        const int h = 1 + ur * K + vv;          // 16-bit word of the record holding tap (ur, vv)
-                        sts16(bb + (uint32_t)vv * P.bplane + off, (uint16_t)(rec[h >> 1] >> (16 * (h & 1))));
-                    }
-                }
-                bold[bslot * 128 + t] = (uint16_t)(valid ? off : 0xFFFFu);
-                fence_proxy_async();
-                tc_warp_arrive(bar_bfull + 8 * bslot);
-                ++ub;
-                if (++bslot == (uint32_t)P.nb) bslot = 0;
+                for (int j = 0; j < K * K; ++j) sts16(bb + (uint32_t)j * P.bplane + old, (uint16_t)0);
             }
+            if (valid) {
+#pragma unroll
+                for (int j = 0; j < K * K; ++j)     // 16-bit word 1 + j of the record holds tap j
+                    sts16(bb + (uint32_t)j * P.bplane + off, (uint16_t)(rec[(1 + j) >> 1] >> (16 * ((1 + j) & 1))));
+            }
+            bold[bslot * 128 + t] = (uint16_t)(valid ? off : 0xFFFFu);
+            fence_proxy_async();
+            tc_warp_arrive(bar_bfull + 8 * bslot);
+            if (++bslot == (uint32_t)P.nb) bslot = 0;
         }
     }
     tc_fence_before();
@@ -570,8 +580,8 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     TcParams P;
     memset(&P, 0, sizeof(P));
     const int Dloc = p->tc_dloc, m = p->tc_maxslabs;
-    const uint32_t nmax = Dloc > 128 ? 96u : 128u;
-    P.bplane = nmax * 32u; P.b_lbo = nmax * 16u; P.bbuf_bytes = (uint32_t)k * P.bplane;
+    const uint32_t nmax = (uint32_t)tc_nmax(k, Dloc);
+    P.bplane = nmax * 32u; P.b_lbo = nmax * 16u; P.bbuf_bytes = (uint32_t)(k * k) * P.bplane;
     P.wslab_bytes = (uint32_t)Dloc * 32u;
     P.xslot_bytes = (uint32_t)((g.xbox + 127) / 128 * 128);
     // Shared memory: output staging (optional) | B operand buffers | z slabs | weight slabs | input boxes | tables
@@ -581,7 +591,7 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     int b_ost = 0, b_nx = 0, b_nb = 0, b_nz = 0, b_nw = 0;
     for (int ost = can_stage ? 1 : 0; ost >= 0; --ost)
         for (int nx = 3; nx >= 2; --nx)
-            for (int nb = 4; nb >= 2; --nb)
+            for (int nb = 3; nb >= 2; --nb)
                 for (int nz = 2 * m; nz >= m; --nz) {
                     const size_t fixed = 1024 + (ost ? 16384 : 0) + (size_t)nb * P.bbuf_bytes + (size_t)nz * kTcSlab +
                                          (size_t)nx * P.xslot_bytes + tables;
@@ -631,19 +641,19 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     if (g.layout == 1) {
         P.nloads = 1; P.load_dw[0] = 0; P.load_dh[0] = 0; P.load_off[0] = 0;
         P.a_lbo = (uint32_t)((g.PH + k - 1) * g.IW) * px; P.a_sbo = (uint32_t)g.IW * px;
-        for (int u = 0; u < k; ++u) for (int v = 0; v < k; ++v) P.tap_off[u * k + v] = (uint32_t)(u * g.IW + v) * px;
+        P.tap_row_step = (uint32_t)g.IW * px; P.tap_col_step = px;
     } else if (g.layout == 2) {
         const uint32_t copy = 2u * 16u * (uint32_t)g.IW * px;
         P.nloads = k;
         for (int u = 0; u < k; ++u) { P.load_dw[u] = 0; P.load_dh[u] = u; P.load_off[u] = (uint32_t)u * copy; }
         P.a_lbo = 16u * (uint32_t)g.IW * px; P.a_sbo = (uint32_t)g.IW * px;
-        for (int u = 0; u < k; ++u) for (int v = 0; v < k; ++v) P.tap_off[u * k + v] = (uint32_t)u * copy + (uint32_t)v * px;
+        P.tap_row_step = copy; P.tap_col_step = px;
     } else {
         P.nloads = k * k;
         for (int u = 0; u < k; ++u) for (int v = 0; v < k; ++v) {
             P.load_dw[u * k + v] = v; P.load_dh[u * k + v] = u; P.load_off[u * k + v] = (uint32_t)(u * k + v) * 4096u;
-            P.tap_off[u * k + v] = (uint32_t)(u * k + v) * 4096u;
         }
+        P.tap_row_step = (uint32_t)k * 4096u; P.tap_col_step = 4096u;
         P.a_lbo = 2048u; P.a_sbo = 128u;
     }
     P.xbox_bytes = g.xbox;

@@ -36,6 +36,10 @@ struct TcChunk {
     int32_t reserved0, reserved1;
 };
 
+// Most intermediate channels one chunk of the tensor-core GDW path holds: its k*k B operands (32 bytes per
+// channel each) must fit shared memory twice, and two GDW accumulators must fit beside the PW accumulator in TMEM.
+inline int tc_nmax(int k, int dloc) { return k >= 4 ? 32 : (dloc > 128 ? 96 : 128); }
+
 struct Tile {
     int TN = 0, PH = 0, PW = 0;      // images x rows x columns of output pixels per 128-row tile
     int tiles_n = 0, tiles_h = 0, tiles_w = 0;

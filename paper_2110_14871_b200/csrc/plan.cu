@@ -132,7 +132,7 @@ static void build_tc_chunks(gdws_plan_s *p)
     if (p->stride != 1 || p->k > 5 || p->C % 8 || p->D % 8 || p->Dpad > 1024) return;
     p->tc_nparts = (p->Dpad + 255) / 256;
     p->tc_dloc = round_up((p->Dpad + p->tc_nparts - 1) / p->tc_nparts, 16);
-    const int nmax = p->tc_dloc > 128 ? 96 : 128;
+    const int nmax = tc_nmax(p->k, p->tc_dloc);
     p->tc_rec_hw = round_up(1 + p->k * p->k, 8);
     int slab = 0;
     for (int c0 = 0; c0 < p->C; c0 += 16) {
