@@ -38,6 +38,7 @@ static_assert(sizeof(TcChunk) == 32, "chunk table entries are copied as two 16-b
 
 constexpr int kTcThreads = 512;
 constexpr int kTcNU = 4;              // chunks in flight per ring (barriers per ring)
+static_assert(kTcNU == 4, "unit parity is taken from bit 2 of the unit index");
 constexpr int kTcMaxNB = 4;           // B operand buffers of the GDW stage (one chunk each: k*k planes)
 constexpr int kTcMaxNX = 4;           // input box slots
 constexpr int kTcMaxTaps = 25;
@@ -85,9 +86,24 @@ __device__ __forceinline__ uint64_t make_sdesc_plain(uint32_t saddr, uint32_t lb
     return d;
 }
 
+// Bounded wait of every role but the MMA warp: each poll lets the hardware suspend the thread until the phase
+// completes (or 16 us pass), so that waiting warps issue next to nothing.  The MMA warp is a single
+// instruction stream whose shared-memory latency sets the pace of the whole pipeline; polls of a dozen other
+// warps in front of it in the shared-memory queue slowed it down several times.
+__device__ __forceinline__ void tc_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+{
+    if (mbar_try_wait(bar, parity)) return;
+    if (*abort_flag) return;
+    for (uint32_t it = 0; it < (1u << 16); ++it) {     // bounded: about a second
+        if (mbar_try_wait_suspend(bar, parity, 16384u)) return;
+        if (*abort_flag) return;
+    }
+    *abort_flag = 1;
+    atomicOr(status, code);
+}
 __device__ __forceinline__ void tc_warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
 {
-    if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, abort_flag, status, code);
+    if ((threadIdx.x & 31) == 0) tc_wait(bar, parity, abort_flag, status, code);
     __syncwarp();
 }
 __device__ __forceinline__ void tc_warp_arrive(uint32_t bar)
@@ -177,6 +193,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         uint32_t xslot = 0, xpar = 0, bslot = 0, bpar = 0, zhead = 0, whead = 0;
         int q = 0;                  // chunk index of unit u within its work item
         int qp = 0, itp = 0;        // the same for unit u - 1, and its work item
+        uint32_t buf = 0, accpar = 1;   // accumulator of unit u - 1's work item, parity of its "free" phase to wait for
         for (int u = 0; u <= total; ++u) {
             if (u < total) {
                 const int npad = tab[q].npad, flags = tab[q].flags;
@@ -204,10 +221,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             }
             if (u > 0) {
                 const int v = u - 1;
-                const int buf = itp % P.nacc;
-                if (qp == 0 && itp >= P.nacc)
-                    mbar_wait(bar_accfree + 8 * buf, ((itp / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
-                const uint32_t up = (uint32_t)(v & (kTcNU - 1)), par = (uint32_t)(v / kTcNU) & 1u;
+                if (qp == 0 && itp >= P.nacc) mbar_wait(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
+                const uint32_t up = (uint32_t)(v & (kTcNU - 1)), par = (uint32_t)(v >> 2) & 1u;
                 mbar_wait(bar_wfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
                 mbar_wait(bar_zsfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
                 tc_fence_after();
@@ -225,9 +240,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     if (qp == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
                 }
                 __syncwarp();
-                zhead = (zhead + (uint32_t)ns) % (uint32_t)P.nz;
-                whead = (whead + (uint32_t)ns) % (uint32_t)P.nw;
-                if (++qp == P.nchunks) { qp = 0; ++itp; }
+                zhead += (uint32_t)ns;
+                if (zhead >= (uint32_t)P.nz) zhead -= (uint32_t)P.nz;
+                whead += (uint32_t)ns;
+                if (whead >= (uint32_t)P.nw) whead -= (uint32_t)P.nw;
+                if (++qp == P.nchunks) {
+                    qp = 0; ++itp;
+                    if (++buf == (uint32_t)P.nacc) { buf = 0; accpar ^= 1; }
+                }
             }
         }
     } else if (warp == 1) {
@@ -246,7 +266,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     const TcChunk ch = tab[q];
                     if (!(ch.flags & 1)) continue;
                     if (box >= P.nx)
-                        mbar_wait_relaxed<500>(bar_xfree + 8 * xslot, (uint32_t)((box / P.nx) - 1) & 1u, &abort_flag, P.status,
+                        tc_wait(bar_xfree + 8 * xslot, (uint32_t)((box / P.nx) - 1) & 1u, &abort_flag, P.status,
                                                kStatusWaitStage);
                     mbar_expect_tx(bar_xfull + 8 * xslot, (uint32_t)P.xbox_bytes);
                     const uint32_t dst = x_s + xslot * P.xslot_bytes;
@@ -269,7 +289,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 const int ns = ch.npad >> 4;
                 while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
                     const int o = ring.oldest;
-                    mbar_wait_relaxed<500>(bar_pwdone + 8 * (o & (kTcNU - 1)), (uint32_t)(o / kTcNU) & 1u, &abort_flag, P.status,
+                    tc_wait(bar_pwdone + 8 * (o & (kTcNU - 1)), (uint32_t)(o / kTcNU) & 1u, &abort_flag, P.status,
                                            kStatusWaitStage);
                     ring.free_slabs += tab[o % P.nchunks].npad >> 4;
                     ++ring.oldest;
