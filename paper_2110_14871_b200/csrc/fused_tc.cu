@@ -36,7 +36,10 @@ namespace gdws {
 
 static_assert(sizeof(TcChunk) == 32, "chunk table entries are copied as two 16-byte words");
 
-constexpr int kTcThreads = 512;
+constexpr int kTcConvWarps = 8;        // converter warps 4 .. 11 (two per TMEM lane quarter)
+constexpr int kTcEpiWarp0 = 4 + kTcConvWarps, kTcBuildWarp0 = kTcEpiWarp0 + 4;
+constexpr int kTcThreads = (kTcBuildWarp0 + 4) * 32;
+static_assert(kTcEpiWarp0 % 4 == 0, "a warp reads the TMEM lanes of quarter warp % 4");
 constexpr int kTcNU = 4;              // chunks in flight per ring (barriers per ring)
 static_assert(kTcNU == 4, "unit parity is taken from bit 2 of the unit index");
 constexpr int kTcMaxNB = 4;           // B operand buffers of the GDW stage (one chunk each: k*k planes)
@@ -122,19 +125,24 @@ template <int K>
 __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_constant__ TcParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    // xfull[4] xfree[4] | bfull[4] bfree[4] | zfull[2] | zsfull[4] pwdone[4] wfull[4] | accfull[2] accfree[2]
-    __shared__ __align__(8) uint64_t bars[2 * kTcMaxNX + 2 * kTcMaxNB + 2 + 3 * kTcNU + 4];
+    // dwready[4] | zfull[2] zfree[2] | pwready[4] pwdone[4] | bfree[4] xfree[4] | accfull[2] accfree[2]
+    __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t base_s = smem_u32(base);
     const uint32_t o_s = base_s, b_s = base_s + P.off_b, z_s = base_s + P.off_z, w_s = base_s + P.off_w, x_s = base_s + P.off_x;
-    const uint32_t bar_xfull = smem_u32(&bars[0]), bar_xfree = bar_xfull + 8 * kTcMaxNX;
-    const uint32_t bar_bfull = bar_xfree + 8 * kTcMaxNX, bar_bfree = bar_bfull + 8 * kTcMaxNB;
-    const uint32_t bar_zfull = bar_bfree + 8 * kTcMaxNB;
-    const uint32_t bar_zsfull = bar_zfull + 16, bar_pwdone = bar_zsfull + 8 * kTcNU, bar_wfull = bar_pwdone + 8 * kTcNU;
-    const uint32_t bar_accfull = bar_wfull + 8 * kTcNU, bar_accfree = bar_accfull + 16;
+    // dwready: the B operands (4 builder warps) and the input box (the loader's arrive, with the box's bytes when the
+    // chunk opens a window) of a chunk are in place.  zfull: its GDW products are done.  zfree: the converter has read
+    // them out of TMEM.  pwready: the chunk's z slabs (8 converter warps) and its pointwise weights (the loader's
+    // arrive with their bytes) are in place.  pwdone: its PW products are done.  bfree / xfree: arrived by the
+    // converter once the GDW products that read a B buffer / the last ones that read a box are done.
+    const uint32_t bar_dwready = smem_u32(&bars[0]);
+    const uint32_t bar_zfull = bar_dwready + 32, bar_zfree = bar_zfull + 16;
+    const uint32_t bar_pwready = bar_zfree + 16, bar_pwdone = bar_pwready + 8 * kTcNU;
+    const uint32_t bar_bfree = bar_pwdone + 8 * kTcNU, bar_xfree = bar_bfree + 8 * kTcMaxNB;
+    const uint32_t bar_accfull = bar_xfree + 8 * kTcMaxNX, bar_accfree = bar_accfull + 16;
     TcChunk *tab = reinterpret_cast<TcChunk *>(base + P.off_tab);
     float *bias_sm = reinterpret_cast<float *>(tab + P.nchunks);
     uint16_t *bold = reinterpret_cast<uint16_t *>(bias_sm + P.Dpad_tot);     // [nb][128]: what each builder thread wrote last
@@ -142,15 +150,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
 
     if (tid == 0) {
         abort_flag = 0;
-        for (int i = 0; i < kTcMaxNX; ++i) { mbar_init(bar_xfull + 8 * i, 1); mbar_init(bar_xfree + 8 * i, 1); }
-        for (int i = 0; i < kTcMaxNB; ++i) { mbar_init(bar_bfull + 8 * i, 4); mbar_init(bar_bfree + 8 * i, 1); }
+        for (int i = 0; i < 4; ++i) mbar_init(bar_dwready + 8 * i, 5);
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_zfull + 8 * i, 1);
+            mbar_init(bar_zfull + 8 * i, 1); mbar_init(bar_zfree + 8 * i, kTcConvWarps);
             mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4);
         }
-        for (int i = 0; i < kTcNU; ++i) {
-            mbar_init(bar_zsfull + 8 * i, 4); mbar_init(bar_pwdone + 8 * i, 1); mbar_init(bar_wfull + 8 * i, 1);
-        }
+        for (int i = 0; i < kTcNU; ++i) { mbar_init(bar_pwready + 8 * i, kTcConvWarps + 1); mbar_init(bar_pwdone + 8 * i, 1); }
+        for (int i = 0; i < kTcMaxNB; ++i) mbar_init(bar_bfree + 8 * i, 1);
+        for (int i = 0; i < kTcMaxNX; ++i) mbar_init(bar_xfree + 8 * i, 1);
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512u);
@@ -173,87 +180,91 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const int my_items = ((int)P.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const int total = my_items * P.nchunks;
     const int tiles_hw = P.tiles_h * P.tiles_w;
+    const uint32_t p_hi = (128u >> 4) | (1u << 14);     // descriptor high word: 8-row groups 128 bytes apart, version 1
 
+    // The two issue warps are single instruction streams that pace the pipeline: a satisfied mbarrier wait costs them
+    // some 140 cycles and a tcgen05.commit some 80, against 24 per tcgen05.mma (measured), while the tensor-core work of
+    // a chunk is a few hundred cycles.  Hence one wait and one commit per chunk and warp, the GDW and the PW products
+    // issued by different warps, and descriptors advanced as 32-bit words.
     if (warp == 0) {
-        // ---------------- MMA issue ----------------
-        // The whole warp walks the loop and waits; one elected lane issues.  This lane's instruction stream bounds
-        // the pipeline (a chunk is a few hundred tensor-core cycles), so descriptors are advanced as 32-bit words.
-        // Unit u: the k*k GDW products of chunk u, then the PW products of chunk u-1, whose z the converter
-        // rounds meanwhile.  The GDW accumulator u&1 is free again once the converter has announced the slabs of
-        // chunk u-2 (it reads TMEM before that), which this warp has waited for before the PW products of u-2.
-        const uint32_t idesc_pw = make_idesc(P.Dloc, false);
+        // ---------------- GDW issue: the k*k products of chunk u into accumulator u & 1 ----------------
         const uint32_t a_hi = ((P.a_sbo >> 4) & 0x3FFFu) | (1u << 14);
-        const uint32_t p_hi = (128u >> 4) | (1u << 14);               // 8-row groups 128 bytes apart: every other operand
         const uint32_t a_lo0 = ((x_s & 0x3FFFFu) >> 4) | (((P.a_lbo >> 4) & 0x3FFFu) << 16);
         const uint32_t b_lo0 = ((b_s & 0x3FFFFu) >> 4) | (((P.b_lbo >> 4) & 0x3FFFu) << 16);
+        const uint32_t xstep = P.xslot_bytes >> 4, bstep = P.bbuf_bytes >> 4, pstep = P.bplane >> 4;
+        const uint32_t rstep = P.tap_row_step >> 4, cstep = P.tap_col_step >> 4;
+        uint32_t xslot = 0, bslot = 0;
+        int q = 0;
+        for (int u = 0; u < total; ++u) {
+            const int npad = tab[q].npad, flags = tab[q].flags;
+            mbar_wait(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
+            if (u >= 2) mbar_wait(bar_zfree + 8 * (u & 1), (uint32_t)((u >> 1) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+            tc_fence_after();
+            if (elect_one()) {
+                const uint32_t idesc = make_idesc(npad, false);
+                const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
+                const uint32_t a_lo = a_lo0 + xslot * xstep, b_lo = b_lo0 + bslot * bstep;
+#pragma unroll
+                for (int ur = 0; ur < K; ++ur)
+#pragma unroll
+                    for (int v = 0; v < K; ++v)
+                        umma_bf16_words(d_z, a_lo + (uint32_t)ur * rstep + (uint32_t)v * cstep, a_hi,
+                                        b_lo + (uint32_t)(ur * K + v) * pstep, p_hi, idesc, (ur | v) != 0);
+                umma_commit(bar_zfull + 8 * (u & 1));
+            }
+            __syncwarp();
+            if (++bslot == (uint32_t)P.nb) bslot = 0;
+            if (flags & 2) { if (++xslot == (uint32_t)P.nx) xslot = 0; }
+            if (++q == P.nchunks) q = 0;
+        }
+    } else if (warp == 3) {
+        // ---------------- PW issue: chunk v's slabs times its weights into the work item's accumulator ----------------
+        const uint32_t idesc_pw = make_idesc(P.Dloc, false);
         const uint32_t z_lo0 = ((z_s & 0x3FFFFu) >> 4) | ((2048u >> 4) << 16);
         const uint32_t w_lo0 = ((w_s & 0x3FFFFu) >> 4) | ((((uint32_t)P.Dloc * 16u) >> 4) << 16);
-        const uint32_t xstep = P.xslot_bytes >> 4, bstep = P.bbuf_bytes >> 4, pstep = P.bplane >> 4;
-        const uint32_t rstep = P.tap_row_step >> 4, cstep = P.tap_col_step >> 4, wstep = P.wslab_bytes >> 4;
-        uint32_t xslot = 0, xpar = 0, bslot = 0, bpar = 0, zhead = 0, whead = 0;
-        int q = 0;                  // chunk index of unit u within its work item
-        int qp = 0, itp = 0;        // the same for unit u - 1, and its work item
-        uint32_t buf = 0, accpar = 1;   // accumulator of unit u - 1's work item, parity of its "free" phase to wait for
-        for (int u = 0; u <= total; ++u) {
-            if (u < total) {
-                const int npad = tab[q].npad, flags = tab[q].flags;
-                if (flags & 1) mbar_wait(bar_xfull + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitOperand);
-                mbar_wait(bar_bfull + 8 * bslot, bpar, &abort_flag, P.status, kStatusWaitOperand);
-                tc_fence_after();
-                if (elect_one()) {
-                    const uint32_t idesc = make_idesc(npad, false);
-                    const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
-                    const uint32_t a_lo = a_lo0 + xslot * xstep, b_lo = b_lo0 + bslot * bstep;
+        const uint32_t wstep = P.wslab_bytes >> 4;
+        uint32_t zhead = 0, whead = 0, buf = 0, accpar = 1;
+        int q = 0, it = 0;
+        for (int v = 0; v < total; ++v) {
+            const int ns = tab[q].npad >> 4;
+            if (q == 0 && it >= P.nacc) mbar_wait(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
+            mbar_wait(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
+            tc_fence_after();
+            if (elect_one()) {
+                const uint32_t d_y = tmem + buf * 128u;
+                if (zhead + (uint32_t)ns <= (uint32_t)P.nz && whead + (uint32_t)ns <= (uint32_t)P.nw) {
+                    const uint32_t z_lo = z_lo0 + zhead * (kTcSlab >> 4), w_lo = w_lo0 + whead * wstep;
 #pragma unroll
-                    for (int ur = 0; ur < K; ++ur)
-#pragma unroll
-                        for (int v = 0; v < K; ++v)
-                            umma_bf16_words(d_z, a_lo + (uint32_t)ur * rstep + (uint32_t)v * cstep, a_hi,
-                                            b_lo + (uint32_t)(ur * K + v) * pstep, p_hi, idesc, (ur | v) != 0);
-                    umma_commit(bar_bfree + 8 * bslot);
-                    umma_commit(bar_zfull + 8 * (u & 1));
-                    if (flags & 2) umma_commit(bar_xfree + 8 * xslot);
-                }
-                __syncwarp();
-                if (++bslot == (uint32_t)P.nb) { bslot = 0; bpar ^= 1; }
-                if (flags & 2) { if (++xslot == (uint32_t)P.nx) { xslot = 0; xpar ^= 1; } }
-                if (++q == P.nchunks) q = 0;
-            }
-            if (u > 0) {
-                const int v = u - 1;
-                if (qp == 0 && itp >= P.nacc) mbar_wait(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
-                const uint32_t up = (uint32_t)(v & (kTcNU - 1)), par = (uint32_t)(v >> 2) & 1u;
-                mbar_wait(bar_wfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
-                mbar_wait(bar_zsfull + 8 * up, par, &abort_flag, P.status, kStatusWaitOperand);
-                tc_fence_after();
-                const int ns = tab[qp].npad >> 4;
-                if (elect_one()) {
-                    const uint32_t d_y = tmem + (uint32_t)(buf * 128);
+                    for (int s = 0; s < 8; ++s)      // a chunk has at most 8 slabs (128 intermediate channels)
+                        if (s < ns)
+                            umma_bf16_words(d_y, z_lo + (uint32_t)s * (kTcSlab >> 4), p_hi, w_lo + (uint32_t)s * wstep, p_hi, idesc_pw,
+                                            (q | s) != 0);
+                } else {                              // the chunk wraps around the end of a ring
                     uint32_t zh = zhead, wh = whead;
 #pragma unroll 1
                     for (int s = 0; s < ns; ++s) {
-                        umma_bf16_words(d_y, z_lo0 + zh * (kTcSlab >> 4), p_hi, w_lo0 + wh * wstep, p_hi, idesc_pw, (qp | s) != 0);
+                        umma_bf16_words(d_y, z_lo0 + zh * (kTcSlab >> 4), p_hi, w_lo0 + wh * wstep, p_hi, idesc_pw, (q | s) != 0);
                         if (++zh == (uint32_t)P.nz) zh = 0;
                         if (++wh == (uint32_t)P.nw) wh = 0;
                     }
-                    umma_commit(bar_pwdone + 8 * up);
-                    if (qp == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
                 }
-                __syncwarp();
-                zhead += (uint32_t)ns;
-                if (zhead >= (uint32_t)P.nz) zhead -= (uint32_t)P.nz;
-                whead += (uint32_t)ns;
-                if (whead >= (uint32_t)P.nw) whead -= (uint32_t)P.nw;
-                if (++qp == P.nchunks) {
-                    qp = 0; ++itp;
-                    if (++buf == (uint32_t)P.nacc) { buf = 0; accpar ^= 1; }
-                }
+                umma_commit(bar_pwdone + 8 * (v & 3));
+                if (q == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
+            }
+            __syncwarp();
+            zhead += (uint32_t)ns;
+            if (zhead >= (uint32_t)P.nz) zhead -= (uint32_t)P.nz;
+            whead += (uint32_t)ns;
+            if (whead >= (uint32_t)P.nw) whead -= (uint32_t)P.nw;
+            if (++q == P.nchunks) {
+                q = 0; ++it;
+                if (++buf == (uint32_t)P.nacc) { buf = 0; accpar ^= 1; }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------- input loader ----------------
-            int box = 0;
+            int box = 0, u = 0;
             uint32_t xslot = 0;
             for (int it = 0; it < my_items; ++it) {
                 const int item = (int)blockIdx.x + it * (int)gridDim.x;
@@ -262,17 +273,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 tile -= bn * tiles_hw;
                 const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
                 const int n0 = bn * P.TN, hi0 = bh * P.PH - P.pad, wi0 = bw * P.PW - P.pad;
-                for (int q = 0; q < P.nchunks; ++q) {
-                    const TcChunk ch = tab[q];
-                    if (!(ch.flags & 1)) continue;
+                for (int q = 0; q < P.nchunks; ++q, ++u) {
+                    const int cbase = tab[q].cbase, flags = tab[q].flags;
+                    const uint32_t bar = bar_dwready + 8 * (u & 3);
+                    // this barrier's last phase (chunk u - 4) must be complete before anything counts towards chunk u
+                    if (u >= 4) tc_wait(bar, (uint32_t)((u >> 2) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                    if (!(flags & 1)) { mbar_arrive(bar); continue; }
                     if (box >= P.nx)
-                        tc_wait(bar_xfree + 8 * xslot, (uint32_t)((box / P.nx) - 1) & 1u, &abort_flag, P.status,
-                                               kStatusWaitStage);
-                    mbar_expect_tx(bar_xfull + 8 * xslot, (uint32_t)P.xbox_bytes);
+                        tc_wait(bar_xfree + 8 * xslot, (uint32_t)((box / P.nx) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                    mbar_expect_tx(bar, (uint32_t)P.xbox_bytes);
                     const uint32_t dst = x_s + xslot * P.xslot_bytes;
                     for (int l = 0; l < P.nloads; ++l)
-                        tma_load_5d(dst + P.load_off[l], &P.tmap_x, 0, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, ch.cbase >> 3,
-                                    bar_xfull + 8 * xslot);
+                        tma_load_5d(dst + P.load_off[l], &P.tmap_x, 0, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, cbase >> 3, bar);
                     ++box;
                     if (++xslot == (uint32_t)P.nx) xslot = 0;
                 }
@@ -289,13 +301,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 const int ns = ch.npad >> 4;
                 while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
                     const int o = ring.oldest;
-                    tc_wait(bar_pwdone + 8 * (o & (kTcNU - 1)), (uint32_t)(o / kTcNU) & 1u, &abort_flag, P.status,
-                                           kStatusWaitStage);
+                    tc_wait(bar_pwdone + 8 * (o & 3), (uint32_t)(o >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
                     ring.free_slabs += tab[o % P.nchunks].npad >> 4;
                     ++ring.oldest;
                 }
                 const int part = ((int)blockIdx.x + it * (int)gridDim.x) % P.nparts;
-                const uint32_t bar = bar_wfull + 8 * (v & (kTcNU - 1));
+                const uint32_t bar = bar_pwready + 8 * (v & 3);
                 mbar_expect_tx(bar, (uint32_t)ns * P.wslab_bytes);
                 const uint16_t *src = P.pw + ((size_t)part * P.nslabs_total + ch.slab0) * 16 * P.Dloc;
                 const int first = ns < P.nw - ring.head ? ns : P.nw - ring.head;
@@ -306,57 +317,68 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 if (++q == P.nchunks) { q = 0; ++it; }
             }
         }
-    } else if (warp >= 4 && warp < 8) {
+    } else if (warp >= 4 && warp < 4 + kTcConvWarps) {
         // ---------------- converter: z (fp32, TMEM) -> bf16 operand slabs ----------------
-        const int lg = warp & 3;
+        // Two warps per TMEM lane quarter; each takes every other 16-column granule of the chunk (at most 4), reads
+        // them with one wait, rounds and stores them.  Warp 4's first lane also releases, on behalf of the GDW issue
+        // warp, the B buffer and (after a window's last chunk) the input box that the chunk's products have read.
+        const int lg = warp & 3, half = (warp - 4) >> 2;
         const uint32_t r = (uint32_t)(lg * 32 + lane);
         SlabRing ring;
         ring.free_slabs = P.nz;
+        uint32_t bslot = 0, xslot = 0;
         int q = 0;
         for (int v = 0; v < total; ++v) {
-            const int ns = tab[q].npad >> 4;
+            const int ns = tab[q].npad >> 4, flags = tab[q].flags;
             while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
                 const int o = ring.oldest;
-                tc_warp_wait(bar_pwdone + 8 * (o & (kTcNU - 1)), (uint32_t)(o / kTcNU) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                tc_warp_wait(bar_pwdone + 8 * (o & 3), (uint32_t)(o >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
                 ring.free_slabs += tab[o % P.nchunks].npad >> 4;
                 ++ring.oldest;
             }
             tc_warp_wait(bar_zfull + 8 * (v & 1), (uint32_t)(v >> 1) & 1u, &abort_flag, P.status, kStatusWaitMma);
+            if (warp == 4 && lane == 0) {
+                mbar_arrive(bar_bfree + 8 * bslot);
+                if (flags & 2) mbar_arrive(bar_xfree + 8 * xslot);
+            }
+            if (++bslot == (uint32_t)P.nb) bslot = 0;
+            if (flags & 2) { if (++xslot == (uint32_t)P.nx) xslot = 0; }
             tc_fence_after();
             const uint32_t taddr = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(kTcZCol + 128 * (v & 1));
-            int slab = ring.head;
-            auto put = [&](const uint32_t (&acc)[16]) {
-                uint4 lo, hi;
-                lo.x = pack_bf16x2(__uint_as_float(acc[0]), __uint_as_float(acc[1]));
-                lo.y = pack_bf16x2(__uint_as_float(acc[2]), __uint_as_float(acc[3]));
-                lo.z = pack_bf16x2(__uint_as_float(acc[4]), __uint_as_float(acc[5]));
-                lo.w = pack_bf16x2(__uint_as_float(acc[6]), __uint_as_float(acc[7]));
-                hi.x = pack_bf16x2(__uint_as_float(acc[8]), __uint_as_float(acc[9]));
-                hi.y = pack_bf16x2(__uint_as_float(acc[10]), __uint_as_float(acc[11]));
-                hi.z = pack_bf16x2(__uint_as_float(acc[12]), __uint_as_float(acc[13]));
-                hi.w = pack_bf16x2(__uint_as_float(acc[14]), __uint_as_float(acc[15]));
-                const uint32_t addr = z_s + (uint32_t)slab * kTcSlab + r * 16u;
-                sts128(addr, lo);              // channels 0 .. 7 of the slab for this pixel: first core-matrix plane
-                sts128(addr + 2048u, hi);      // channels 8 .. 15: second plane
-                if (++slab == P.nz) slab = 0;
-            };
-#pragma unroll 1
-            for (int g = 0; g < ns; g += 2) {
-                uint32_t acc0[16], acc1[16];
-                tmem_ld16(taddr + (uint32_t)(g * 16), acc0);
-                if (g + 1 < ns) tmem_ld16(taddr + (uint32_t)(g * 16 + 16), acc1);
-                tmem_ld_wait();
-                put(acc0);
-                if (g + 1 < ns) put(acc1);
+            uint32_t acc[4][16];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (2 * j + half < ns) tmem_ld16(taddr + (uint32_t)((2 * j + half) * 16), acc[j]);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int g = 2 * j + half;
+                if (g < ns) {
+                    uint4 lo, hi;
+                    lo.x = pack_bf16x2(__uint_as_float(acc[j][0]), __uint_as_float(acc[j][1]));
+                    lo.y = pack_bf16x2(__uint_as_float(acc[j][2]), __uint_as_float(acc[j][3]));
+                    lo.z = pack_bf16x2(__uint_as_float(acc[j][4]), __uint_as_float(acc[j][5]));
+                    lo.w = pack_bf16x2(__uint_as_float(acc[j][6]), __uint_as_float(acc[j][7]));
+                    hi.x = pack_bf16x2(__uint_as_float(acc[j][8]), __uint_as_float(acc[j][9]));
+                    hi.y = pack_bf16x2(__uint_as_float(acc[j][10]), __uint_as_float(acc[j][11]));
+                    hi.z = pack_bf16x2(__uint_as_float(acc[j][12]), __uint_as_float(acc[j][13]));
+                    hi.w = pack_bf16x2(__uint_as_float(acc[j][14]), __uint_as_float(acc[j][15]));
+                    int slab = ring.head + g;
+                    if (slab >= P.nz) slab -= P.nz;
+                    const uint32_t addr = z_s + (uint32_t)slab * kTcSlab + r * 16u;
+                    sts128(addr, lo);              // channels 0 .. 7 of the slab for this pixel: first core-matrix plane
+                    sts128(addr + 2048u, hi);      // channels 8 .. 15: second plane
+                }
             }
             fence_proxy_async();
             tc_fence_before();
-            tc_warp_arrive(bar_zsfull + 8 * (v & (kTcNU - 1)));
+            tc_warp_arrive(bar_pwready + 8 * (v & 3));
+            tc_warp_arrive(bar_zfree + 8 * (v & 1));
             ring.head = (ring.head + ns) % P.nz;
             ring.free_slabs -= ns;
             if (++q == P.nchunks) q = 0;
         }
-    } else if (warp >= 8 && warp < 12) {
+    } else if (warp >= kTcEpiWarp0 && warp < kTcEpiWarp0 + 4) {
         // ---------------- epilogue: TMEM -> bias / ReLU -> bf16 -> global ----------------
         const int lg = warp & 3;
         const int r = lg * 32 + lane;
@@ -364,7 +386,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         const int tn = r / hw;
         const int rem = r - tn * hw;
         const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
-        const bool issuer = warp == 8 && lane == 0;
+        const bool issuer = warp == kTcEpiWarp0 && lane == 0;
         for (int it = 0; it < my_items; ++it) {
             const int item = (int)blockIdx.x + it * (int)gridDim.x;
             int tile = item / P.nparts;
@@ -430,11 +452,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             }
         }
         if (P.ostage && issuer) bulk_wait_all();
-    } else if (warp >= 12) {
+    } else if (warp >= kTcBuildWarp0) {
         // ---------------- builder: filter taps -> B operands of the GDW products ----------------
         // Thread t owns intermediate slot t of the current chunk.  The B operand of tap (ur, v) is a [n x 16]
         // K-major matrix whose row t has the tap's value in column `channel of slot t inside the window`.
-        const int t = tid - 384;
+        const int t = tid - kTcBuildWarp0 * 32;
         constexpr int RW = (1 + K * K + 7) / 8 * 4;         // 32-bit words of a filter record
         const uint32_t rowoff = (uint32_t)((t >> 3) * 128 + (t & 7) * 16);
         uint32_t rec[RW], nxt[RW];
@@ -476,7 +498,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             }
             bold[bslot * 128 + t] = (uint16_t)(valid ? off : 0xFFFFu);
             fence_proxy_async();
-            tc_warp_arrive(bar_bfull + 8 * bslot);
+            tc_warp_arrive(bar_dwready + 8 * (v & 3));
             if (++bslot == (uint32_t)P.nb) bslot = 0;
         }
     }
