@@ -46,6 +46,7 @@ constexpr int kTcMaxNB = 4;           // B operand buffers of the GDW stage (one
 constexpr int kTcMaxNX = 4;           // input box slots
 constexpr int kTcMaxTaps = 25;
 constexpr int kTcZCol = 256;          // TMEM columns 256..511: two GDW accumulators of up to 128 columns
+constexpr uint32_t kTcSw32 = 6u << 29;   // descriptor high word: layout type "32-byte swizzle"
 constexpr int kTcSlab = 4096;         // bytes of one z slab: 128 pixels x 16 channels of bf16
 constexpr int kTcMaxChunks = 256;
 
@@ -64,30 +65,12 @@ struct alignas(64) TcParams {
     int load_dw[kTcMaxTaps], load_dh[kTcMaxTaps];
     uint32_t load_off[kTcMaxTaps];
     uint32_t tap_row_step, tap_col_step;   // the A operand of tap (u, v) starts u * row_step + v * col_step bytes into the box
-    uint32_t a_lbo, a_sbo;       // GDW A operand: bytes between the two 8-channel planes, between 8-pixel groups
+    uint32_t a_sbo;              // GDW A operand: bytes between 8-pixel groups
     int nb, nx, nz, nw, nacc;
-    uint32_t bbuf_bytes, bplane, b_lbo, xslot_bytes, wslab_bytes;
+    uint32_t bbuf_bytes, bplane, xslot_bytes, wslab_bytes;
     uint32_t off_b, off_z, off_w, off_x, off_tab;    // from the 1024-aligned base; the output staging comes first
     int ostage, rec_hw, nslabs_total, bias_len;
 };
-
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *tmap, int c0, int c1, int c2, int c3, int c4,
-                                            uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar) : "memory");
-}
-
-// Shared-memory matrix descriptor without swizzle (descriptor version 1): K-major canonical layout.
-__device__ __forceinline__ uint64_t make_sdesc_plain(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= 1ull << 46;
-    return d;
-}
 
 // Bounded wait of every role but the MMA warp: each poll lets the hardware suspend the thread until the phase
 // completes (or 16 us pass), so that waiting warps issue next to nothing.  The MMA warp is a single
@@ -125,7 +108,7 @@ template <int K>
 __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_constant__ TcParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    // dwready[4] | zfull[2] zfree[2] | pwready[4] pwdone[4] | bfree[4] xfree[4] | accfull[2] accfree[2]
+    // dwready[4] | zfull[2] (2 unused) | pwready[4] pwdone[4] | bfree[4] xfree[4] | accfull[2] accfree[2]
     __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -134,13 +117,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const uint32_t base_s = smem_u32(base);
     const uint32_t o_s = base_s, b_s = base_s + P.off_b, z_s = base_s + P.off_z, w_s = base_s + P.off_w, x_s = base_s + P.off_x;
     // dwready: the B operands (4 builder warps) and the input box (the loader's arrive, with the box's bytes when the
-    // chunk opens a window) of a chunk are in place.  zfull: its GDW products are done.  zfree: the converter has read
-    // them out of TMEM.  pwready: the chunk's z slabs (8 converter warps) and its pointwise weights (the loader's
+    // chunk opens a window) of a chunk are in place.  zfull: its GDW products are done.  pwready: the chunk's z slabs (8 converter warps) and its pointwise weights (the loader's
     // arrive with their bytes) are in place.  pwdone: its PW products are done.  bfree / xfree: arrived by the
     // converter once the GDW products that read a B buffer / the last ones that read a box are done.
     const uint32_t bar_dwready = smem_u32(&bars[0]);
-    const uint32_t bar_zfull = bar_dwready + 32, bar_zfree = bar_zfull + 16;
-    const uint32_t bar_pwready = bar_zfree + 16, bar_pwdone = bar_pwready + 8 * kTcNU;
+    const uint32_t bar_zfull = bar_dwready + 32;
+    const uint32_t bar_pwready = bar_zfull + 32, bar_pwdone = bar_pwready + 8 * kTcNU;
     const uint32_t bar_bfree = bar_pwdone + 8 * kTcNU, bar_xfree = bar_bfree + 8 * kTcMaxNB;
     const uint32_t bar_accfull = bar_xfree + 8 * kTcMaxNX, bar_accfree = bar_accfull + 16;
     TcChunk *tab = reinterpret_cast<TcChunk *>(base + P.off_tab);
@@ -152,7 +134,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         abort_flag = 0;
         for (int i = 0; i < 4; ++i) mbar_init(bar_dwready + 8 * i, 5);
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_zfull + 8 * i, 1); mbar_init(bar_zfree + 8 * i, kTcConvWarps);
+            mbar_init(bar_zfull + 8 * i, 1);
             mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4);
         }
         for (int i = 0; i < kTcNU; ++i) { mbar_init(bar_pwready + 8 * i, kTcConvWarps + 1); mbar_init(bar_pwdone + 8 * i, 1); }
@@ -180,85 +162,89 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const int my_items = ((int)P.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const int total = my_items * P.nchunks;
     const int tiles_hw = P.tiles_h * P.tiles_w;
-    const uint32_t p_hi = (128u >> 4) | (1u << 14);     // descriptor high word: 8-row groups 128 bytes apart, version 1
+    const uint32_t p_hi = (256u >> 4) | (1u << 14) | kTcSw32;   // descriptor high word: 8-row groups 256 bytes apart, version 1, 32-byte swizzle
 
-    // The two issue warps are single instruction streams that pace the pipeline: a satisfied mbarrier wait costs them
-    // some 140 cycles and a tcgen05.commit some 80, against 24 per tcgen05.mma (measured), while the tensor-core work of
-    // a chunk is a few hundred cycles.  Hence one wait and one commit per chunk and warp, the GDW and the PW products
-    // issued by different warps, and descriptors advanced as 32-bit words.
+    // The issue warp is a single instruction stream that paces the pipeline: a satisfied mbarrier wait costs it some
+    // 140 cycles and a tcgen05.commit some 80, against 24 per tcgen05.mma (measured), while the tensor-core work of a
+    // chunk is a few hundred cycles.  Hence one wait and one commit per chunk and stage, and descriptors advanced as
+    // 32-bit words.  Both stages are issued by the same warp: products into different accumulators issued alternately
+    // (by two warps) ran several times slower than the same products issued stage by stage.
     if (warp == 0) {
-        // ---------------- GDW issue: the k*k products of chunk u into accumulator u & 1 ----------------
-        const uint32_t a_hi = ((P.a_sbo >> 4) & 0x3FFFu) | (1u << 14);
-        const uint32_t a_lo0 = ((x_s & 0x3FFFFu) >> 4) | (((P.a_lbo >> 4) & 0x3FFFu) << 16);
-        const uint32_t b_lo0 = ((b_s & 0x3FFFFu) >> 4) | (((P.b_lbo >> 4) & 0x3FFFu) << 16);
+        // ---------------- MMA issue ----------------
+        // Unit u: the k*k GDW products of chunk u into accumulator u & 1, then the PW products of chunk u-1, whose z
+        // the converter rounds meanwhile.  Accumulator u & 1 is free again once the converter has announced the slabs
+        // of chunk u-2 (it reads TMEM before that), which this warp waited for before the PW products of chunk u-2.
+        const uint32_t a_hi = ((P.a_sbo >> 4) & 0x3FFFu) | (1u << 14) | kTcSw32;
+        const uint32_t a_lo0 = ((x_s & 0x3FFFFu) >> 4) | (1u << 16);
+        const uint32_t b_lo0 = ((b_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t xstep = P.xslot_bytes >> 4, bstep = P.bbuf_bytes >> 4, pstep = P.bplane >> 4;
         const uint32_t rstep = P.tap_row_step >> 4, cstep = P.tap_col_step >> 4;
-        uint32_t xslot = 0, bslot = 0;
-        int q = 0;
-        for (int u = 0; u < total; ++u) {
-            const int npad = tab[q].npad, flags = tab[q].flags;
-            mbar_wait(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
-            if (u >= 2) mbar_wait(bar_zfree + 8 * (u & 1), (uint32_t)((u >> 1) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
-            tc_fence_after();
-            if (elect_one()) {
-                const uint32_t idesc = make_idesc(npad, false);
-                const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
-                const uint32_t a_lo = a_lo0 + xslot * xstep, b_lo = b_lo0 + bslot * bstep;
-#pragma unroll
-                for (int ur = 0; ur < K; ++ur)
-#pragma unroll
-                    for (int v = 0; v < K; ++v)
-                        umma_bf16_words(d_z, a_lo + (uint32_t)ur * rstep + (uint32_t)v * cstep, a_hi,
-                                        b_lo + (uint32_t)(ur * K + v) * pstep, p_hi, idesc, (ur | v) != 0);
-                umma_commit(bar_zfull + 8 * (u & 1));
-            }
-            __syncwarp();
-            if (++bslot == (uint32_t)P.nb) bslot = 0;
-            if (flags & 2) { if (++xslot == (uint32_t)P.nx) xslot = 0; }
-            if (++q == P.nchunks) q = 0;
-        }
-    } else if (warp == 3) {
-        // ---------------- PW issue: chunk v's slabs times its weights into the work item's accumulator ----------------
         const uint32_t idesc_pw = make_idesc(P.Dloc, false);
-        const uint32_t z_lo0 = ((z_s & 0x3FFFFu) >> 4) | ((2048u >> 4) << 16);
-        const uint32_t w_lo0 = ((w_s & 0x3FFFFu) >> 4) | ((((uint32_t)P.Dloc * 16u) >> 4) << 16);
+        const uint32_t z_lo0 = ((z_s & 0x3FFFFu) >> 4) | (1u << 16);
+        const uint32_t w_lo0 = ((w_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t wstep = P.wslab_bytes >> 4;
+        uint32_t xslot = 0, bslot = 0;
         uint32_t zhead = 0, whead = 0, buf = 0, accpar = 1;
-        int q = 0, it = 0;
-        for (int v = 0; v < total; ++v) {
-            const int ns = tab[q].npad >> 4;
-            if (q == 0 && it >= P.nacc) mbar_wait(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
-            mbar_wait(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
-            tc_fence_after();
-            if (elect_one()) {
-                const uint32_t d_y = tmem + buf * 128u;
-                if (zhead + (uint32_t)ns <= (uint32_t)P.nz && whead + (uint32_t)ns <= (uint32_t)P.nw) {
-                    const uint32_t z_lo = z_lo0 + zhead * (kTcSlab >> 4), w_lo = w_lo0 + whead * wstep;
+        int q = 0;                  // chunk index of unit u within its work item
+        int qp = 0, itp = 0;        // the same for unit u - 1, and its work item
+        for (int u = 0; u <= total; ++u) {
+            if (u < total) {
+                const int npad = tab[q].npad, flags = tab[q].flags;
+                mbar_wait(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint32_t idesc = make_idesc(npad, false);
+                    const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
+                    const uint32_t a_lo = a_lo0 + xslot * xstep, b_lo = b_lo0 + bslot * bstep;
 #pragma unroll
-                    for (int s = 0; s < 8; ++s)      // a chunk has at most 8 slabs (128 intermediate channels)
-                        if (s < ns)
-                            umma_bf16_words(d_y, z_lo + (uint32_t)s * (kTcSlab >> 4), p_hi, w_lo + (uint32_t)s * wstep, p_hi, idesc_pw,
-                                            (q | s) != 0);
-                } else {                              // the chunk wraps around the end of a ring
-                    uint32_t zh = zhead, wh = whead;
-#pragma unroll 1
-                    for (int s = 0; s < ns; ++s) {
-                        umma_bf16_words(d_y, z_lo0 + zh * (kTcSlab >> 4), p_hi, w_lo0 + wh * wstep, p_hi, idesc_pw, (q | s) != 0);
-                        if (++zh == (uint32_t)P.nz) zh = 0;
-                        if (++wh == (uint32_t)P.nw) wh = 0;
-                    }
+                    for (int ur = 0; ur < K; ++ur)
+#pragma unroll
+                        for (int v = 0; v < K; ++v)
+                            umma_bf16_words(d_z, a_lo + (uint32_t)ur * rstep + (uint32_t)v * cstep, a_hi,
+                                            b_lo + (uint32_t)(ur * K + v) * pstep, p_hi, idesc, (ur | v) != 0);
+                    umma_commit(bar_zfull + 8 * (u & 1));
                 }
-                umma_commit(bar_pwdone + 8 * (v & 3));
-                if (q == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
+                __syncwarp();
+                if (++bslot == (uint32_t)P.nb) bslot = 0;
+                if (flags & 2) { if (++xslot == (uint32_t)P.nx) xslot = 0; }
+                if (++q == P.nchunks) q = 0;
             }
-            __syncwarp();
-            zhead += (uint32_t)ns;
-            if (zhead >= (uint32_t)P.nz) zhead -= (uint32_t)P.nz;
-            whead += (uint32_t)ns;
-            if (whead >= (uint32_t)P.nw) whead -= (uint32_t)P.nw;
-            if (++q == P.nchunks) {
-                q = 0; ++it;
-                if (++buf == (uint32_t)P.nacc) { buf = 0; accpar ^= 1; }
+            if (u > 0) {
+                const int v = u - 1;
+                const int ns = tab[qp].npad >> 4;
+                if (qp == 0 && itp >= P.nacc) mbar_wait(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
+                mbar_wait(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint32_t d_y = tmem + buf * 128u;
+                    if (zhead + (uint32_t)ns <= (uint32_t)P.nz && whead + (uint32_t)ns <= (uint32_t)P.nw) {
+                        const uint32_t z_lo = z_lo0 + zhead * (kTcSlab >> 4), w_lo = w_lo0 + whead * wstep;
+#pragma unroll
+                        for (int s = 0; s < 8; ++s)      // a chunk has at most 8 slabs (128 intermediate channels)
+                            if (s < ns)
+                                umma_bf16_words(d_y, z_lo + (uint32_t)s * (kTcSlab >> 4), p_hi, w_lo + (uint32_t)s * wstep, p_hi,
+                                                idesc_pw, (qp | s) != 0);
+                    } else {                              // the chunk wraps around the end of a ring
+                        uint32_t zh = zhead, wh = whead;
+#pragma unroll 1
+                        for (int s = 0; s < ns; ++s) {
+                            umma_bf16_words(d_y, z_lo0 + zh * (kTcSlab >> 4), p_hi, w_lo0 + wh * wstep, p_hi, idesc_pw, (qp | s) != 0);
+                            if (++zh == (uint32_t)P.nz) zh = 0;
+                            if (++wh == (uint32_t)P.nw) wh = 0;
+                        }
+                    }
+                    umma_commit(bar_pwdone + 8 * (v & 3));
+                    if (qp == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
+                }
+                __syncwarp();
+                zhead += (uint32_t)ns;
+                if (zhead >= (uint32_t)P.nz) zhead -= (uint32_t)P.nz;
+                whead += (uint32_t)ns;
+                if (whead >= (uint32_t)P.nw) whead -= (uint32_t)P.nw;
+                if (++qp == P.nchunks) {
+                    qp = 0; ++itp;
+                    if (++buf == (uint32_t)P.nacc) { buf = 0; accpar ^= 1; }
+                }
             }
         }
     } else if (warp == 1) {
@@ -284,7 +270,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     mbar_expect_tx(bar, (uint32_t)P.xbox_bytes);
                     const uint32_t dst = x_s + xslot * P.xslot_bytes;
                     for (int l = 0; l < P.nloads; ++l)
-                        tma_load_5d(dst + P.load_off[l], &P.tmap_x, 0, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, cbase >> 3, bar);
+                        tma_load_4d(dst + P.load_off[l], &P.tmap_x, cbase, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, bar);
                     ++box;
                     if (++xslot == (uint32_t)P.nx) xslot = 0;
                 }
@@ -365,15 +351,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     hi.w = pack_bf16x2(__uint_as_float(acc[j][14]), __uint_as_float(acc[j][15]));
                     int slab = ring.head + g;
                     if (slab >= P.nz) slab -= P.nz;
-                    const uint32_t addr = z_s + (uint32_t)slab * kTcSlab + r * 16u;
-                    sts128(addr, lo);              // channels 0 .. 7 of the slab for this pixel: first core-matrix plane
-                    sts128(addr + 2048u, hi);      // channels 8 .. 15: second plane
+                    const uint32_t addr = z_s + (uint32_t)slab * kTcSlab + r * 32u;
+                    const uint32_t sw = ((r >> 2) & 1u) << 4;   // 32-byte swizzle: address bit 4 ^= bit 7
+                    sts128(addr + sw, lo);                 // channels 0 .. 7 of the slab for this pixel
+                    sts128(addr + (sw ^ 16u), hi);         // channels 8 .. 15
                 }
             }
             fence_proxy_async();
             tc_fence_before();
             tc_warp_arrive(bar_pwready + 8 * (v & 3));
-            tc_warp_arrive(bar_zfree + 8 * (v & 1));
             ring.head = (ring.head + ns) % P.nz;
             ring.free_slabs -= ns;
             if (++q == P.nchunks) q = 0;
@@ -458,7 +444,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         // K-major matrix whose row t has the tap's value in column `channel of slot t inside the window`.
         const int t = tid - kTcBuildWarp0 * 32;
         constexpr int RW = (1 + K * K + 7) / 8 * 4;         // 32-bit words of a filter record
-        const uint32_t rowoff = (uint32_t)((t >> 3) * 128 + (t & 7) * 16);
+        const uint32_t rowoff = (uint32_t)t * 32u, rowsw = (uint32_t)(t >> 2) & 1u;   // row of slot t; 32-byte swizzle phase
         uint32_t rec[RW], nxt[RW];
         auto load_rec = [&](const TcChunk &ch, uint32_t (&dst)[RW]) {
             if (t < ch.npad) {
@@ -483,7 +469,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             if (v + 1 < total) load_rec(tab[q], nxt);
             const uint32_t cw = rec[0] & 0xFFFFu;
             const bool valid = cw != 0xFFFFu;
-            const uint32_t off = (cw >> 3) * P.b_lbo + rowoff + (cw & 7u) * 2u;
+            const uint32_t off = rowoff + ((((cw >> 3) & 1u) ^ rowsw) << 4) + (cw & 7u) * 2u;
             if (v >= P.nb) tc_warp_wait(bar_bfree + 8 * bslot, (uint32_t)((v / P.nb) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
             const uint32_t bb = b_s + bslot * P.bbuf_bytes;
             const uint32_t old = bold[bslot * 128 + t];
@@ -531,8 +517,8 @@ __global__ void tc_pack_filt_kernel(const void *__restrict__ dw, int is_bf16, in
     }
 }
 
-// pw_w[D][G] -> [part][slab][8-channel plane][output channel][8] bf16: per 16 intermediate slots one K-major
-// operand slab of the pointwise product, core matrices of 8 output channels x 8 slots stored contiguously.
+// pw_w[D][G] -> [part][slab][output channel][16] bf16: per 16 intermediate slots one K-major operand slab of the
+// pointwise product, 32 bytes per output channel, 32-byte swizzle.
 __global__ void tc_pack_pw_kernel(const void *__restrict__ pw, int is_bf16, int D, int G, int Dloc, int nslabs,
                                   const TcChunk *__restrict__ chunks, uint16_t *__restrict__ out)
 {
@@ -542,13 +528,13 @@ __global__ void tc_pack_pw_kernel(const void *__restrict__ pw, int is_bf16, int 
     for (int e = threadIdx.x; e < (ch.npad >> 4) * per_slab; e += blockDim.x) {
         const int s = e / per_slab;
         int rem = e - s * per_slab;
-        const int kg = rem / (8 * Dloc);
-        rem -= kg * 8 * Dloc;
-        const int dl = rem >> 3, el = rem & 7;
-        const int t = s * 16 + kg * 8 + el, d = part * Dloc + dl;
+        const int dl = rem >> 4, kk = rem & 15;
+        const int t = s * 16 + kk, d = part * Dloc + dl;
         float val = 0.f;
         if (t < ch.n && d < D) val = tc_load_weight(pw, (size_t)d * G + ch.i0 + t, is_bf16);
-        out[((size_t)part * nslabs + ch.slab0 + s) * per_slab + (size_t)kg * 8 * Dloc + dl * 8 + el] = float_to_bf16_bits(val);
+        // row dl of the slab: 32 bytes, its two 16-byte halves swapped in rows 4..7 of every 8 (32-byte swizzle)
+        out[((size_t)part * nslabs + ch.slab0 + s) * per_slab + dl * 16 + ((((kk >> 3) ^ ((dl >> 2) & 1))) << 3) + (kk & 7)] =
+            float_to_bf16_bits(val);
     }
 }
 
@@ -623,9 +609,9 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     memset(&P, 0, sizeof(P));
     const int Dloc = p->tc_dloc, m = p->tc_maxslabs;
     const uint32_t nmax = (uint32_t)tc_nmax(k, Dloc);
-    P.bplane = nmax * 32u; P.b_lbo = nmax * 16u; P.bbuf_bytes = (uint32_t)(k * k) * P.bplane;
+    P.bplane = nmax * 32u; P.bbuf_bytes = (uint32_t)(k * k) * P.bplane;
     P.wslab_bytes = (uint32_t)Dloc * 32u;
-    P.xslot_bytes = (uint32_t)((g.xbox + 127) / 128 * 128);
+    P.xslot_bytes = (uint32_t)((g.xbox + 255) / 256 * 256);
     // Shared memory: output staging (optional) | B operand buffers | z slabs | weight slabs | input boxes | tables
     const bool can_stage = p->D % 64 == 0 && Dloc % 64 == 0 && ((uintptr_t)y->ptr & 15) == 0 && nitems > p->sm_count;
     const size_t tables = (size_t)nchunks * sizeof(TcChunk) + (size_t)p->tc_nparts * Dloc * 4 + kTcMaxNB * 256 + 256;
@@ -655,16 +641,16 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     if (smem < (size_t)kMaxSmem / 2 + 4096) smem = (size_t)kMaxSmem / 2 + 4096;   // one block per SM: it owns all of TMEM
     if (smem > (size_t)kMaxSmem) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: shared memory plan exceeds the limit");
 
-    {   // x as a rank-5 tensor, innermost first: 8 channels, width, height, batch, 8-channel group
-        const cuuint64_t dims[5] = {8, (cuuint64_t)x->w, (cuuint64_t)x->h, (cuuint64_t)x->n, (cuuint64_t)(p->C / 8)};
-        const cuuint64_t strides[4] = {(cuuint64_t)p->C * 2, (cuuint64_t)x->w * p->C * 2, (cuuint64_t)x->h * x->w * p->C * 2, 16};
-        cuuint32_t box[5] = {8, (cuuint32_t)g.IW, 0, (cuuint32_t)g.TN, 2};
+    {   // x as a rank-4 tensor, innermost first: channels, width, height, batch; a box holds 16 channels (32 bytes) per pixel
+        const cuuint64_t dims[4] = {(cuuint64_t)p->C, (cuuint64_t)x->w, (cuuint64_t)x->h, (cuuint64_t)x->n};
+        const cuuint64_t strides[3] = {(cuuint64_t)p->C * 2, (cuuint64_t)x->w * p->C * 2, (cuuint64_t)x->h * x->w * p->C * 2};
+        cuuint32_t box[4] = {16, (cuuint32_t)g.IW, 0, (cuuint32_t)g.TN};
         box[2] = (cuuint32_t)(g.layout == 1 ? g.PH + k - 1 : g.PH);
-        const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-        const CUresult r = encode(&P.tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x->ptr, dims, strides, box, estr,
-                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        const CUresult r = encode(&P.tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, x->ptr, dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled (x, rank 5) failed with code %d", (int)r);
+        if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled (x) failed with code %d", (int)r);
     }
     if (P.ostage) {
         const cuuint64_t dims[4] = {(cuuint64_t)p->D, (cuuint64_t)Wo, (cuuint64_t)Ho, (cuuint64_t)x->n};
@@ -679,16 +665,16 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
         P.tmap_y = P.tmap_x;
     }
     // Where each copy of the box goes, and where the A operand of tap (u, v) starts.
-    const uint32_t px = 16;      // bytes of one staged pixel within a plane (8 channels)
+    const uint32_t px = 32;      // bytes of one staged pixel (16 channels)
     if (g.layout == 1) {
         P.nloads = 1; P.load_dw[0] = 0; P.load_dh[0] = 0; P.load_off[0] = 0;
-        P.a_lbo = (uint32_t)((g.PH + k - 1) * g.IW) * px; P.a_sbo = (uint32_t)g.IW * px;
+        P.a_sbo = 8u * (uint32_t)g.IW * px / 8u;
         P.tap_row_step = (uint32_t)g.IW * px; P.tap_col_step = px;
     } else if (g.layout == 2) {
-        const uint32_t copy = 2u * 16u * (uint32_t)g.IW * px;
+        const uint32_t copy = 16u * (uint32_t)g.IW * px;
         P.nloads = k;
         for (int u = 0; u < k; ++u) { P.load_dw[u] = 0; P.load_dh[u] = u; P.load_off[u] = (uint32_t)u * copy; }
-        P.a_lbo = 16u * (uint32_t)g.IW * px; P.a_sbo = (uint32_t)g.IW * px;
+        P.a_sbo = (uint32_t)g.IW * px;
         P.tap_row_step = copy; P.tap_col_step = px;
     } else {
         P.nloads = k * k;
@@ -696,7 +682,7 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
             P.load_dw[u * k + v] = v; P.load_dh[u * k + v] = u; P.load_off[u * k + v] = (uint32_t)(u * k + v) * 4096u;
         }
         P.tap_row_step = (uint32_t)k * 4096u; P.tap_col_step = 4096u;
-        P.a_lbo = 2048u; P.a_sbo = 128u;
+        P.a_sbo = 256u;
     }
     P.xbox_bytes = g.xbox;
     P.y = (uint16_t *)y->ptr; P.filt = p->d_tc_filt; P.pw = p->d_tc_pw; P.bias = p->d_bias; P.chunks = p->d_tc_chunks;
