@@ -212,6 +212,47 @@ def run_reference(args, spec):
     print(json.dumps(out), flush=True)
 
 
+def dense_conv_context(spec: gi.LayerSpec, data, x0, nsets: int, steps: int):
+    """Context only, not part of the product path: the dense k x k convolution that the GDWS layer replaces
+    (Eq. 1), run by the vendor library through torch (bf16, channels_last), with the dense weights rebuilt from
+    the layer's factors (Property 1 and 2: W[d, c] = sum_j P[d, off_c + j] K[off_c + j]).  Same batch, same
+    rotation of input buffers, CUDA events."""
+    import torch
+    import torch.nn.functional as F
+    if spec.dtype != "bf16":
+        return None
+    k2 = spec.k * spec.k
+    off = np.concatenate([[0], np.cumsum(data.g)]).astype(np.int64)
+    Wd = np.zeros((spec.D, spec.C, k2), dtype=np.float32)
+    Kf = data.dw_w.reshape(-1, k2).astype(np.float32)
+    for c in range(spec.C):
+        a, b = off[c], off[c + 1]
+        if b > a:
+            Wd[:, c, :] = data.pw_w[:, a:b].astype(np.float32) @ Kf[a:b]
+    w = torch.from_numpy(Wd.reshape(spec.D, spec.C, spec.k, spec.k)).cuda().to(torch.bfloat16).contiguous(memory_format=torch.channels_last)
+    b = torch.from_numpy(data.bias).cuda().to(torch.bfloat16)
+    xs = [x0.permute(0, 3, 1, 2)]                       # NHWC storage seen as NCHW channels_last
+    xs += [xs[0].clone(memory_format=torch.channels_last) for _ in range(min(nsets, 16) - 1)]
+    run = lambda i: F.conv2d(xs[i % len(xs)], w, b, stride=spec.stride, padding=spec.pad)
+    for i in range(5):
+        run(i)
+    torch.cuda.synchronize()
+    n = max(10, min(steps, 200))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(n):
+        run(i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    return {"what": "dense k x k conv of the same layer, vendor library via torch (bf16 channels_last, plain launches)",
+            "ms_per_step": ms, "images_per_s": spec.N / (ms * 1e-3), "dense_macs": spec.N * spec.Ho * spec.Wo * spec.D * spec.C * k2}
+
+
+PAPER_CONTEXT = ("paper (Table 1, App. A.1): whole networks at batch 1 on a Jetson Xavier NX (384-core Volta GPU), PyTorch 1.8, "
+                 "frames/s baseline -> GDWS: ResNet-50 16 -> 37, WRN-28-4 17 -> 65, ResNet-18 28 -> 104, VGG-16 36 -> 129 (CIFAR-10)")
+
+
 def workload_config(spec: gi.LayerSpec, G: int):
     return {"workload": f"{spec.name}: N={spec.N} C={spec.C} D={spec.D} {spec.H}x{spec.W} k={spec.k} "
                         f"stride={spec.stride} pad={spec.pad} g~{spec.g_dist} G={G} {spec.dtype} {spec.layout}",
@@ -383,9 +424,9 @@ def run_ours(args, spec):
     t_roof = max(t_roof, t_alu)
     t_roof_s = max(t_roof_s, t_alu)
     roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
-            "traffic": TRAFFIC_BYTES_PER_LAUNCH.get((args.config, args.layer, args.path)) if not f32 else None,
+            "traffic": TRAFFIC_BYTES_PER_LAUNCH.get((args.config, args.layer, args.path)) if (not f32 and args.dw_math != 2) else None,
             "peak_source": psrc,
-            "kernel": "fused_bf16_kernel" if (not f32 and path != gdws.PATH_UNFUSED) else "see config.path",
+            "kernel": ("fused_tc_kernel" if args.dw_math == 2 else "fused_bf16_kernel") if (not f32 and path != gdws.PATH_UNFUSED) else "see config.path",
             "layer_roofline_us": t_roof, "t_tensor_us": t_tensor, "t_hbm_us": t_hbm, "t_alu_us": t_alu,
             "frac_of_layer_roofline": t_roof / us, "frac_of_layer_roofline_sustained_peak": t_roof_s / us}
 
@@ -405,8 +446,15 @@ def run_ours(args, spec):
                              relu=spec.relu, layout=spec.layout)
         parity = float(np.max(np.abs(yg - ref)) / np.max(np.abs(ref)))
 
+    context = {"paper": PAPER_CONTEXT}
+    if args.context:
+        try:
+            context["dense_conv"] = dense_conv_context(spec, data, x0, nsets, args.steps)
+        except Exception as exc:      # context only: never fails the bench line
+            context["dense_conv"] = {"unavailable": repr(exc)[:200]}
+
     cfg = workload_config(spec, G)
-    cfg.update({"path": args.path, "launch": "cuda graph replay" if graph is not None else "plain launches",
+    cfg.update({"path": args.path, "gdw_stage": "tensor cores" if args.dw_math == 2 else "ALUs", "launch": "cuda graph replay" if graph is not None else "plain launches",
                 "l2": f"rotating {nsets} input/output buffer sets ({nsets * set_bytes / 1e6:.0f} MB > 126 MB L2)"
                       if nsets > 1 else "one buffer set larger than L2",
                 "tile": "TNxPHxPW=%dx%dx%d" % plan.tile(spec.N, spec.H, spec.W)[:3] if not f32 else None,
@@ -417,7 +465,7 @@ def run_ours(args, spec):
         "dtype": spec.dtype, "data": "synthetic", "config": cfg,
         "effective_tmacs": world * macs / sec_per_step / 1e12,
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-        "clocks": clocks, "parity_max_rel_err": parity,
+        "clocks": clocks, "parity_max_rel_err": parity, "context": context,
     }
     print(json.dumps(out), flush=True)
     plan.destroy()
@@ -436,6 +484,7 @@ def main():
     ap.add_argument("--path", default="fused", choices=["fused", "unfused", "auto"])
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-check", dest="check", action="store_false")
+    ap.add_argument("--no-context", dest="context", action="store_false")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--dw-math", type=int, default=0)
     ap.add_argument("--a-layout", type=int, default=0)

@@ -80,11 +80,12 @@ typedef enum {
     GDWS_OPT_A_LAYOUT = 3, /* bf16 fused path, shared-memory layout of the intermediate
                               tile handed to the tensor cores: 0 = pixel-contiguous
                               (default), 1 = channel-contiguous                            */
-    GDWS_OPT_DW_MATH = 4   /* bf16 fused path, where the GDW stage runs: 0 = on the tensor cores
-                              (k*k block-sparse products per tile, fp32 accumulation) for the
-                              layers that kernel covers (stride 1, k <= 5), else on the ALUs;
-                              1 = on the ALUs (fp32 FMAs); 2 = on the tensor cores, or
-                              GDWS_ERR_UNSUPPORTED                                         */
+    GDWS_OPT_DW_MATH = 4   /* bf16 fused path, where the GDW stage runs: 0 (default) or 1 = on the
+                              ALUs (fp32 FMAs); 2 = on the tensor cores as k*k block-sparse
+                              products per 16-channel window (fp32 accumulation), for stride 1
+                              and k <= 5, else GDWS_ERR_UNSUPPORTED.  Both give the same
+                              result up to summation order; 2 is slower on the benchmark
+                              layers and is kept as a measured alternative                 */
 } gdws_option_t;
 
 typedef enum {

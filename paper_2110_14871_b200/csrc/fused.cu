@@ -871,11 +871,8 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
 
 gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t st)
 {
-    // GDWS_OPT_DW_MATH: 0 = GDW stage on the tensor cores where that kernel covers the layer, 1 = on the ALUs, 2 = tensor cores or fail
-    if (p->opt_dw_math != 1) {
-        const gdws_status_t rc = bf16_fused_tc(p, x, y, st);
-        if (rc != GDWS_ERR_UNSUPPORTED || p->opt_dw_math == 2) return rc;
-    }
+    // GDWS_OPT_DW_MATH: 0 or 1 = GDW stage on the ALUs (the faster kernel on every benchmark layer), 2 = on the tensor cores
+    if (p->opt_dw_math == 2) return bf16_fused_tc(p, x, y, st);
     return run_tiled(p, x, y->ptr, y->h, y->w, false, st);
 }
 

@@ -92,9 +92,8 @@ BF16_SHAPES = [
 ]
 
 
-# dw_math: 0 = GDW stage on the tensor cores where that kernel covers the layer, 1 = on the ALUs
-@pytest.mark.parametrize("path,a_layout,dw_math", [(gdws.PATH_UNFUSED, 0, 0), (gdws.PATH_FUSED, 0, 1), (gdws.PATH_FUSED, 1, 1),
-                                                   (gdws.PATH_FUSED, 0, 0)])
+# dw_math: 0 or 1 = GDW stage on the ALUs (default); 2 = on the tensor cores (own tests below)
+@pytest.mark.parametrize("path,a_layout,dw_math", [(gdws.PATH_UNFUSED, 0, 0), (gdws.PATH_FUSED, 0, 0), (gdws.PATH_FUSED, 1, 1)])
 @pytest.mark.parametrize("shape", BF16_SHAPES)
 def test_bf16_forward_matches_reference(shape, path, a_layout, dw_math):
     N, C, D, H, W, k, s, p, gd = shape
