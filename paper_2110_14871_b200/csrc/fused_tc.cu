@@ -4,28 +4,26 @@
 // tap (u,v) the GDW output of a tile of 128 pixels and a window of 16 input channels is
 //     z[pixel, i] += x[pixel shifted by (u,v), c] * B_uv[c, i],   B_uv[c, i] = K[i,u,v] if c = c(i), else 0,
 // i.e. a [128 x 16] x [16 x n] product per tap whose B operand has one non-zero per column.  The A operand is
-// not copied per tap: the staged input box lies in shared memory as [8-channel group][row][column][8 channels],
-// which for every tap is a valid K-major tensor-core operand (8 consecutive pixels of an output row are 8
-// consecutive 16-byte entries) that differs from the next tap's only in its start address.  The fp32 result
-// z (128 lanes x n columns of TMEM) is read back by four converter warps, rounded to bf16 and written as the
-// K-major A operand of the pointwise stage (Property 1: W_P is M x G), whose products accumulate in a second
-// TMEM region over all windows of the tile.  The ALUs only round z, scatter the filter taps into the B
-// operands and run the epilogue; they execute no multiply of the GDW stage.
+// not copied per tap: the staged input box lies in shared memory as [row][column][16 channels] (32 bytes per
+// pixel, 32-byte swizzle, written by TMA), which for every tap is a valid K-major tensor-core operand (8
+// consecutive pixels of an output row are 8 consecutive 32-byte rows) that differs from the next tap's only in
+// its start address.  The fp32 result z (128 lanes x n columns of TMEM) is read back by the converter warps,
+// rounded to bf16 and written as the K-major A operand of the pointwise stage (Property 1: W_P is M x G), whose
+// products accumulate in a second TMEM region over all windows of the tile.  The ALUs only round z, scatter the
+// filter taps into the B operands and run the epilogue; they execute no multiply of the GDW stage.
 //
-// One persistent block of 16 warps per SM walks over work items (tile of 128 output pixels x block of up to
+// One persistent block of 20 warps per SM walks over work items (tile of 128 output pixels x block of up to
 // 256 output channels).  Roles, coupled by mbarriers only:
-//   warp 0 (one lane)  issues every tcgen05.mma: for chunk u the k*k GDW products, then the PW products of
-//                      chunk u-1 (whose z is being converted meanwhile);
-//   warp 1 (one lane)  fetches the input boxes by TMA (rank-5 view of x: 8 channels, W, H, N, C/8);
+//   warp 0             issues every tcgen05.mma (one elected lane): for chunk u the k*k GDW products, then the
+//                      PW products of chunk u-1 (whose z is being converted meanwhile);
+//   warp 1 (one lane)  fetches the input boxes by TMA (x as a rank-4 tensor: C, W, H, N; 16 channels per box);
 //   warp 2 (one lane)  streams the packed pointwise weights (bulk copies into a ring of 16-channel slabs);
-//   warps 4-7          converter: TMEM z -> bf16 -> ring of 16-channel operand slabs;
-//   warps 8-11         epilogue: TMEM y -> bias, ReLU, bf16 -> global memory (TMA store or direct);
-//   warps 12-15        builder: one thread per intermediate channel of the chunk scatters its k taps of a filter
-//                      row into a B operand buffer that is otherwise zero, and clears what it wrote when the
-//                      buffer comes back.
-// All operands use the un-swizzled K-major canonical layout: core matrices of 8 rows x 16 bytes stored
-// contiguously, `leading byte offset` between the two core matrices along K, `stride byte offset` between
-// 8-row groups.  Every wait is bounded (see mbar_wait).
+//   warps 4-11         converter: TMEM z -> bf16 -> ring of 16-channel operand slabs (two warps per lane quarter);
+//   warps 12-15        epilogue: TMEM y -> bias, ReLU, bf16 -> global memory (TMA store or direct);
+//   warps 16-19        builder: one thread per intermediate channel of the chunk scatters its k*k taps into B
+//                      operand planes that are otherwise zero, and clears what it wrote when the buffer comes back.
+// All operands are K-major with 32-byte rows and the 32-byte swizzle (address bit 4 ^= bit 7), 8-row groups
+// `stride byte offset` apart.  Every wait is bounded (see mbar_wait, tc_wait).
 #include <string.h>
 
 #include <algorithm>
@@ -51,7 +49,7 @@ constexpr int kTcSlab = 4096;         // bytes of one z slab: 128 pixels x 16 ch
 constexpr int kTcMaxChunks = 256;
 
 struct alignas(64) TcParams {
-    CUtensorMap tmap_x;          // x as (8, W, H, N, C/8) bf16
+    CUtensorMap tmap_x;          // x as (C, W, H, N) bf16, box (16, IW, rows, TN), 32-byte swizzle
     CUtensorMap tmap_y;          // y as (D, Wo, Ho, N) bf16, box (64, PW, PH, TN), 128-byte swizzle (when ostage != 0)
     uint16_t *y;
     const uint16_t *filt;
@@ -117,8 +115,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const uint32_t base_s = smem_u32(base);
     const uint32_t o_s = base_s, b_s = base_s + P.off_b, z_s = base_s + P.off_z, w_s = base_s + P.off_w, x_s = base_s + P.off_x;
     // dwready: the B operands (4 builder warps) and the input box (the loader's arrive, with the box's bytes when the
-    // chunk opens a window) of a chunk are in place.  zfull: its GDW products are done.  pwready: the chunk's z slabs (8 converter warps) and its pointwise weights (the loader's
-    // arrive with their bytes) are in place.  pwdone: its PW products are done.  bfree / xfree: arrived by the
+    // chunk opens a window) of a chunk are in place.  zfull: its GDW products are done.  pwready: the chunk's z slabs
+    // (8 converter warps) and its pointwise weights (the loader's arrive with their bytes) are in place.  pwdone: its PW products are done.  bfree / xfree: arrived by the
     // converter once the GDW products that read a B buffer / the last ones that read a box are done.
     const uint32_t bar_dwready = smem_u32(&bars[0]);
     const uint32_t bar_zfull = bar_dwready + 32;
