@@ -9,7 +9,12 @@ warm-up, then successive inferences between two CUDA events, no host I/O in the 
 region), adapted to one layer and a batch.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--config C] [--layer L] [--path fused|unfused] [--no-graph]
+                    [--config C] [--layer L] [--path fused|unfused] [--no-graph] [--chain]
+
+A timed region is exactly K steps; it is repeated (--repeats, default: enough repeats for some tens of
+milliseconds) with a CUDA event between repeats, and the median region gives ms_per_step.  With CUDA graphs
+(default) every warm-up and timed launch is a graph node, whatever K is.  `--config 3 --chain` times the
+16 chained layers of config 3 as one graph (a step = the whole chain over the batch).
 
 Prints ONE JSON line.  With --gpus N > 1 (under torchrun) every rank runs an
 independent replica on its own GPU (the path has no exchange step); the value is the
@@ -60,9 +65,9 @@ def layer_numbers(spec: gi.LayerSpec, G: int):
     return px, macs, nbytes
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
-# summarised under profiles/ (key: config, layer, path).  An entry is removed when its kernel changes.
-TRAFFIC_BYTES_PER_LAUNCH = {(1, 0, "fused"): 9181696}   # y (8.39 MB) stays in L2 within the captured launch
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu captures
+# summarised under profiles/ (key: config, layer, path, GDW stage).  An entry is removed when its kernel changes.
+TRAFFIC_BYTES_PER_LAUNCH = {}
 
 
 def layer_roofline_us(macs, nbytes, peaks, sustained=False):
@@ -87,6 +92,34 @@ def slowest_rank(value: float, device=None) -> float:
 def aggregate_value(units_per_rank: float, world: int, seconds_slowest: float) -> float:
     """Whole-job throughput of `world` independent replicas: all units over the slowest rank's time."""
     return world * units_per_rank / seconds_slowest
+
+
+def percentile(v, q):
+    v = sorted(v)
+    return v[min(len(v) - 1, max(0, int(round(q * (len(v) - 1)))))]
+
+
+def timed_regions(run_region, repeats):
+    """Runs `run_region` `repeats` times back to back with a CUDA event between them; returns the
+    milliseconds of each region (device time on the current stream)."""
+    import torch
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+    evs[0].record()
+    for r in range(repeats):
+        run_region()
+        evs[r + 1].record()
+    torch.cuda.synchronize()
+    return [evs[r].elapsed_time(evs[r + 1]) for r in range(repeats)]
+
+
+def choose_repeats(args, region_ms_estimate):
+    """Repeats of the K-step region: given, or enough for about 60 ms of timed work (at least 5, at most 2000),
+    never more than about 20 s in total."""
+    if args.repeats > 0:
+        return args.repeats
+    r = int(np.ceil(60.0 / max(region_ms_estimate, 1e-3)))
+    r = max(5, min(2000, r))
+    return max(1, min(r, int(20000.0 / max(region_ms_estimate, 1e-3))))
 
 
 class ClockSampler:
@@ -328,9 +361,10 @@ def run_ours(args, spec):
     step(0)
     launches_per_step = plan.launch_count() - l0
 
-    graph = None
+    # Launch mode.  With graphs, two graphs cover any K: one of `nsets` launches (one per buffer set) and one of
+    # K mod nsets launches, so that every warm-up and timed launch is a graph node.
+    graphs = None
     if not args.no_graph:
-        g = torch.cuda.CUDAGraph()
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
@@ -338,35 +372,36 @@ def run_ours(args, spec):
                 plan.forward(xs[i], ys[i], spec.layout, stream=side, **wargs)
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
-        with torch.cuda.graph(g, stream=side):
-            for i in range(nsets):
-                plan.forward(xs[i], ys[i], spec.layout, stream=torch.cuda.current_stream(), **wargs)
-        graph = g
 
-    def run_steps(k):
-        if graph is None:
-            for i in range(k):
+        def capture(count):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(count):
+                    plan.forward(xs[i % nsets], ys[i % nsets], spec.layout, stream=torch.cuda.current_stream(), **wargs)
+            return g
+        graphs = (capture(nsets), capture(args.steps % nsets) if args.steps % nsets else None)
+
+    def run_region():
+        if graphs is None:
+            for i in range(args.steps):
                 step(i)
         else:
-            full, rem = divmod(k, nsets)
-            for _ in range(full):
-                graph.replay()
-            for i in range(rem):
-                step(i)
+            for _ in range(args.steps // nsets):
+                graphs[0].replay()
+            if graphs[1] is not None:
+                graphs[1].replay()
 
-    for _ in range(3):
-        run_steps(max(args.warmup, 3))
+    for _ in range(max(3, -(-args.warmup // max(1, args.steps)))):     # at least W warm-up steps, in whole regions
+        run_region()
     torch.cuda.synchronize()
+    probe = timed_regions(run_region, 3)
+    repeats = choose_repeats(args, min(probe))
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clk:
-        ev0.record()
-        run_steps(args.steps)
-        ev1.record()
-        torch.cuda.synchronize()
-    ms = ev0.elapsed_time(ev1)
+        region_ms = timed_regions(run_region, repeats)
+    ms = statistics.median(region_ms)
     if world > 1:
         dist.barrier()
         ms = slowest_rank(ms, device="cuda")
@@ -407,7 +442,9 @@ def run_ours(args, spec):
     clocks = clk.summary()
     props = torch.cuda.get_device_properties(local)
     sm_mhz = float(clocks.get("sm_max_mhz") or 1965)
-    alu_tflops = 2.0 * props.multi_processor_count * 128 * sm_mhz * 1e6 / 1e12
+    derived_tflops = 2.0 * props.multi_processor_count * 128 * sm_mhz * 1e6 / 1e12
+    fma_per_clk, fma_tmacs = gdws.measure_fma_rate(gdws.FMA_F32)       # measured now, on this device
+    alu_tflops = 2.0 * fma_tmacs
     dw_macs = px * G * spec.k * spec.k
     t_alu = 2.0 * dw_macs / (alu_tflops * 1e12) * 1e6
     # Layer roofline: the slower of the Eq. 3 MACs at the tensor peak and the compulsory bytes at the copy bandwidth.
@@ -421,13 +458,14 @@ def run_ours(args, spec):
         achieved, peak, runit = nbytes / sec_per_step / 1e9, peaks["hbm_gbs"], "GB/s"
         psrc = peaks["source"] + " copy"
     roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
-            "traffic": TRAFFIC_BYTES_PER_LAUNCH.get((args.config, args.layer, args.path)) if (not f32 and args.dw_math != 2) else None,
+            "traffic": TRAFFIC_BYTES_PER_LAUNCH.get((args.config, args.layer, args.path, args.dw_math)) if not f32 else None,
             "peak_source": psrc,
             "kernel": ("fused_tc_kernel" if args.dw_math == 2 else "fused_bf16_kernel") if (not f32 and path != gdws.PATH_UNFUSED) else "see config.path",
             "layer_roofline_us": t_roof, "t_tensor_us": t_tensor, "t_hbm_us": t_hbm,
             "frac_of_layer_roofline": t_roof / us, "frac_of_layer_roofline_sustained_peak": t_roof_s / us,
             "gdw_on_alus": {"t_alu_us": t_alu, "peak_tflops": alu_tflops,
-                            "peak_source": "derived: SMs x 128 fp32 FMA lanes x max SM clock",
+                            "peak_source": "measured in this run: independent fp32 FMAs on all SMs (gdws_measure_fma_rate)",
+                            "fma_per_clk_per_sm": fma_per_clk, "derived_peak_tflops": derived_tflops,
                             "frac_of_max_tensor_hbm_alu": max(t_roof, t_alu) / us}}
 
     cpu_v, cpu_n, cpu_reps, cpu_dt, cores = oracle_throughput(spec, target_s=args.cpu_seconds)
@@ -454,7 +492,9 @@ def run_ours(args, spec):
             context["dense_conv"] = {"unavailable": repr(exc)[:200]}
 
     cfg = workload_config(spec, G)
-    cfg.update({"path": args.path, "gdw_stage": "tensor cores" if args.dw_math == 2 else "ALUs", "launch": "cuda graph replay" if graph is not None else "plain launches",
+    cfg.update({"path": args.path, "gdw_stage": "tensor cores" if args.dw_math == 2 else "ALUs", "launch": "cuda graph replay (every warm-up and timed launch is a graph node)" if graphs is not None else "plain launches",
+                "timing": {"repeats_of_the_k_step_region": repeats, "region_ms_median": ms, "region_ms_p10": percentile(region_ms, 0.1),
+                           "region_ms_p90": percentile(region_ms, 0.9), "timed_ms_total": float(sum(region_ms))},
                 "l2": f"rotating {nsets} input/output buffer sets ({nsets * set_bytes / 1e6:.0f} MB > 126 MB L2)"
                       if nsets > 1 else "one buffer set larger than L2",
                 "tile": "TNxPHxPW=%dx%dx%d" % plan.tile(spec.N, spec.H, spec.W)[:3] if not f32 else None,
@@ -473,6 +513,107 @@ def run_ours(args, spec):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------
+def run_chain(args):
+    """Config 3: the 16 chained 3x3 layers (ReLU between them), a step = the whole chain over the batch.
+    One CUDA graph holds the 16 launches; y of layer l is x of layer l+1.  The metric is end-to-end images/s,
+    the roofline the sum of the layers' rooflines."""
+    import torch
+
+    from paper_2110_14871_b200 import build as gbuild
+    from paper_2110_14871_b200 import gdws
+
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("--chain runs on one GPU")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(0)
+    gbuild.build_library()
+    peaks = load_peaks()
+    layers = gi.config_layers(3)
+    N = layers[0].N
+    gen = torch.Generator(device="cuda").manual_seed(3000)
+    acts = [torch.randn((N, layers[0].H, layers[0].W, layers[0].C), generator=gen, device="cuda").to(torch.bfloat16)]
+    plans, macs_total, roof_total, per_layer = [], 0, 0.0, []
+    for spec in layers:
+        rng = np.random.Generator(np.random.PCG64(spec.seed))
+        g = gi.make_g(rng, spec.C, spec.g_dist)
+        G = int(g.sum())
+        dw = torch.from_numpy(gi.round_to_bf16((rng.standard_normal((G, spec.k, spec.k)) / spec.k).astype(np.float32))).to(torch.bfloat16).cuda()
+        pw = torch.from_numpy(gi.round_to_bf16((rng.standard_normal((spec.D, G)) / np.sqrt(G)).astype(np.float32))).to(torch.bfloat16).cuda()
+        b = torch.from_numpy((rng.standard_normal(spec.D) * 0.1).astype(np.float32)).cuda()
+        plan = gdws.Plan(spec.C, spec.D, spec.k, spec.stride, spec.pad, g)
+        plan.set_option(gdws.OPT_RELU, int(spec.relu))
+        plan.set_option(gdws.OPT_PATH, gdws.PATH_FUSED)
+        plan.set_option(gdws.OPT_DW_MATH, args.dw_math)
+        plan.pack_weights(dw, pw, b)
+        plans.append(plan)
+        acts.append(torch.empty((N, spec.Ho, spec.Wo, spec.D), dtype=torch.bfloat16, device="cuda"))
+        _, macs, nbytes = layer_numbers(spec, G)
+        t_roof, _, _ = layer_roofline_us(macs, nbytes, peaks)
+        macs_total += macs
+        roof_total += t_roof
+        per_layer.append(t_roof)
+
+    def chain(stream):
+        for l, plan in enumerate(plans):
+            plan.forward(acts[l], acts[l + 1], "NHWC", stream=stream)
+
+    chain(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    for plan in plans:
+        plan.status()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = None
+    if not args.no_graph:
+        with torch.cuda.stream(side):
+            chain(side)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            chain(torch.cuda.current_stream())
+    steps = args.steps if args.steps != 20000 else 20
+
+    def run_region():
+        for _ in range(steps):
+            if graph is None:
+                chain(torch.cuda.current_stream())
+            else:
+                graph.replay()
+
+    for _ in range(3):
+        run_region()
+    torch.cuda.synchronize()
+    probe = timed_regions(run_region, 2)
+    repeats = choose_repeats(args, min(probe))
+    with ClockSampler(0) as clk:
+        region_ms = timed_regions(run_region, repeats)
+    ms = statistics.median(region_ms)
+    for plan in plans:
+        plan.status()
+    sec = ms / 1e3 / steps
+    out = {
+        "metric": "GDWS 16-layer chain end-to-end images/sec", "value": N / sec, "unit": UNIT, "n_gpus": 1, "steps": steps,
+        "warmup": 3 * steps, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"c3 chain: N={N}, 16 layers 64@32x32 ... 512@4x4, k=3, g~U[1,9], ReLU between layers, bf16 NHWC",
+                   "global_batch": N, "launch": "one cuda graph of the 16 launches" if graph is not None else "plain launches",
+                   "gdw_stage": "tensor cores" if args.dw_math == 2 else "ALUs",
+                   "l2": "each layer reads what the previous one wrote (0.03-67 MB per tensor, 126 MB L2), as a chained network does",
+                   "timing": {"repeats_of_the_k_step_region": repeats, "region_ms_p10": percentile(region_ms, 0.1),
+                              "region_ms_p90": percentile(region_ms, 0.9)}},
+        "effective_tmacs": macs_total / sec / 1e12,
+        "roofline": {"bound": "sum of the layers' rooflines", "layer_roofline_us_sum": roof_total, "frac_of_summed_layer_rooflines": roof_total / (sec * 1e6),
+                     "per_layer_roofline_us": per_layer, "peak_source": peaks["source"]},
+        "gpu_launches": len(plans) * steps * repeats, "clocks": clk.summary(),
+    }
+    print(json.dumps(out), flush=True)
+    for plan in plans:
+        plan.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -489,7 +630,14 @@ def main():
     ap.add_argument("--dw-math", type=int, default=0)
     ap.add_argument("--a-layout", type=int, default=0)
     ap.add_argument("--tile", type=int, default=0)
+    ap.add_argument("--repeats", type=int, default=0, help="repeats of the K-step timed region (0: choose)")
+    ap.add_argument("--chain", action="store_true", help="config 3: the 16 chained layers as one step")
     args = ap.parse_args()
+    if args.chain:
+        if args.config != 3 or args.impl != "ours":
+            raise SystemExit("--chain is the 16-layer chain of config 3 (our arm)")
+        run_chain(args)
+        return
     spec = gi.config_layers(args.config)[args.layer]
     if args.impl == "reference":
         if args.steps == 20000:

@@ -230,8 +230,11 @@ GDWS_API gdws_status_t gdws_forward_host(gdws_plan_t *plan, const gdws_tensor_t 
  *     GDWS_ERR_UNSUPPORTED (nothing is launched).
  *   - The plan must have been built with its device current (that is where the plan's own tables
  *     were allocated); otherwise GDWS_ERR_INVALID_ARG.
- *   - The first call on each device looks up the scratch array's device address
- *     (cudaGetSymbolAddress).  Make that first call outside any stream capture.
+ *   - The scratch array's device address is looked up once per device (cudaGetSymbolAddress): when
+ *     a plan sets up its tables on that device (gdws_plan with the device current), which is also
+ *     the moment the CUDA runtime may load the array's module and commit its 16 MiB there -- a
+ *     set-up cost of the allocating phase, not of this call.  Build the plan, and make the first
+ *     call on a device, outside any stream capture.
  *   - All calls on one GPU share the one array, whatever the plan or stream, and it keeps what the
  *     last call left there.  Nothing has to be cleared: each call overwrites every element of z that
  *     it reads.  Two calls whose kernels may overlap on the GPU (different streams) race on it:
@@ -250,6 +253,28 @@ GDWS_API size_t gdws_static_scratch_bytes(void);
  * (the kernel then skipped its remaining work; outputs of that launch are undefined).
  */
 GDWS_API gdws_status_t gdws_status(gdws_plan_t *plan);
+
+/*
+ * gdws_measure_fma_rate -- diagnostic: multiply-adds per clock and SM (and per second on the whole
+ * current device, in 1e12) that the plain ALUs sustain, measured with a kernel of independent
+ * register-to-register multiply-adds.  This is the bound of a GDW stage (Section 3.1, Definition:
+ * K*K multiply-adds per intermediate channel and output pixel) that runs on the ALUs.
+ *   kind  0: fma.rn.f32, 1: fma.rn.f32x2, 2: fma.rn.bf16x2, 3: fma.rn.f32.bf16 (bf16 factors, fp32 sum)
+ * Allocates a few KB on the current device, runs for a few milliseconds, synchronises.  Either output
+ * pointer may be NULL (HOST).  Errors: GDWS_ERR_INVALID_ARG, GDWS_ERR_ARCH, GDWS_ERR_CUDA.
+ */
+GDWS_API gdws_status_t gdws_measure_fma_rate(int kind, double *macs_per_clk_per_sm, double *tmacs_per_s);
+
+/*
+ * gdws_selftest_wait -- diagnostic of the error path behind GDWS_ERR_DEVICE_TIMEOUT: enqueues a
+ * one-block kernel in which one thread waits, with a limit of `polls` polls (at most 65536), on a
+ * shared-memory barrier that nothing ever completes.  The wait runs out, the thread records the
+ * condition in the plan's status word and raises the block's abort flag, which releases a second
+ * waiter; the kernel then returns by itself (it uses no copies and no tensor memory).  The next
+ * gdws_status(plan) reports GDWS_ERR_DEVICE_TIMEOUT once and clears the word.  (No counterpart in
+ * the paper.)  Errors: GDWS_ERR_INVALID_ARG, GDWS_ERR_ARCH, GDWS_ERR_CUDA.
+ */
+GDWS_API gdws_status_t gdws_selftest_wait(gdws_plan_t *plan, unsigned int polls, void *stream);
 
 /* Number of kernels this plan has launched so far (all entry points). */
 GDWS_API int64_t gdws_launch_count(const gdws_plan_t *plan);

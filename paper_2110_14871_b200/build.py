@@ -8,7 +8,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
-SOURCES = ["plan.cu", "f32.cu", "bf16.cu", "fused.cu", "fused_tc.cu", "api.cu", "static_ws.cu"]
+SOURCES = ["plan.cu", "f32.cu", "bf16.cu", "fused.cu", "fused_tc.cu", "api.cu", "static_ws.cu", "diag.cu"]
 HEADERS = [os.path.join(CSRC, "gdws_internal.h"), os.path.join(CSRC, "sm100.cuh"), os.path.join(_ROOT, "include", "gdws.h")]
 LIB_PATH = os.path.join(_HERE, "libgdws.so")
 

@@ -21,6 +21,10 @@ gdws_status_t check_tensor(const char *name, const gdws_tensor_t *t)
 
 size_t tensor_bytes(const gdws_tensor_t *t) { return (size_t)t->n * t->c * t->h * t->w * dtype_size(t->dtype); }
 
+}  // namespace
+
+namespace gdws {
+
 gdws_status_t check_pair(const gdws_plan_s *p, const gdws_tensor_t *x, const gdws_tensor_t *y)
 {
     gdws_status_t st = check_tensor("x", x);
@@ -43,6 +47,10 @@ gdws_status_t check_pair(const gdws_plan_s *p, const gdws_tensor_t *x, const gdw
         return fail(GDWS_ERR_INVALID_ARG, "x and y overlap");
     return GDWS_OK;
 }
+
+}  // namespace gdws
+
+namespace {
 
 gdws_status_t prepare(gdws_plan_s *p)
 {
@@ -212,15 +220,21 @@ gdws_status_t gdws_status(gdws_plan_t *p)
 {
     if (!p) return fail(GDWS_ERR_INVALID_ARG, "gdws_status: plan is NULL");
     if (p->device < 0) return GDWS_OK;
-    int word = 0;
-    cudaError_t e = cudaDeviceSynchronize();
-    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
-    e = cudaMemcpy(&word, p->d_status, sizeof(int), cudaMemcpyDeviceToHost);
-    if (e != cudaSuccess) return cuda_fail(e, "status read");
-    if (word) {
-        cudaMemset(p->d_status, 0, sizeof(int));
-        return fail(GDWS_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel expired (status word 0x%x)", word);
+    // the status word lives on the plan's device: wait for that device, whichever is current
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (cur != p->device) {
+        e = cudaSetDevice(p->device);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaSetDevice");
     }
+    int word = 0;
+    e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(&word, p->d_status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && word) e = cudaMemset(p->d_status, 0, sizeof(int));
+    if (cur != p->device) cudaSetDevice(cur);
+    if (e != cudaSuccess) return cuda_fail(e, "status read");
+    if (word) return fail(GDWS_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel expired (status word 0x%x)", word);
     return GDWS_OK;
 }
 

@@ -70,7 +70,7 @@ gdws_status_t bf16_pack(gdws_plan_s *p, const void *dw_w, const void *pw_w, cons
     const int k2 = p->k * p->k;
     const long long tot_pw = (long long)p->nchunks * p->Dpad * kChunk;
     int blocks = (int)((tot_pw + 255) / 256);
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > sm_count_of(p) * 8) blocks = sm_count_of(p) * 8;
     pack_pw_kernel<<<blocks, 256, 0, st>>>(pw_w, is_bf16, p->D, p->Dpad, p->G, p->nchunks, p->d_pw_img);
     int blocks2 = (p->Gpad * p->wstride + 255) / 256;
     pack_dw_kernel<<<blocks2, 256, 0, st>>>(dw_w, is_bf16, p->G, p->Gpad, k2, p->wstride, p->d_chan, p->d_chunk_meta,
@@ -147,7 +147,7 @@ gdws_status_t bf16_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cu
     s.Wo = gdws_out_dim(x->w, p->k, p->stride, p->pad);
     const long long total = (long long)s.N * s.Ho * s.Wo * (s.Gpad / 8);
     long long blocks = (total + 255) / 256;
-    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    if (blocks > (long long)sm_count_of(p) * 32) blocks = (long long)sm_count_of(p) * 32;
     gdw_bf16_kernel<<<(int)blocks, 256, 0, st>>>(s, (const uint16_t *)x->ptr, p->d_dw, p->d_chan, (uint16_t *)z);
     p->launches++;
     cudaError_t e = cudaGetLastError();
@@ -177,7 +177,7 @@ constexpr int kPwMaxStages = 8;
 __global__ void __launch_bounds__(kPwThreads, 1) pw_bf16_tc_kernel(const __grid_constant__ PwParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * kPwMaxStages + 4];   // full[8] free[8] acc_full[2] acc_free[2]
+    __shared__ __align__(8) uint64_t bars[2 * kPwMaxStages + 4 + 1];   // full[8] free[8] acc_full[2] acc_free[2] drain
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -185,12 +185,15 @@ __global__ void __launch_bounds__(kPwThreads, 1) pw_bf16_tc_kernel(const __grid_
     const uint32_t st_s = smem_u32(base);
     const uint32_t bar_full = smem_u32(&bars[0]), bar_free = smem_u32(&bars[kPwMaxStages]);
     const uint32_t bar_accfull = smem_u32(&bars[2 * kPwMaxStages]), bar_accfree = bar_accfull + 16;
+    const uint32_t bar_drain = bar_accfull + 32;
+    volatile int *const vabort = &abort_flag;
     const uint32_t b_bytes = (uint32_t)P.Dpad * kChunk * 2;
 
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < kPwMaxStages; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_free + 8 * i, 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4); }
+        mbar_init(bar_drain, 1);
         fence_mbar_init();
     }
     __syncwarp();
@@ -205,10 +208,12 @@ __global__ void __launch_bounds__(kPwThreads, 1) pw_bf16_tc_kernel(const __grid_
         if (lane == 0) {        // ---------------- loader ----------------
             uint32_t s = 0, par = 1;
             int it = 0;
-            for (int tl = 0; tl < my_tiles; ++tl) {
+            bool stop = false;
+            for (int tl = 0; tl < my_tiles && !stop; ++tl) {
                 const int row0 = ((int)blockIdx.x + tl * (int)gridDim.x) * kTileRows;
                 for (int q = 0; q < P.nchunks; ++q, ++it) {
                     if (it >= P.ns) mbar_wait(bar_free + 8 * s, par, &abort_flag, P.status, kStatusWaitStage);
+                    if (*vabort) { stop = true; break; }      // a wait ran out somewhere: no new copies
                     const uint32_t dst = st_s + s * (uint32_t)P.stage_bytes;
                     mbar_expect_tx(bar_full + 8 * s, 16384u + b_bytes);
                     tma_load_2d(dst, &P.tmap, q * kChunk, row0, bar_full + 8 * s);
@@ -216,6 +221,9 @@ __global__ void __launch_bounds__(kPwThreads, 1) pw_bf16_tc_kernel(const __grid_
                     if (++s == (uint32_t)P.ns) { s = 0; par ^= 1; }
                 }
             }
+            // Teardown: no copy into this block's shared memory may be in flight when it ends.  The last phase armed
+            // on each stage completes when its copies have landed.
+            for (int j = 0; j < P.ns && j < it; ++j) mbar_wait_drain(bar_full + 8 * j, (uint32_t)((it - 1 - j) / P.ns) & 1u);
         }
     } else if (warp == 1) {
         if (lane == 0) {        // ---------------- MMA issue ----------------
@@ -235,6 +243,9 @@ __global__ void __launch_bounds__(kPwThreads, 1) pw_bf16_tc_kernel(const __grid_
                 }
                 umma_commit(bar_accfull + 8 * buf);
             }
+            // Teardown: all issued products complete before the tensor memory is freed (bounded, ignores the abort flag).
+            umma_commit(bar_drain);
+            mbar_wait_drain(bar_drain, 0);
         }
     } else {
         // ---------------- epilogue warps ----------------

@@ -153,10 +153,10 @@ fused_f32_kernel(F32Shape s, const float *__restrict__ x, const float *__restric
     }
 }
 
-static int grid_for(long long total, int block)
+static int grid_for(const gdws_plan_s *p, long long total, int block)
 {
     long long b = (total + block - 1) / block;
-    const long long cap = 148LL * 16;
+    const long long cap = (long long)sm_count_of(p) * 16;
     return (int)(b < 1 ? 1 : (b > cap ? cap : b));
 }
 
@@ -164,7 +164,7 @@ gdws_status_t f32_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, const float 
 {
     const F32Shape s = make_shape(p, x->layout, x->n, x->h, x->w);
     const long long total = (long long)s.N * s.G * s.Ho * s.Wo;
-    gdw_f32_kernel<<<grid_for(total, 256), 256, 0, st>>>(s, (const float *)x->ptr, dw_w, p->d_chan, z);
+    gdw_f32_kernel<<<grid_for(p, total, 256), 256, 0, st>>>(s, (const float *)x->ptr, dw_w, p->d_chan, z);
     p->launches++;
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "gdw_f32_kernel launch");
@@ -184,7 +184,7 @@ gdws_status_t f32_pointwise(gdws_plan_s *p, const float *z, const float *pw_w, c
         s.yc = 1; s.yw = s.D; s.yh = (long long)s.Wo * s.D; s.yn = s.yh * s.Ho;
     }
     const long long total = (long long)s.N * s.D * s.Ho * s.Wo;
-    pw_f32_kernel<<<grid_for(total, 256), 256, 0, st>>>(s, z, pw_w, bias, (float *)y->ptr);
+    pw_f32_kernel<<<grid_for(p, total, 256), 256, 0, st>>>(s, z, pw_w, bias, (float *)y->ptr);
     p->launches++;
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "pw_f32_kernel launch");

@@ -102,12 +102,37 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
     asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
-// One bf16 element of the staged input as fp32.
-__device__ __forceinline__ float lds_bf16(uint32_t addr)
+// One bf16 element of the staged input, as loaded: the 16 bits sit in the low half of the register.
+__device__ __forceinline__ uint32_t lds_bf16(uint32_t addr)
 {
     uint32_t v;
     asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));
-    return __uint_as_float(v << 16);
+    return v;
+}
+// The depthwise multiply-add.  Filter taps are kept as fp32 words whose value is a bf16 (low half zero) and
+// inputs as loaded (bf16 in the low half): the mixed-precision FMA of sm_100 takes the two bf16 halves as they
+// are and accumulates in fp32 with one rounding, which is the fp32 FMA of the widened values without the
+// widening instruction (a shift per input on the 16-lane integer pipe, which holds the issue port for two
+// cycles: measured, a third of the depthwise warps' time).
+__device__ __forceinline__ float fma_bf(uint32_t w, uint32_t x, float acc)
+{
+    asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\t"
+        "mov.b32 {wl, wh}, %1;\n\t"
+        "mov.b32 {xl, xh}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, wh, xl, %0;\n\t}"
+        : "+f"(acc) : "r"(w), "r"(x));
+    return acc;
+}
+// The first tap starts the sum: w * x + 0.
+__device__ __forceinline__ float mul_bf(uint32_t w, uint32_t x)
+{
+    float r;
+    asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\t"
+        "mov.b32 {wl, wh}, %1;\n\t"
+        "mov.b32 {xl, xh}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, wh, xl, 0f00000000;\n\t}"
+        : "=f"(r) : "r"(w), "r"(x));
+    return r;
 }
 
 // Where the 8 bf16 results of pixel group `o` (rows 8o..8o+7 of the tile) and intermediate
@@ -193,7 +218,7 @@ __device__ __forceinline__ DwShare dw_rows_share(const FusedParams &P, int kk, i
     return sh;
 }
 template <int K, int S, int PS, bool KMAJOR>
-__device__ __forceinline__ void dw_rows(const DwShare &sh, uint32_t xs, int clb, const float (&w)[K * K], bool live_i,
+__device__ __forceinline__ void dw_rows(const DwShare &sh, uint32_t xs, int clb, const uint32_t (&w)[K * K], bool live_i,
                                         uint32_t a_stage)
 {
     float acc[4][8];
@@ -203,7 +228,7 @@ __device__ __forceinline__ void dw_rows(const DwShare &sh, uint32_t xs, int clb,
         constexpr int NX = 7 * S + K;
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
-            float xr[NX];
+            uint32_t xr[NX];
 #pragma unroll
             for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * sh.rowb + j * PS);
 #pragma unroll
@@ -213,9 +238,9 @@ __device__ __forceinline__ void dw_rows(const DwShare &sh, uint32_t xs, int clb,
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         // the first tap starts the sum
-                        float a = u == 0 ? w[0] * xr[e * S] : fmaf(w[u * K], xr[e * S], acc[ro][e]);
+                        float a = u == 0 ? mul_bf(w[0], xr[e * S]) : fma_bf(w[u * K], xr[e * S], acc[ro][e]);
 #pragma unroll
-                        for (int v = 1; v < K; ++v) a = fmaf(w[u * K + v], xr[e * S + v], a);
+                        for (int v = 1; v < K; ++v) a = fma_bf(w[u * K + v], xr[e * S + v], a);
                         acc[ro][e] = a;
                     }
                 }
@@ -251,7 +276,7 @@ __device__ __forceinline__ DwShare dw_quads_share(const FusedParams &P, int kk, 
     return sh;
 }
 template <int S, int PS, bool KMAJOR>
-__device__ __forceinline__ void dw_quads_k3(const DwShare &sh, uint32_t xs, int clb, const float (&w)[9], bool live_i,
+__device__ __forceinline__ void dw_quads_k3(const DwShare &sh, uint32_t xs, int clb, const uint32_t (&w)[9], bool live_i,
                                             uint32_t a_stage)
 {
 #pragma unroll
@@ -263,7 +288,7 @@ __device__ __forceinline__ void dw_quads_k3(const DwShare &sh, uint32_t xs, int 
             constexpr int NX = 3 * S + 3;           // input columns feeding 4 output columns
 #pragma unroll
             for (int r = 0; r < NR; ++r) {
-                float xr[NX];
+                uint32_t xr[NX];
 #pragma unroll
                 for (int j = 0; j < NX; ++j) xr[j] = lds_bf16(base + r * sh.rowb + j * PS);
 #pragma unroll
@@ -272,9 +297,9 @@ __device__ __forceinline__ void dw_quads_k3(const DwShare &sh, uint32_t xs, int 
                     if (u >= 0 && u < 3) {
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            float a = u == 0 ? w[0] * xr[e * S] : fmaf(w[u * 3], xr[e * S], acc[ro * 4 + e]);
-                            a = fmaf(w[u * 3 + 1], xr[e * S + 1], a);
-                            acc[ro * 4 + e] = fmaf(w[u * 3 + 2], xr[e * S + 2], a);
+                            float a = u == 0 ? mul_bf(w[0], xr[e * S]) : fma_bf(w[u * 3], xr[e * S], acc[ro * 4 + e]);
+                            a = fma_bf(w[u * 3 + 1], xr[e * S + 1], a);
+                            acc[ro * 4 + e] = fma_bf(w[u * 3 + 2], xr[e * S + 2], a);
                         }
                     }
                 }
@@ -315,8 +340,7 @@ __device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, in
                 for (int u = 0; u < K; ++u)
 #pragma unroll
                     for (int v = 0; v < K; ++v)
-                        acc = fmaf(__uint_as_float(lds32(wsm + (uint32_t)(u * K + v) * 4)),
-                                   lds_bf16(xp + (uint32_t)(u * P.IW + v) * P.ps), acc);
+                        acc = fma_bf(lds32(wsm + (uint32_t)(u * K + v) * 4), lds_bf16(xp + (uint32_t)(u * P.IW + v) * P.ps), acc);
                 out[e] = acc;
             }
         }
@@ -356,12 +380,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
 {
     constexpr bool ZOUT = VAR == 1, SPLIT = VAR == 2;
     extern __shared__ uint8_t smem_raw[];
-    // a_free[4] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2] | w_full[8] w_free[8] | open[4]
-    __shared__ __align__(8) uint64_t bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots + 4 + 2 * kMaxSlots + 4];
+    // a_free[4] | b_full[8] b_free[8] | x_full[8] x_free[8] | acc_full[2] acc_free[2] | w_full[8] w_free[8] | open[4] | drain
+    __shared__ __align__(8) uint64_t bars[4 + 2 * kMaxBUnits + 2 * kMaxSlots + 4 + 2 * kMaxSlots + 4 + 1];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ uint32_t xinfo[kMaxSlots];      // per filter-ring slot: input slot (bits 0-7) and phase parity (bit 8) of the chunk's box
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile int *const vabort = &abort_flag;
     // With few tiles, nsplit blocks share a tile: each does the whole depthwise stage and its share of the output channels.
     // (worked out where it is needed, not kept in registers through the depthwise loop)
 #define GDWS_BLOCK_SHARE                                                                                     \
@@ -381,6 +406,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const uint32_t bar_accfree = bar_accfull + 16;
     const uint32_t bar_wfull = bar_accfull + 32, bar_wfree = bar_wfull + 8 * kMaxSlots;
     const uint32_t bar_open = bar_wfree + 8 * kMaxSlots;       // a group's next chunk may start (two per group, alternating)
+    const uint32_t bar_drain = bar_open + 32;                  // the MMA warp's last commit, awaited before TMEM is freed
     const uint32_t wblock = (uint32_t)kChunk * P.wstride * 4;             // one chunk's filters
     const uint32_t w_s = x_s + (uint32_t)P.nslots * P.slot_bytes;         // ring of nwslots filter blocks
     int4 *meta_tab = reinterpret_cast<int4 *>(base + (w_s - a_s) + (size_t)P.nwslots * wblock);
@@ -395,6 +421,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             mbar_init(bar_accfull + 8 * i, 1);
             mbar_init(bar_accfree + 8 * i, kEpiWarps);
         }
+        mbar_init(bar_drain, 1);
         for (int i = 0; i < kMaxBUnits; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
         for (int i = 0; i < kMaxSlots; ++i) {
             mbar_init(bar_xfull + 8 * i, 1);
@@ -488,13 +515,24 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     __syncwarp();
                 }
             }
+            // Teardown: everything this warp issued has to be complete before the block frees its tensor memory
+            // and gives back its shared memory (after an abort the waits above return at once, and products may have
+            // been issued on operands that were not there: their results are undefined, but they too must have ended).
+            // One more commit covers all earlier products; its wait is bounded and does not look at the abort flag.
+            if (lane == 0) {
+                umma_commit(bar_drain);
+                mbar_wait_drain(bar_drain, 0);
+            }
+            __syncwarp();
         } else if (!ZOUT && warp == kCtrlWarp + 1 && lane == 0) {
             // ---------------- pointwise-weight loader (one thread): ring of nsb units ----------------
             GDWS_BLOCK_SHARE;
             uint32_t sb = 0, pb = 1;          // parity of the "slot free" phase awaited (first round: nothing to wait for)
-            int q = 0, h = 0;
+            int q = 0, h = 0, issued = 0;
             for (int u = 0; u < total_units; ++u) {
                 if (u >= P.nsb) mbar_wait_relaxed<kPollNs>(bar_bfree + 8 * sb, pb, &abort_flag, P.status, kStatusWaitStage);
+                if (*vabort) break;                    // a wait ran out somewhere: no new copies
+                ++issued;
                 const uint32_t bytes = (uint32_t)(h ? rows1 : rows0) * 128u;
                 mbar_expect_tx(bar_bfull + 8 * sb, bytes);
                 bulk_g2s(b_s + sb * P.unit_bytes, P.pw_img + ((size_t)q * P.Dpad_tot + part * P.Dpad + h * 256) * kChunk, bytes,
@@ -502,6 +540,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
                 if (++h == P.nhalf) { h = 0; if (++q == P.nchunks) q = 0; }
             }
+            // Teardown: the block's shared memory must not be given back while a copy into it is in flight.  The last
+            // phase armed on each ring slot completes when its copy has landed (earlier phases completed before it).
+            for (int j = 0; j < P.nsb && j < issued; ++j)
+                mbar_wait_drain(bar_bfull + 8 * j, (uint32_t)((issued - 1 - j) / P.nsb) & 1u);
         } else if (warp == kCtrlWarp + 2 && lane == 0) {
             // ---------------- input loader (one thread): ring of boxes, ring of filter blocks ----------------
             GDWS_BLOCK_SHARE;
@@ -509,7 +551,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             uint32_t wslot = 0, wpar = 1;
             uint32_t cur_x = 0;               // slot and "full" phase parity of the box the current chunks read
             int gq = 0, gb = 0;
-            for (int tl = 0; tl < my_tiles; ++tl) {
+            bool stop = false;
+            for (int tl = 0; tl < my_tiles && !stop; ++tl) {
                 int tile = bid + tl * nblocks;
                 const int bn = tile / tiles_hw;
                 tile -= bn * tiles_hw;
@@ -517,6 +560,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 const int n0 = bn * P.TN, hi0 = bh * P.PH * P.stride - P.pad, wi0 = bw * P.PW * P.stride - P.pad;
                 for (int q = 0; q < P.nchunks; ++q, ++gq) {
                     const int4 meta = meta_tab[q];
+                    if (*vabort) { stop = true; break; }        // a wait ran out somewhere: no new copies
                     if (meta.y & 4) {         // first chunk of a box: fetch the box
                         if (gb >= P.nslots) mbar_wait_relaxed<kPollNs>(bar_xfree + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitStage);
                         mbar_expect_tx(bar_xfull + 8 * xslot, (uint32_t)P.box_bytes);
@@ -532,6 +576,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     if (++wslot == (uint32_t)P.nwslots) { wslot = 0; wpar ^= 1; }
                 }
             }
+            // Teardown, as for the weight ring: gb boxes and gq filter blocks were requested.
+            for (int j = 0; j < P.nslots && j < gb; ++j)
+                mbar_wait_drain(bar_xfull + 8 * j, (uint32_t)((gb - 1 - j) / P.nslots) & 1u);
+            for (int j = 0; j < P.nwslots && j < gq; ++j)
+                mbar_wait_drain(bar_wfull + 8 * j, (uint32_t)((gq - 1 - j) / P.nwslots) & 1u);
         } else if (warp == kCtrlWarp + 3) {
             // ---------------- gate warp ----------------
             // Waits, chunk by chunk, until the chunk's filters and input box have landed and its operand stage
@@ -671,7 +720,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             const uint32_t xslot = xinfo[wslot] & 0xffu;
             const uint32_t xs = x_s + xslot * (uint32_t)P.slot_bytes;
             const uint32_t wsm = w_s + wslot * wblock + (uint32_t)(il * P.wstride) * 4;   // this thread's filter
-            float w[K * K];
+            uint32_t w[K * K];                            // taps: fp32 words holding bf16 values
             int clb;                                      // channel index inside the staged box
             if (MODE != 0) {
                 constexpr int NV = (K * K + 4) / 4;       // 16-byte pieces holding the taps and the channel index
@@ -682,13 +731,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     wv[4 * j] = t.x; wv[4 * j + 1] = t.y; wv[4 * j + 2] = t.z; wv[4 * j + 3] = t.w;
                 }
 #pragma unroll
-                for (int j = 0; j < K * K; ++j) w[j] = __uint_as_float(wv[j]);
+                for (int j = 0; j < K * K; ++j) w[j] = wv[j];
                 clb = (int)wv[K * K];
             } else {
                 clb = (int)lds32(wsm + (uint32_t)(K * K) * 4);
             }
             if (MODE == 1) dw_rows<K, S, PS, ZOUT>(share, xs, clb, w, live_i, a_stage);
-            else if (MODE == 2) dw_quads_k3<S, PS, ZOUT>(share, xs, clb, reinterpret_cast<const float (&)[9]>(w), live_i, a_stage);
+            else if (MODE == 2) dw_quads_k3<S, PS, ZOUT>(share, xs, clb, reinterpret_cast<const uint32_t (&)[9]>(w), live_i, a_stage);
             else dw_generic<K>(P, xs, clb, wsm, il, run, live_i, a_stage);
             fence_proxy_async();      // every thread: its own writes become visible to the tensor-core proxy
             __syncwarp();

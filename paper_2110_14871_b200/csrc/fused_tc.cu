@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
 {
     extern __shared__ uint8_t smem_raw[];
     // dwready[4] | zfull[2] (2 unused) | pwready[4] pwdone[4] | bfree[4] xfree[4] | accfull[2] accfree[2]
-    __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4];
+    __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4 + 1];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -123,6 +123,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const uint32_t bar_pwready = bar_zfull + 32, bar_pwdone = bar_pwready + 8 * kTcNU;
     const uint32_t bar_bfree = bar_pwdone + 8 * kTcNU, bar_xfree = bar_bfree + 8 * kTcMaxNB;
     const uint32_t bar_accfull = bar_xfree + 8 * kTcMaxNX, bar_accfree = bar_accfull + 16;
+    const uint32_t bar_drain = bar_accfull + 32;       // the issue warp's last commit, awaited before TMEM is freed
+    volatile int *const vabort = &abort_flag;
     TcChunk *tab = reinterpret_cast<TcChunk *>(base + P.off_tab);
     float *bias_sm = reinterpret_cast<float *>(tab + P.nchunks);
     uint16_t *bold = reinterpret_cast<uint16_t *>(bias_sm + P.Dpad_tot);     // [nb][128]: what each builder thread wrote last
@@ -138,6 +140,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         for (int i = 0; i < kTcNU; ++i) { mbar_init(bar_pwready + 8 * i, kTcConvWarps + 1); mbar_init(bar_pwdone + 8 * i, 1); }
         for (int i = 0; i < kTcMaxNB; ++i) mbar_init(bar_bfree + 8 * i, 1);
         for (int i = 0; i < kTcMaxNX; ++i) mbar_init(bar_xfree + 8 * i, 1);
+        mbar_init(bar_drain, 1);
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512u);
@@ -245,12 +248,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 }
             }
         }
+        // Teardown: one more commit covers every product issued before it (after an abort, products may have been issued
+        // on operands that were not there; they must have ended all the same); its wait is bounded and ignores the abort flag.
+        if (lane == 0) {
+            umma_commit(bar_drain);
+            mbar_wait_drain(bar_drain, 0);
+        }
+        __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------- input loader ----------------
             int box = 0, u = 0;
             uint32_t xslot = 0;
-            for (int it = 0; it < my_items; ++it) {
+            bool stop = false;
+            for (int it = 0; it < my_items && !stop; ++it) {
                 const int item = (int)blockIdx.x + it * (int)gridDim.x;
                 int tile = item / P.nparts;
                 const int bn = tile / tiles_hw;
@@ -262,6 +273,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     const uint32_t bar = bar_dwready + 8 * (u & 3);
                     // this barrier's last phase (chunk u - 4) must be complete before anything counts towards chunk u
                     if (u >= 4) tc_wait(bar, (uint32_t)((u >> 2) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                    if (*vabort) { stop = true; break; }       // a wait ran out somewhere: no new copies
                     if (!(flags & 1)) { mbar_arrive(bar); continue; }
                     if (box >= P.nx)
                         tc_wait(bar_xfree + 8 * xslot, (uint32_t)((box / P.nx) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
@@ -273,13 +285,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     if (++xslot == (uint32_t)P.nx) xslot = 0;
                 }
             }
+            // Teardown: no box copy may be in flight when the block ends.  This thread arrived for units 0 .. u-1; the
+            // last phase of each of the four barriers completes once its box (if any) has landed and the builder warps
+            // have arrived, and the phases before it completed earlier (bounded wait).
+            for (int j = 0; j < 4 && j < u; ++j) {
+                const int v = u - 1 - j;
+                mbar_wait_drain(bar_dwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u);
+            }
         }
     } else if (warp == 2) {
         if (lane == 0) {
             // ---------------- pointwise-weight loader ----------------
             SlabRing ring;
             ring.free_slabs = P.nw;
-            int q = 0, it = 0;
+            int q = 0, it = 0, issued = 0;
             for (int v = 0; v < total; ++v) {
                 const TcChunk ch = tab[q];
                 const int ns = ch.npad >> 4;
@@ -289,6 +308,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     ring.free_slabs += tab[o % P.nchunks].npad >> 4;
                     ++ring.oldest;
                 }
+                if (*vabort) break;                            // a wait ran out somewhere: no new copies
+                issued = v + 1;
                 const int part = ((int)blockIdx.x + it * (int)gridDim.x) % P.nparts;
                 const uint32_t bar = bar_pwready + 8 * (v & 3);
                 mbar_expect_tx(bar, (uint32_t)ns * P.wslab_bytes);
@@ -299,6 +320,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 ring.head = (ring.head + ns) % P.nw;
                 ring.free_slabs -= ns;
                 if (++q == P.nchunks) { q = 0; ++it; }
+            }
+            // Teardown: the last phase armed on each pwready barrier completes when its weights have landed and the
+            // converter warps have arrived (bounded wait).
+            for (int j = 0; j < kTcNU && j < issued; ++j) {
+                const int v = issued - 1 - j;
+                mbar_wait_drain(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u);
             }
         }
     } else if (warp >= 4 && warp < 4 + kTcConvWarps) {

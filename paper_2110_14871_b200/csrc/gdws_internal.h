@@ -123,9 +123,17 @@ gdws_status_t fail(gdws_status_t st, const char *fmt, ...);
 gdws_status_t cuda_fail(cudaError_t e, const char *what);
 gdws_status_t ensure_device(gdws_plan_s *p);   // allocate device tables on the current device
 gdws_status_t check_arch();
+// x and y of a forward call against the plan: pointers, alignment, extents, dtype/layout pair, no overlap
+gdws_status_t check_pair(const gdws_plan_s *p, const gdws_tensor_t *x, const gdws_tensor_t *y);
+// static_ws.cu: looks up (once per device, the device being current) the address of the built-in scratch array
+gdws_status_t static_scratch_prepare(int device);
 bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *t);
 
 inline size_t dtype_size(gdws_dtype_t d) { return d == GDWS_F32 ? 4 : 2; }
+
+// SMs of the plan's device; a plan built without a device (host-side queries only) assumes a B200's 148.
+constexpr int kB200Sms = 148;
+inline int sm_count_of(const gdws_plan_s *p) { return p->sm_count > 0 ? p->sm_count : kB200Sms; }
 
 // f32.cu
 gdws_status_t f32_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, const float *dw_w, float *z, cudaStream_t s);

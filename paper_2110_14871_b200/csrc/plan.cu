@@ -55,20 +55,24 @@ static void free_device(gdws_plan_s *p)
     cudaGetDevice(&cur);
     cudaSetDevice(p->device);
     cudaDeviceSynchronize();
-    cudaFree(p->d_off);
-    cudaFree(p->d_chan);
-    cudaFree(p->d_chunk_meta);
-    cudaFree(p->d_dw);
-    cudaFree(p->d_dwpack);
-    cudaFree(p->d_pw_img);
-    cudaFree(p->d_bias);
-    cudaFree(p->d_status);
-    cudaFree(p->d_tc_chunks);
-    cudaFree(p->d_tc_filt);
-    cudaFree(p->d_tc_pw);
-    p->d_tc_chunks = nullptr; p->d_tc_filt = nullptr; p->d_tc_pw = nullptr;
-    cudaFree(p->stage_x);
-    cudaFree(p->stage_y);
+    // every pointer is cleared as it is freed: a plan that outlives a failed set-up is set up again from scratch
+    auto release = [](auto *&ptr) { cudaFree(ptr); ptr = nullptr; };
+    release(p->d_off);
+    release(p->d_chan);
+    release(p->d_chunk_meta);
+    release(p->d_dw);
+    release(p->d_dwpack);
+    release(p->d_pw_img);
+    release(p->d_bias);
+    release(p->d_status);
+    release(p->d_tc_chunks);
+    release(p->d_tc_filt);
+    release(p->d_tc_pw);
+    release(p->stage_x);
+    release(p->stage_y);
+    p->stage_x_bytes = 0;
+    p->stage_y_bytes = 0;
+    p->packed = false;
     cudaSetDevice(cur);
     p->device = -1;
 }
@@ -106,6 +110,7 @@ gdws_status_t ensure_device(gdws_plan_s *p)
     }
 #undef GDWS_TRY_ALLOC
     p->device = dev;
+    if (cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) p->sm_count = 0;
     e = cudaMemcpy(p->d_off, p->off.data(), sizeof(int32_t) * (p->C + 1), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_chan, p->chan.data(), sizeof(int32_t) * p->Gpad, cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
@@ -118,6 +123,9 @@ gdws_status_t ensure_device(gdws_plan_s *p)
         free_device(p);
         return cuda_fail(e, "plan table upload");
     }
+    // The built-in scratch array of gdws_forward_static is part of a module that the first look-up of its
+    // address may load (committing its 16 MiB on this device): do that here, where allocation is expected.
+    static_scratch_prepare(dev);
     return GDWS_OK;
 }
 
@@ -203,7 +211,7 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *out)
     if (n < 1 || Ho < 1 || Wo < 1) return false;
     const int cbox = p->cbox;
     if (cbox <= 0) return false;            // some chunk reads more than 128 channels: no fused kernel
-    const int sms = p->sm_count > 0 ? p->sm_count : 148;
+    const int sms = sm_count_of(p);
     double best = 1e300;
     bool found = false;
     const int forced = p->opt_tile;

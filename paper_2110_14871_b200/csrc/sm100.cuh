@@ -60,17 +60,22 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // (barriers stay matched, TMEM is freed) and the kernel ends.  The first few thousand polls
 // are back to back (waits in the pipeline are short and a sleeping waiter wakes up late).
 constexpr uint32_t kSpinLimit = 1u << 22;
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+__device__ __forceinline__ void mbar_wait_limited(uint32_t bar, uint32_t parity, uint32_t limit, volatile int *abort_flag,
+                                                  int *status, int code)
 {
     if (mbar_try_wait(bar, parity)) return;           // the common case costs one shared-memory round trip
     if (*abort_flag) return;
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return;
         if (it > 4096) __nanosleep(64);
         if ((it & 1023) == 1023 && *abort_flag) return;
     }
     *abort_flag = 1;
     atomicOr(status, code);
+}
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+{
+    mbar_wait_limited(bar, parity, kSpinLimit, abort_flag, status, code);
 }
 // The same for waiters that run ahead of the pipeline (loaders, the gate warp, epilogue warps): each poll
 // lets the hardware suspend the thread for up to SUSPEND_NS or until the phase completes, so that polling

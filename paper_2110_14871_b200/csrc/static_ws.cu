@@ -1,6 +1,8 @@
 // gdws_forward_static: the unfused forward (GDW kernel -> z -> PW kernel) for callers that must not
 // allocate device memory.  The intermediate z lives in a fixed array that is part of the library
 // image, so nothing is asked of the CUDA allocator, neither here nor by the caller.
+#include <mutex>
+
 #include "gdws_internal.h"
 
 using namespace gdws;
@@ -11,25 +13,32 @@ static __device__ __align__(256) unsigned char g_static_scratch[GDWS_STATIC_SCRA
 namespace {
 
 // In host code `g_static_scratch` is only a handle of the symbol, not a device address; the address
-// a kernel can use has to be looked up, once per device, with that device current.
+// a kernel can use has to be looked up, once per device, with that device current.  The table is
+// shared by all host threads, hence the lock.
 void *g_scratch_addr[64] = {};
+std::mutex g_scratch_lock;
 
 gdws_status_t scratch_address(int device, void **out)
 {
     if (device < 0 || device >= 64) return fail(GDWS_ERR_UNSUPPORTED, "device index %d is outside 0..63", device);
+    std::lock_guard<std::mutex> hold(g_scratch_lock);
     if (!g_scratch_addr[device]) {
         void *ptr = nullptr;
         cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
         if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static scratch)");
         g_scratch_addr[device] = ptr;
     }
-    *out = g_scratch_addr[device];
+    if (out) *out = g_scratch_addr[device];
     return GDWS_OK;
 }
 
 bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
 
 }  // namespace
+
+// Called while a plan sets up its device tables, i.e. in the phase that allocates anyway: this translation
+// unit holds no kernel, so its module (and with it the array) may only be loaded by this first look-up.
+gdws_status_t gdws::static_scratch_prepare(int device) { return scratch_address(device, nullptr); }
 
 extern "C" {
 
@@ -38,18 +47,10 @@ size_t gdws_static_scratch_bytes(void) { return (size_t)GDWS_STATIC_SCRATCH_BYTE
 gdws_status_t gdws_forward_static(gdws_plan_t *p, const gdws_tensor_t *x, const void *dw_w, const void *pw_w,
                                   const float *bias, gdws_tensor_t *y, void *stream)
 {
-    if (!p || !x || !y) return fail(GDWS_ERR_INVALID_ARG, "gdws_forward_static: NULL argument");
-    if (!x->ptr || !y->ptr || !aligned16(x->ptr) || !aligned16(y->ptr))
-        return fail(GDWS_ERR_INVALID_ARG, "gdws_forward_static: tensor pointers must be non-NULL and 16-byte aligned");
-    if (x->n < 1 || x->h < 1 || x->w < 1 || x->c != p->C || y->c != p->D || y->n != x->n)
-        return fail(GDWS_ERR_INVALID_ARG, "gdws_forward_static: tensor extents do not match the plan");
-    if (x->dtype != y->dtype || x->layout != y->layout || (x->dtype != GDWS_F32 && x->dtype != GDWS_BF16) ||
-        (x->layout != GDWS_NCHW && x->layout != GDWS_NHWC))
-        return fail(GDWS_ERR_INVALID_ARG, "gdws_forward_static: x and y must share a valid dtype and layout");
-    const int Ho = gdws_out_dim(x->h, p->k, p->stride, p->pad), Wo = gdws_out_dim(x->w, p->k, p->stride, p->pad);
-    if (Ho < 1 || Wo < 1 || y->h != Ho || y->w != Wo)
-        return fail(GDWS_ERR_INVALID_ARG, "gdws_forward_static: y must be %dx%d for this input", Ho, Wo);
-    if (x->dtype == GDWS_BF16 && x->layout != GDWS_NHWC) return fail(GDWS_ERR_UNSUPPORTED, "bf16 tensors must be NHWC");
+    if (!p) return fail(GDWS_ERR_INVALID_ARG, "gdws_forward_static: plan is NULL");
+    gdws_status_t st = check_pair(p, x, y);      // the checks of gdws_forward, overlap of x and y included
+    if (st != GDWS_OK) return st;
+    if (bias && ((uintptr_t)bias & 3)) return fail(GDWS_ERR_INVALID_ARG, "gdws_forward_static: bias must be 4-byte aligned");
     if (x->dtype == GDWS_BF16 && (p->C % 8 || p->D % 8)) return fail(GDWS_ERR_UNSUPPORTED, "bf16 kernels need C %% 8 == 0 and D %% 8 == 0");
     // The plan's own tables were allocated when it was built on a device; this call never allocates.
     if (p->device < 0)
@@ -59,7 +60,7 @@ gdws_status_t gdws_forward_static(gdws_plan_t *p, const gdws_tensor_t *x, const 
     if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
     if (dev != p->device) return fail(GDWS_ERR_INVALID_ARG, "plan lives on device %d but device %d is current", p->device, dev);
     if (!p->arch_ok) {
-        gdws_status_t st = check_arch();
+        st = check_arch();
         if (st != GDWS_OK) return st;
         p->arch_ok = true;
     }
@@ -69,7 +70,7 @@ gdws_status_t gdws_forward_static(gdws_plan_t *p, const gdws_tensor_t *x, const 
                     "gdws_forward_static: the intermediate needs %zu bytes, the built-in scratch holds %zu; use gdws_forward",
                     need, (size_t)GDWS_STATIC_SCRATCH_BYTES);
     void *z = nullptr;
-    gdws_status_t st = scratch_address(dev, &z);
+    st = scratch_address(dev, &z);
     if (st != GDWS_OK) return st;
     cudaStream_t cs = (cudaStream_t)stream;
     if (x->dtype == GDWS_F32) {

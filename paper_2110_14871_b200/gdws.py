@@ -28,6 +28,7 @@ EXPORTS = [
     "gdws_out_dim", "gdws_pack_weights", "gdws_workspace_bytes", "gdws_set_workspace", "gdws_forward",
     "gdws_depthwise", "gdws_pointwise", "gdws_forward_host", "gdws_status", "gdws_launch_count",
     "gdws_last_error", "gdws_version", "gdws_destroy", "gdws_forward_static", "gdws_static_scratch_bytes",
+    "gdws_measure_fma_rate", "gdws_selftest_wait",
 ]
 
 
@@ -93,6 +94,10 @@ def lib() -> ctypes.CDLL:
     L.gdws_static_scratch_bytes.restype = ctypes.c_size_t
     L.gdws_status.argtypes = [vp]
     L.gdws_status.restype = ci
+    L.gdws_measure_fma_rate.argtypes = [ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    L.gdws_measure_fma_rate.restype = ci
+    L.gdws_selftest_wait.argtypes = [vp, ctypes.c_uint, vp]
+    L.gdws_selftest_wait.restype = ci
     L.gdws_launch_count.argtypes = [vp]
     L.gdws_launch_count.restype = i64
     L.gdws_last_error.argtypes = []
@@ -115,6 +120,16 @@ def version() -> str:
 
 def static_scratch_bytes() -> int:
     return int(lib().gdws_static_scratch_bytes())
+
+
+FMA_F32, FMA_F32X2, FMA_BF16X2, FMA_F32_BF16 = range(4)
+
+
+def measure_fma_rate(kind: int = FMA_F32) -> Tuple[float, float]:
+    """gdws_measure_fma_rate: (multiply-adds per clock and SM, 1e12 multiply-adds per second on the device)."""
+    per_clk, tmacs = ctypes.c_double(), ctypes.c_double()
+    _check(lib().gdws_measure_fma_rate(kind, ctypes.byref(per_clk), ctypes.byref(tmacs)))
+    return per_clk.value, tmacs.value
 
 
 def out_dim(size: int, k: int, stride: int, pad: int) -> int:
@@ -260,3 +275,7 @@ class Plan:
 
     def status(self) -> None:
         _check(lib().gdws_status(self._h))
+
+    def selftest_wait(self, polls: int = 64, stream=None) -> None:
+        """gdws_selftest_wait: a bounded wait that runs out; the next status() raises GDWS_ERR_DEVICE_TIMEOUT once."""
+        _check(lib().gdws_selftest_wait(self._h, polls, _stream(stream)))

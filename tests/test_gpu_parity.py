@@ -249,3 +249,37 @@ def test_forward_host_matches_device_forward():
     ref, _ = run_oracle(data)
     assert rel_err(yh.float().numpy(), ref) <= TOL["bf16"]
     plan.destroy()
+
+
+# ------------------------------------------------------------------ diagnostics
+def test_bounded_wait_reports_once_and_plan_stays_usable():
+    """A wait that nothing satisfies runs out after its poll limit: the kernel returns by itself, the
+    status word reports the time-out once, and the same plan then runs a normal forward."""
+    spec = small_spec("t", 2, 16, 16, 8, 8, 3, 1, 1, ("uniform", 1, 9), "bf16", "NHWC", seed=81)
+    data = gi.make_layer(spec)
+    plan = make_plan(data, path=gdws.PATH_FUSED)
+    plan.status()
+    plan.selftest_wait(polls=32)
+    torch.cuda.synchronize()
+    with pytest.raises(gdws.GdwsError) as e:
+        plan.status()
+    assert e.value.status == gdws.ERR_DEVICE_TIMEOUT
+    plan.status()                                   # cleared by the report
+    x, dw, pw = (to_device(a, "bf16") for a in (data.x, data.dw_w, data.pw_w))
+    b = torch.from_numpy(data.bias).cuda()
+    y = torch.full((spec.N, spec.Ho, spec.Wo, spec.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    plan.forward(x, y, "NHWC", dw, pw, b)
+    torch.cuda.synchronize()
+    plan.status()
+    ref, _ = run_oracle(data)
+    assert rel_err(y.float().cpu().numpy().astype(np.float64), ref) <= TOL["bf16"]
+    plan.destroy()
+
+
+def test_fma_rate_measurement_is_plausible():
+    """The ALU multiply-add rate that bench.py reports as the bound of a GDW stage on the ALUs: between
+    half and all of the 128 fp32 lanes of an SM, and the packed forms no faster in multiply-adds."""
+    per_clk, tmacs = gdws.measure_fma_rate(gdws.FMA_F32)
+    assert 64.0 <= per_clk <= 130.0 and tmacs > 5.0
+    per_clk2, _ = gdws.measure_fma_rate(gdws.FMA_F32X2)
+    assert 64.0 <= per_clk2 <= 135.0

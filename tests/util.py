@@ -23,6 +23,32 @@ def rel_err(y: np.ndarray, ref: np.ndarray) -> float:
     return float(np.max(np.abs(y.astype(np.float64) - ref)) / max(np.max(np.abs(ref)), 1e-30))
 
 
+GUARD_BYTES = 4096
+_SENTINEL = 0x5A
+
+
+class Guarded:
+    """A device tensor of `shape` carved out of a larger byte buffer, with GUARD_BYTES of a sentinel
+    before and after it.  check() fails if a kernel wrote outside the tensor (the role a memory checker
+    would play)."""
+
+    def __init__(self, shape, dtype, fill=None):
+        n = int(np.prod(shape))
+        esz = torch.empty((), dtype=dtype).element_size()
+        body = (n * esz + 255) // 256 * 256
+        self.raw = torch.full((GUARD_BYTES + body + GUARD_BYTES,), _SENTINEL, dtype=torch.uint8, device="cuda")
+        self.t = self.raw[GUARD_BYTES:GUARD_BYTES + n * esz].view(dtype).view(shape)
+        self._tail = GUARD_BYTES + n * esz
+        if fill is not None:
+            self.t.fill_(fill)
+
+    def check(self, what="buffer"):
+        before = self.raw[:GUARD_BYTES]
+        after = self.raw[self._tail:]
+        assert bool((before == _SENTINEL).all()), f"bytes before {what} were overwritten"
+        assert bool((after == _SENTINEL).all()), f"bytes after {what} were overwritten"
+
+
 def make_plan(data: gi.LayerData, path=gdws.PATH_AUTO, a_layout=0, dw_math=0, tile=0) -> gdws.Plan:
     s = data.spec
     plan = gdws.Plan(s.C, s.D, s.k, s.stride, s.pad, data.g)
@@ -45,12 +71,14 @@ def run_gpu(data: gi.LayerData, path=gdws.PATH_AUTO, a_layout=0, dw_math=0, tile
     b = torch.from_numpy(data.bias).cuda()
     tdt = torch.float32 if s.dtype == "f32" else torch.bfloat16
     shape = (s.N, s.D, s.Ho, s.Wo) if s.layout == "NCHW" else (s.N, s.Ho, s.Wo, s.D)
-    y = torch.full(shape, float("nan"), dtype=tdt, device="cuda") if poison else torch.empty(shape, dtype=tdt, device="cuda")
+    yg = Guarded(shape, tdt, fill=float("nan") if poison else 0.0)
+    y = yg.t
     code = gdws.F32 if s.dtype == "f32" else gdws.BF16
+    wsg = None
     if path == gdws.PATH_UNFUSED:
         nbytes = plan.workspace_bytes(code, s.N, s.H, s.W)
-        ws = torch.full((nbytes // 2 + 128,), -1, dtype=torch.int16, device="cuda")
-        plan.set_workspace(ws)
+        wsg = Guarded((nbytes,), torch.uint8, fill=0xFF)
+        plan.set_workspace(wsg.t)
     if prepack and s.dtype == "bf16":
         plan.pack_weights(dw, pw, b)
         plan.forward(x, y, s.layout)
@@ -58,6 +86,9 @@ def run_gpu(data: gi.LayerData, path=gdws.PATH_AUTO, a_layout=0, dw_math=0, tile
         plan.forward(x, y, s.layout, dw, pw, b)
     torch.cuda.synchronize()
     plan.status()
+    yg.check("y")
+    if wsg is not None:
+        wsg.check("the workspace")
     out = y.float().cpu().numpy().astype(np.float64)
     plan.destroy()
     return out
