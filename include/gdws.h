@@ -266,6 +266,15 @@ GDWS_API gdws_status_t gdws_status(gdws_plan_t *plan);
 GDWS_API gdws_status_t gdws_measure_fma_rate(int kind, double *macs_per_clk_per_sm, double *tmacs_per_s);
 
 /*
+ * gdws_measure_code_size -- diagnostic: instructions per clock and warp scheduler that `threads` threads per SM
+ * (128, 256 or 512) sustain on independent fp32 multiply-adds in a loop whose body is `body_instructions` long
+ * (64, 128, 160, 256, 512 or 1024; 16 bytes each).  Bodies beyond about 2 KB no longer fit the instruction cache
+ * next to a scheduler; the rate then is that of instruction fetch.  This sizes the kernels' hot loops.  (No
+ * counterpart in the paper.)  Allocates a few KB, runs for about a millisecond, synchronises.
+ */
+GDWS_API gdws_status_t gdws_measure_code_size(int body_instructions, int threads, double *instructions_per_clk_per_scheduler);
+
+/*
  * gdws_selftest_wait -- diagnostic of the error path behind GDWS_ERR_DEVICE_TIMEOUT: enqueues a
  * one-block kernel in which one thread waits, with a limit of `polls` polls (at most 65536), on a
  * shared-memory barrier that nothing ever completes.  The wait runs out, the thread records the

@@ -53,6 +53,36 @@ __global__ void __launch_bounds__(1024, 1) fma_rate_kernel(float *sink, long lon
     if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
 }
 
+// The same independent fp32 multiply-adds with a loop body of BODY instructions (16 bytes each): shows where straight-line
+// code stops fitting the instruction cache next to a scheduler and runs at the speed of instruction fetch instead.
+template <int BODY>
+__global__ void __launch_bounds__(512, 1) code_size_kernel(float *sink, long long *cycles, int total_fma, float seed)
+{
+    float a[32], w[9], x[10];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) a[i] = seed * (float)i;
+#pragma unroll
+    for (int i = 0; i < 9; ++i) w[i] = seed + (float)i + (float)threadIdx.x;
+#pragma unroll
+    for (int i = 0; i < 10; ++i) x[i] = seed * 3.f + (float)i + (float)threadIdx.x;
+    __syncthreads();
+    const int iters = total_fma / BODY;
+    const long long t0 = clock64();
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int b = 0; b < BODY / 32; ++b)
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(a[i]) : "f"(w[b % 9]), "f"(x[(i + b) % 10]));
+    }
+    const long long t1 = clock64();
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) s += a[i];
+    if (s == 123.456f) sink[threadIdx.x] = s;
+    if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
+}
+
 // One block; nothing ever arrives at its mbarrier.  Lane 0 of warp 0 waits with the given poll limit, runs out,
 // records the code and raises the abort flag; lane 0 of warp 1 waits with the library's normal limit and is
 // released by that flag.  No copies, no tensor memory: the kernel returns by itself.
@@ -126,6 +156,53 @@ gdws_status_t gdws_measure_fma_rate(int kind, double *macs_per_clk_per_sm, doubl
     const double macs_sm = (double)iters * kRateBody * kRateAcc * threads * per_instr;
     if (macs_per_clk_per_sm) *macs_per_clk_per_sm = worst > 0 ? macs_sm / (double)worst : 0.0;
     if (tmacs_per_s) *tmacs_per_s = ms > 0.f ? macs_sm * sms / (ms * 1e-3) / 1e12 : 0.0;
+    return GDWS_OK;
+}
+
+gdws_status_t gdws_measure_code_size(int body_instructions, int threads, double *instructions_per_clk_per_scheduler)
+{
+    if (threads != 128 && threads != 256 && threads != 512)
+        return fail(GDWS_ERR_INVALID_ARG, "gdws_measure_code_size: threads must be 128, 256 or 512");
+    gdws_status_t st = check_arch();
+    if (st != GDWS_OK) return st;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "device query");
+    float *sink = nullptr;
+    long long *cyc = nullptr;
+    e = cudaMalloc((void **)&sink, 4096);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&cyc, sizeof(long long) * (size_t)sms);
+    if (e != cudaSuccess) { cudaFree(sink); return cuda_fail(e, "cudaMalloc"); }
+    const int total = 1 << 19;
+    bool known = true;
+    for (int pass = 0; pass < 2 && known; ++pass) {
+        const int n = pass == 0 ? 1 << 14 : total;
+        switch (body_instructions) {
+        case 64: code_size_kernel<64><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 128: code_size_kernel<128><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 160: code_size_kernel<160><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 256: code_size_kernel<256><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 512: code_size_kernel<512><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 1024: code_size_kernel<1024><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        default: known = false; break;
+        }
+    }
+    long long worst = 0;
+    if (known) {
+        e = cudaDeviceSynchronize();
+        if (e == cudaSuccess) {
+            std::vector<long long> h((size_t)sms);
+            e = cudaMemcpy(h.data(), cyc, sizeof(long long) * (size_t)sms, cudaMemcpyDeviceToHost);
+            for (long long c : h) worst = c > worst ? c : worst;
+        }
+    }
+    cudaFree(sink);
+    cudaFree(cyc);
+    if (!known) return fail(GDWS_ERR_INVALID_ARG, "gdws_measure_code_size: body must be 64, 128, 160, 256, 512 or 1024 instructions");
+    if (e != cudaSuccess) return cuda_fail(e, "gdws_measure_code_size");
+    if (instructions_per_clk_per_scheduler)
+        *instructions_per_clk_per_scheduler = worst > 0 ? (double)total * (threads / 32) / 4.0 / (double)worst : 0.0;
     return GDWS_OK;
 }
 

@@ -478,12 +478,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 const int buf = tl % P.nacc;
                 const uint32_t d_tmem = tmem + (uint32_t)(buf * P.acc_cols);
                 if (tl >= P.nacc)
-                    mbar_wait(bar_accfree + 8 * buf, ((tl / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                    mbar_wait_call(bar_accfree + 8 * buf, ((tl / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
                 for (int q = 0; q < P.nchunks; ++q, ++gq) {
                     // chunk gq is the (gq >> 1)-th chunk of group gq & 1, which cycles through its own stages
                     const uint32_t sa = ((gq & 1u) << P.spg_shift) + ((gq >> 1) & spg_mask);
                     const uint32_t a_lo = a_lo0 + sa * (16384u >> 4);
-                    mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);   // long there
+                    mbar_wait_call(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);   // long there
                     named_bar_sync(kBarChunk0 + (int)(gq & 3u), kDwGroupWarps * 32 + 32);   // the group has written chunk gq
                     tc_fence_after();
                     if (elect_one()) {
@@ -496,7 +496,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     }
                     if (++sb == (uint32_t)P.nsb) { sb = 0; pb ^= 1; }
                     if (P.nhalf == 2) {       // output channels 256 and up: a second weight unit, a second set of columns
-                        mbar_wait(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
+                        mbar_wait_call(bar_bfull + 8 * sb, pb, &abort_flag, P.status, kStatusWaitOperand);
                         tc_fence_after();
                         if (elect_one()) {
                             const uint32_t b_lo = b_lo0 + sb * b_unit;
@@ -530,7 +530,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             uint32_t sb = 0, pb = 1;          // parity of the "slot free" phase awaited (first round: nothing to wait for)
             int q = 0, h = 0, issued = 0;
             for (int u = 0; u < total_units; ++u) {
-                if (u >= P.nsb) mbar_wait_relaxed<kPollNs>(bar_bfree + 8 * sb, pb, &abort_flag, P.status, kStatusWaitStage);
+                if (u >= P.nsb) mbar_wait_relaxed_call<kPollNs>(bar_bfree + 8 * sb, pb, &abort_flag, P.status, kStatusWaitStage);
                 if (*vabort) break;                    // a wait ran out somewhere: no new copies
                 ++issued;
                 const uint32_t bytes = (uint32_t)(h ? rows1 : rows0) * 128u;
@@ -562,14 +562,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     const int4 meta = meta_tab[q];
                     if (*vabort) { stop = true; break; }        // a wait ran out somewhere: no new copies
                     if (meta.y & 4) {         // first chunk of a box: fetch the box
-                        if (gb >= P.nslots) mbar_wait_relaxed<kPollNs>(bar_xfree + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitStage);
+                        if (gb >= P.nslots) mbar_wait_relaxed_call<kPollNs>(bar_xfree + 8 * xslot, xpar, &abort_flag, P.status, kStatusWaitStage);
                         mbar_expect_tx(bar_xfull + 8 * xslot, (uint32_t)P.box_bytes);
                         tma_load_4d(x_s + xslot * (uint32_t)P.slot_bytes, &P.tmap, meta.z, wi0, hi0, n0, bar_xfull + 8 * xslot);
                         cur_x = xslot | ((xpar ^ 1u) << 8);   // "full" phase parity = the opposite of the "free" parity awaited
                         ++gb;
                         if (++xslot == (uint32_t)P.nslots) { xslot = 0; xpar ^= 1; }
                     }
-                    if (gq >= P.nwslots) mbar_wait_relaxed<kPollNs>(bar_wfree + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitStage);
+                    if (gq >= P.nwslots) mbar_wait_relaxed_call<kPollNs>(bar_wfree + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitStage);
                     xinfo[wslot] = cur_x;                     // published by the arrive below
                     mbar_expect_tx(bar_wfull + 8 * wslot, wblock);
                     bulk_g2s(w_s + wslot * wblock, P.dwpack + (size_t)q * kChunk * P.wstride, wblock, bar_wfull + 8 * wslot);
@@ -595,15 +595,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 for (int q = 0; q < P.nchunks; ++q, ++gq) {
                     const int flags = meta_tab[q].y;
                     const int g = gq & 1, k = gq >> 1;
-                    mbar_wait_relaxed<kPollNs>(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
+                    mbar_wait_relaxed_call<kPollNs>(bar_wfull + 8 * wslot, wpar, &abort_flag, P.status, kStatusWaitOperand);
                     if (flags & 4) {
                         xs_cur = xs_next; xp_cur = xp_next;
                         if (++xs_next == (uint32_t)P.nslots) { xs_next = 0; xp_next ^= 1; }
-                        mbar_wait_relaxed<kPollNs>(bar_xfull + 8 * xs_cur, xp_cur, &abort_flag, P.status, kStatusWaitOperand);
+                        mbar_wait_relaxed_call<kPollNs>(bar_xfull + 8 * xs_cur, xp_cur, &abort_flag, P.status, kStatusWaitOperand);
                     }
                     if ((k >> P.spg_shift) >= 1) {
                         const uint32_t sa = ((uint32_t)g << P.spg_shift) + ((uint32_t)k & ((1u << P.spg_shift) - 1u));
-                        mbar_wait_relaxed<kPollNs>(bar_afree + 8 * sa, ((k >> P.spg_shift) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                        mbar_wait_relaxed_call<kPollNs>(bar_afree + 8 * sa, ((k >> P.spg_shift) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
                     }
                     if (lane == 0) mbar_arrive(bar_open + 8 * (2 * g + (k & 1)));
                     __syncwarp();

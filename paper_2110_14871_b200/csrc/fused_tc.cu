@@ -184,64 +184,64 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         const uint32_t z_lo0 = ((z_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t w_lo0 = ((w_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t wstep = P.wslab_bytes >> 4;
-        uint32_t xslot = 0, bslot = 0;
-        uint32_t zhead = 0, whead = 0, buf = 0, accpar = 1;
+        // The loop below is this warp's whole working set of instructions and is kept near a hundred of them (it has to
+        // stay in the small instruction cache next to the scheduler while the other warps of the block come and go):
+        // tap offsets live in registers, ring positions advance by a compare per slab, waits are calls when they miss.
+        uint32_t tap_a[K * K], tap_b[K * K];
+#pragma unroll
+        for (int ur = 0; ur < K; ++ur)
+#pragma unroll
+            for (int v = 0; v < K; ++v) {
+                tap_a[ur * K + v] = (uint32_t)ur * rstep + (uint32_t)v * cstep;
+                tap_b[ur * K + v] = (uint32_t)(ur * K + v) * pstep;
+            }
+        uint32_t xslot = 0, bslot = 0, a_lo = a_lo0, b_lo = b_lo0;
+        uint32_t zh = 0, wh = 0, z_lo = z_lo0, w_lo = w_lo0, buf = 0, accpar = 1;
         int q = 0;                  // chunk index of unit u within its work item
         int qp = 0, itp = 0;        // the same for unit u - 1, and its work item
         for (int u = 0; u <= total; ++u) {
             if (u < total) {
                 const int npad = tab[q].npad, flags = tab[q].flags;
-                mbar_wait(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
+                mbar_wait_call(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
                 tc_fence_after();
                 if (elect_one()) {
                     const uint32_t idesc = make_idesc(npad, false);
                     const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
-                    const uint32_t a_lo = a_lo0 + xslot * xstep, b_lo = b_lo0 + bslot * bstep;
 #pragma unroll
-                    for (int ur = 0; ur < K; ++ur)
-#pragma unroll
-                        for (int v = 0; v < K; ++v)
-                            umma_bf16_words(d_z, a_lo + (uint32_t)ur * rstep + (uint32_t)v * cstep, a_hi,
-                                            b_lo + (uint32_t)(ur * K + v) * pstep, p_hi, idesc, (ur | v) != 0);
+                    for (int i = 0; i < K * K; ++i)
+                        umma_bf16_words(d_z, a_lo + tap_a[i], a_hi, b_lo + tap_b[i], p_hi, idesc, i != 0);
                     umma_commit(bar_zfull + 8 * (u & 1));
                 }
                 __syncwarp();
-                if (++bslot == (uint32_t)P.nb) bslot = 0;
-                if (flags & 2) { if (++xslot == (uint32_t)P.nx) xslot = 0; }
+                b_lo += bstep;
+                if (++bslot == (uint32_t)P.nb) { bslot = 0; b_lo = b_lo0; }
+                if (flags & 2) {
+                    a_lo += xstep;
+                    if (++xslot == (uint32_t)P.nx) { xslot = 0; a_lo = a_lo0; }
+                }
                 if (++q == P.nchunks) q = 0;
             }
             if (u > 0) {
                 const int v = u - 1;
                 const int ns = tab[qp].npad >> 4;
-                if (qp == 0 && itp >= P.nacc) mbar_wait(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
-                mbar_wait(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
+                if (qp == 0 && itp >= P.nacc) mbar_wait_call(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
+                mbar_wait_call(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
                 tc_fence_after();
-                if (elect_one()) {
-                    const uint32_t d_y = tmem + buf * 128u;
-                    if (zhead + (uint32_t)ns <= (uint32_t)P.nz && whead + (uint32_t)ns <= (uint32_t)P.nw) {
-                        const uint32_t z_lo = z_lo0 + zhead * (kTcSlab >> 4), w_lo = w_lo0 + whead * wstep;
-#pragma unroll
-                        for (int s = 0; s < 8; ++s)      // a chunk has at most 8 slabs (128 intermediate channels)
-                            if (s < ns)
-                                umma_bf16_words(d_y, z_lo + (uint32_t)s * (kTcSlab >> 4), p_hi, w_lo + (uint32_t)s * wstep, p_hi,
-                                                idesc_pw, (qp | s) != 0);
-                    } else {                              // the chunk wraps around the end of a ring
-                        uint32_t zh = zhead, wh = whead;
+                const bool leader = elect_one();
+                const uint32_t d_y = tmem + buf * 128u;
 #pragma unroll 1
-                        for (int s = 0; s < ns; ++s) {
-                            umma_bf16_words(d_y, z_lo0 + zh * (kTcSlab >> 4), p_hi, w_lo0 + wh * wstep, p_hi, idesc_pw, (qp | s) != 0);
-                            if (++zh == (uint32_t)P.nz) zh = 0;
-                            if (++wh == (uint32_t)P.nw) wh = 0;
-                        }
-                    }
+                for (int s = 0; s < ns; ++s) {           // every lane keeps the ring positions, the leader issues
+                    if (leader) umma_bf16_words(d_y, z_lo, p_hi, w_lo, p_hi, idesc_pw, (uint32_t)(qp | s));
+                    z_lo += kTcSlab >> 4;
+                    if (++zh == (uint32_t)P.nz) { zh = 0; z_lo = z_lo0; }
+                    w_lo += wstep;
+                    if (++wh == (uint32_t)P.nw) { wh = 0; w_lo = w_lo0; }
+                }
+                if (leader) {
                     umma_commit(bar_pwdone + 8 * (v & 3));
                     if (qp == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
                 }
                 __syncwarp();
-                zhead += (uint32_t)ns;
-                if (zhead >= (uint32_t)P.nz) zhead -= (uint32_t)P.nz;
-                whead += (uint32_t)ns;
-                if (whead >= (uint32_t)P.nw) whead -= (uint32_t)P.nw;
                 if (++qp == P.nchunks) {
                     qp = 0; ++itp;
                     if (++buf == (uint32_t)P.nacc) { buf = 0; accpar ^= 1; }

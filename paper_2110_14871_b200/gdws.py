@@ -28,7 +28,7 @@ EXPORTS = [
     "gdws_out_dim", "gdws_pack_weights", "gdws_workspace_bytes", "gdws_set_workspace", "gdws_forward",
     "gdws_depthwise", "gdws_pointwise", "gdws_forward_host", "gdws_status", "gdws_launch_count",
     "gdws_last_error", "gdws_version", "gdws_destroy", "gdws_forward_static", "gdws_static_scratch_bytes",
-    "gdws_measure_fma_rate", "gdws_selftest_wait",
+    "gdws_measure_fma_rate", "gdws_measure_code_size", "gdws_selftest_wait",
 ]
 
 
@@ -96,6 +96,8 @@ def lib() -> ctypes.CDLL:
     L.gdws_status.restype = ci
     L.gdws_measure_fma_rate.argtypes = [ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     L.gdws_measure_fma_rate.restype = ci
+    L.gdws_measure_code_size.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_double)]
+    L.gdws_measure_code_size.restype = ci
     L.gdws_selftest_wait.argtypes = [vp, ctypes.c_uint, vp]
     L.gdws_selftest_wait.restype = ci
     L.gdws_launch_count.argtypes = [vp]
@@ -130,6 +132,13 @@ def measure_fma_rate(kind: int = FMA_F32) -> Tuple[float, float]:
     per_clk, tmacs = ctypes.c_double(), ctypes.c_double()
     _check(lib().gdws_measure_fma_rate(kind, ctypes.byref(per_clk), ctypes.byref(tmacs)))
     return per_clk.value, tmacs.value
+
+
+def measure_code_size(body_instructions: int, threads: int = 512) -> float:
+    """gdws_measure_code_size: instructions per clock and scheduler for a loop body of that many instructions."""
+    ipc = ctypes.c_double()
+    _check(lib().gdws_measure_code_size(body_instructions, threads, ctypes.byref(ipc)))
+    return ipc.value
 
 
 def out_dim(size: int, k: int, stride: int, pad: int) -> int:

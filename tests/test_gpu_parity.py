@@ -283,3 +283,11 @@ def test_fma_rate_measurement_is_plausible():
     assert 64.0 <= per_clk <= 130.0 and tmacs > 5.0
     per_clk2, _ = gdws.measure_fma_rate(gdws.FMA_F32X2)
     assert 64.0 <= per_clk2 <= 135.0
+
+
+def test_code_size_cliff_is_where_the_kernels_assume_it():
+    """Loops of 2 KB run from the instruction cache next to a scheduler, loops of 4 KB and more at the speed of
+    instruction fetch: the sizing rule behind the kernels' hot loops."""
+    small = gdws.measure_code_size(128, 512)
+    large = gdws.measure_code_size(1024, 512)
+    assert small > 0.7 and large < 0.65 * small, (small, large)
