@@ -90,6 +90,12 @@ __device__ __forceinline__ void tc_warp_wait(uint32_t bar, uint32_t parity, vola
     if ((threadIdx.x & 31) == 0) tc_wait(bar, parity, abort_flag, status, code);
     __syncwarp();
 }
+// The same with the polling loop as a call: for the warps whose per-chunk code has to stay small.
+__device__ __forceinline__ void tc_warp_wait_call(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+{
+    if ((threadIdx.x & 31) == 0 && !mbar_try_wait(bar, parity)) mbar_wait_relaxed_slow(bar, parity, 16384u, abort_flag, status, code);
+    __syncwarp();
+}
 __device__ __forceinline__ void tc_warp_arrive(uint32_t bar)
 {
     __syncwarp();
@@ -333,21 +339,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         // Two warps per TMEM lane quarter; each takes every other 16-column granule of the chunk (at most 4), reads
         // them with one wait, rounds and stores them.  Warp 4's first lane also releases, on behalf of the GDW issue
         // warp, the B buffer and (after a window's last chunk) the input box that the chunk's products have read.
+        // The per-chunk code is a short loop over pairs of granules (it shares the scheduler's small instruction cache
+        // with the issue, builder and epilogue code of the same quarter), and its waits are calls when they miss.
         const int lg = warp & 3, half = (warp - 4) >> 2;
         const uint32_t r = (uint32_t)(lg * 32 + lane);
+        const uint32_t sw = ((r >> 2) & 1u) << 4;           // 32-byte swizzle: address bit 4 ^= bit 7
+        const uint32_t row_s = z_s + r * 32u;
         SlabRing ring;
         ring.free_slabs = P.nz;
         uint32_t bslot = 0, xslot = 0;
-        int q = 0;
+        int q = 0, qo = 0;                                   // chunk index of unit v and of the ring's oldest unit
         for (int v = 0; v < total; ++v) {
             const int ns = tab[q].npad >> 4, flags = tab[q].flags;
             while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
                 const int o = ring.oldest;
-                tc_warp_wait(bar_pwdone + 8 * (o & 3), (uint32_t)(o >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
-                ring.free_slabs += tab[o % P.nchunks].npad >> 4;
+                tc_warp_wait_call(bar_pwdone + 8 * (o & 3), (uint32_t)(o >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                ring.free_slabs += tab[qo].npad >> 4;
+                if (++qo == P.nchunks) qo = 0;
                 ++ring.oldest;
             }
-            tc_warp_wait(bar_zfull + 8 * (v & 1), (uint32_t)(v >> 1) & 1u, &abort_flag, P.status, kStatusWaitMma);
+            tc_warp_wait_call(bar_zfull + 8 * (v & 1), (uint32_t)(v >> 1) & 1u, &abort_flag, P.status, kStatusWaitMma);
             if (warp == 4 && lane == 0) {
                 mbar_arrive(bar_bfree + 8 * bslot);
                 if (flags & 2) mbar_arrive(bar_xfree + 8 * xslot);
@@ -356,36 +367,38 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             if (flags & 2) { if (++xslot == (uint32_t)P.nx) xslot = 0; }
             tc_fence_after();
             const uint32_t taddr = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(kTcZCol + 128 * (v & 1));
-            uint32_t acc[4][16];
+#pragma unroll 1
+            for (int g = half; g < ns; g += 4) {             // this warp's granules g and g + 2 with one wait
+                uint32_t acc[2][16];
+                const bool two = g + 2 < ns;
+                tmem_ld16(taddr + (uint32_t)(g * 16), acc[0]);
+                if (two) tmem_ld16(taddr + (uint32_t)((g + 2) * 16), acc[1]);
+                tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (2 * j + half < ns) tmem_ld16(taddr + (uint32_t)((2 * j + half) * 16), acc[j]);
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int g = 2 * j + half;
-                if (g < ns) {
-                    uint4 lo, hi;
-                    lo.x = pack_bf16x2(__uint_as_float(acc[j][0]), __uint_as_float(acc[j][1]));
-                    lo.y = pack_bf16x2(__uint_as_float(acc[j][2]), __uint_as_float(acc[j][3]));
-                    lo.z = pack_bf16x2(__uint_as_float(acc[j][4]), __uint_as_float(acc[j][5]));
-                    lo.w = pack_bf16x2(__uint_as_float(acc[j][6]), __uint_as_float(acc[j][7]));
-                    hi.x = pack_bf16x2(__uint_as_float(acc[j][8]), __uint_as_float(acc[j][9]));
-                    hi.y = pack_bf16x2(__uint_as_float(acc[j][10]), __uint_as_float(acc[j][11]));
-                    hi.z = pack_bf16x2(__uint_as_float(acc[j][12]), __uint_as_float(acc[j][13]));
-                    hi.w = pack_bf16x2(__uint_as_float(acc[j][14]), __uint_as_float(acc[j][15]));
-                    int slab = ring.head + g;
-                    if (slab >= P.nz) slab -= P.nz;
-                    const uint32_t addr = z_s + (uint32_t)slab * kTcSlab + r * 32u;
-                    const uint32_t sw = ((r >> 2) & 1u) << 4;   // 32-byte swizzle: address bit 4 ^= bit 7
-                    sts128(addr + sw, lo);                 // channels 0 .. 7 of the slab for this pixel
-                    sts128(addr + (sw ^ 16u), hi);         // channels 8 .. 15
+                for (int j = 0; j < 2; ++j) {
+                    if (j == 0 || two) {
+                        uint4 lo, hi;
+                        lo.x = pack_bf16x2(__uint_as_float(acc[j][0]), __uint_as_float(acc[j][1]));
+                        lo.y = pack_bf16x2(__uint_as_float(acc[j][2]), __uint_as_float(acc[j][3]));
+                        lo.z = pack_bf16x2(__uint_as_float(acc[j][4]), __uint_as_float(acc[j][5]));
+                        lo.w = pack_bf16x2(__uint_as_float(acc[j][6]), __uint_as_float(acc[j][7]));
+                        hi.x = pack_bf16x2(__uint_as_float(acc[j][8]), __uint_as_float(acc[j][9]));
+                        hi.y = pack_bf16x2(__uint_as_float(acc[j][10]), __uint_as_float(acc[j][11]));
+                        hi.z = pack_bf16x2(__uint_as_float(acc[j][12]), __uint_as_float(acc[j][13]));
+                        hi.w = pack_bf16x2(__uint_as_float(acc[j][14]), __uint_as_float(acc[j][15]));
+                        int slab = ring.head + g + 2 * j;
+                        if (slab >= P.nz) slab -= P.nz;
+                        const uint32_t addr = row_s + (uint32_t)slab * kTcSlab;
+                        sts128(addr + sw, lo);                 // channels 0 .. 7 of the slab for this pixel
+                        sts128(addr + (sw ^ 16u), hi);         // channels 8 .. 15
+                    }
                 }
             }
             fence_proxy_async();
             tc_fence_before();
             tc_warp_arrive(bar_pwready + 8 * (v & 3));
-            ring.head = (ring.head + ns) % P.nz;
+            ring.head += ns;
+            if (ring.head >= P.nz) ring.head -= P.nz;
             ring.free_slabs -= ns;
             if (++q == P.nchunks) q = 0;
         }
@@ -485,7 +498,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             }
         };
         if (total > 0) load_rec(tab[0], nxt);
-        uint32_t bslot = 0;
+        uint32_t bslot = 0, bpar = 0;      // B buffer of unit v, and the parity of the "free" phase it waits for
         int q = 0;
         for (int v = 0; v < total; ++v) {
 #pragma unroll
@@ -495,12 +508,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             const uint32_t cw = rec[0] & 0xFFFFu;
             const bool valid = cw != 0xFFFFu;
             const uint32_t off = rowoff + ((((cw >> 3) & 1u) ^ rowsw) << 4) + (cw & 7u) * 2u;
-            if (v >= P.nb) tc_warp_wait(bar_bfree + 8 * bslot, (uint32_t)((v / P.nb) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+            if (v >= P.nb) tc_warp_wait_call(bar_bfree + 8 * bslot, bpar, &abort_flag, P.status, kStatusWaitStage);
             const uint32_t bb = b_s + bslot * P.bbuf_bytes;
             const uint32_t old = bold[bslot * 128 + t];
             if (old != 0xFFFFu) {
-#pragma unroll
-                for (int j = 0; j < K * K; ++j) sts16(bb + (uint32_t)j * P.bplane + old, (uint16_t)0);
+                uint32_t a = bb + old;
+#pragma unroll 1
+                for (int j = 0; j < K * K; ++j, a += P.bplane) sts16(a, (uint16_t)0);
             }
             if (valid) {
 #pragma unroll
@@ -510,7 +524,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             bold[bslot * 128 + t] = (uint16_t)(valid ? off : 0xFFFFu);
             fence_proxy_async();
             tc_warp_arrive(bar_dwready + 8 * (v & 3));
-            if (++bslot == (uint32_t)P.nb) bslot = 0;
+            if (++bslot == (uint32_t)P.nb) { bslot = 0; if (v >= P.nb) bpar ^= 1u; }
         }
     }
     tc_fence_before();
@@ -633,8 +647,8 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     TcParams P;
     memset(&P, 0, sizeof(P));
     const int Dloc = p->tc_dloc, m = p->tc_maxslabs;
-    const uint32_t nmax = (uint32_t)tc_nmax(k, Dloc);
-    P.bplane = nmax * 32u; P.bbuf_bytes = (uint32_t)(k * k) * P.bplane;
+    // a B operand plane holds one 32-byte row per intermediate channel of the layer's largest chunk
+    P.bplane = (uint32_t)m * 16u * 32u; P.bbuf_bytes = (uint32_t)(k * k) * P.bplane;
     P.wslab_bytes = (uint32_t)Dloc * 32u;
     P.xslot_bytes = (uint32_t)((g.xbox + 255) / 256 * 256);
     // Shared memory: output staging (optional) | B operand buffers | z slabs | weight slabs | input boxes | tables
@@ -645,14 +659,17 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     for (int ost = can_stage ? 1 : 0; ost >= 0; --ost)
         for (int nx = 3; nx >= 2; --nx)
             for (int nb = 3; nb >= 2; --nb)
-                for (int nz = 2 * m; nz >= m; --nz) {
+                for (int nz = 3 * m; nz >= m; --nz) {
                     const size_t fixed = 1024 + (ost ? 16384 : 0) + (size_t)nb * P.bbuf_bytes + (size_t)nz * kTcSlab +
                                          (size_t)nx * P.xslot_bytes + tables;
                     if (fixed + (size_t)m * P.wslab_bytes > (size_t)kMaxSmem) continue;
                     int nw = (int)(((size_t)kMaxSmem - fixed) / P.wslab_bytes);
                     if (nw > 3 * m) nw = 3 * m;
-                    const double score = 2.0 * std::min(nw, 2 * m) / m + 0.3 * std::min(nw, 3 * m) / m + 1.5 * nz / m + 0.4 * ost +
-                                         0.25 * nx + 0.15 * nb;
+                    // First two chunks of z slabs (the converter writes one while the PW products of the one before are
+                    // pending: with less, conversion and PW products of consecutive chunks serialise -- seen in a cycle
+                    // trace), then two chunks of weights, then the rest.
+                    const double score = 10.0 * std::min(nz, 2 * m) / m + 6.0 * std::min(nw, 2 * m) / m + 1.0 * std::min(nw, 3 * m) / m +
+                                         0.5 * nz / m + 0.8 * ost + 0.6 * nb + 0.3 * nx;
                     if (score > best_score) { best_score = score; b_ost = ost; b_nx = nx; b_nb = nb; b_nz = nz; b_nw = nw; }
                 }
     if (best_score < 0) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: shared memory does not fit this layer");
