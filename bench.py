@@ -458,9 +458,9 @@ def run_ours(args, spec):
         achieved, peak, runit = nbytes / sec_per_step / 1e9, peaks["hbm_gbs"], "GB/s"
         psrc = peaks["source"] + " copy"
     roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
-            "traffic": TRAFFIC_BYTES_PER_LAUNCH.get((args.config, args.layer, args.path, args.dw_math)) if not f32 else None,
+            "traffic": TRAFFIC_BYTES_PER_LAUNCH.get((args.config, args.layer, args.path, plan.gdw_stage())) if not f32 else None,
             "peak_source": psrc,
-            "kernel": ("fused_tc_kernel" if args.dw_math == 2 else "fused_bf16_kernel") if (not f32 and path != gdws.PATH_UNFUSED) else "see config.path",
+            "kernel": ("fused_tc_kernel" if plan.gdw_stage() == 2 else "fused_bf16_kernel") if (not f32 and path != gdws.PATH_UNFUSED) else "see config.path",
             "layer_roofline_us": t_roof, "t_tensor_us": t_tensor, "t_hbm_us": t_hbm,
             "frac_of_layer_roofline": t_roof / us, "frac_of_layer_roofline_sustained_peak": t_roof_s / us,
             "gdw_on_alus": {"t_alu_us": t_alu, "peak_tflops": alu_tflops,
@@ -492,7 +492,7 @@ def run_ours(args, spec):
             context["dense_conv"] = {"unavailable": repr(exc)[:200]}
 
     cfg = workload_config(spec, G)
-    cfg.update({"path": args.path, "gdw_stage": "tensor cores" if args.dw_math == 2 else "ALUs", "launch": "cuda graph replay (every warm-up and timed launch is a graph node)" if graphs is not None else "plain launches",
+    cfg.update({"path": args.path, "gdw_stage": ("tensor cores" if plan.gdw_stage() == 2 else "ALUs") + (" (chosen by the library)" if args.dw_math == 0 else " (forced)"), "launch": "cuda graph replay (every warm-up and timed launch is a graph node)" if graphs is not None else "plain launches",
                 "timing": {"repeats_of_the_k_step_region": repeats, "region_ms_median": ms, "region_ms_p10": percentile(region_ms, 0.1),
                            "region_ms_p90": percentile(region_ms, 0.9), "timed_ms_total": float(sum(region_ms))},
                 "l2": f"rotating {nsets} input/output buffer sets ({nsets * set_bytes / 1e6:.0f} MB > 126 MB L2)"
@@ -600,7 +600,7 @@ def run_chain(args):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"c3 chain: N={N}, 16 layers 64@32x32 ... 512@4x4, k=3, g~U[1,9], ReLU between layers, bf16 NHWC",
                    "global_batch": N, "launch": "one cuda graph of the 16 launches" if graph is not None else "plain launches",
-                   "gdw_stage": "tensor cores" if args.dw_math == 2 else "ALUs",
+                   "gdw_stage": {1: "ALUs (forced)", 2: "tensor cores (forced)"}.get(args.dw_math, "chosen per layer by the library: " + "".join("T" if pl.gdw_stage() == 2 else "A" for pl in plans)),
                    "l2": "each layer reads what the previous one wrote (0.03-67 MB per tensor, 126 MB L2), as a chained network does",
                    "timing": {"repeats_of_the_k_step_region": repeats, "region_ms_p10": percentile(region_ms, 0.1),
                               "region_ms_p90": percentile(region_ms, 0.9)}},

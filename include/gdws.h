@@ -80,12 +80,12 @@ typedef enum {
     GDWS_OPT_A_LAYOUT = 3, /* bf16 fused path, shared-memory layout of the intermediate
                               tile handed to the tensor cores: 0 = pixel-contiguous
                               (default), 1 = channel-contiguous                            */
-    GDWS_OPT_DW_MATH = 4   /* bf16 fused path, where the GDW stage runs: 0 (default) or 1 = on the
-                              ALUs (fp32 FMAs); 2 = on the tensor cores as k*k block-sparse
+    GDWS_OPT_DW_MATH = 4   /* bf16 fused path, where the GDW stage runs: 1 = on the ALUs (fp32
+                              multiply-adds); 2 = on the tensor cores as k*k block-sparse
                               products per 16-channel window (fp32 accumulation), for stride 1
-                              and k <= 5, else GDWS_ERR_UNSUPPORTED.  Both give the same
-                              result up to summation order; 2 is slower on the benchmark
-                              layers and is kept as a measured alternative                 */
+                              and k <= 5, else GDWS_ERR_UNSUPPORTED; 0 (default) = the library
+                              chooses (see gdws_plan_gdw_stage).  Both give the same result
+                              up to summation order                                         */
 } gdws_option_t;
 
 typedef enum {
@@ -144,6 +144,16 @@ GDWS_API gdws_status_t gdws_plan_tile(const gdws_plan_t *plan, int n, int h, int
 
 /* Output extent H' (or W') for input extent `in`: floor((in + 2 pad - k)/stride) + 1, 0 if negative. */
 GDWS_API int gdws_out_dim(int in, int k, int stride, int pad);
+
+/*
+ * gdws_plan_gdw_stage -- where the fused bf16 kernel of this plan runs the GDW stage (Section 3.1,
+ * Definition) with the current GDWS_OPT_DW_MATH: *stage = 1 (ALUs) or 2 (tensor cores).  With the option
+ * at 0 the choice follows the measured cost of the two kernels: the tensor-core form costs k*k products
+ * per window of 16 input channels whatever their g_c, the ALU form costs in proportion to sum g_c; the
+ * tensor cores are taken for k = 3, stride 1, at most 256 output channels and an average g_c of at
+ * least 4.  Host only; errors: GDWS_ERR_INVALID_ARG.
+ */
+GDWS_API gdws_status_t gdws_plan_gdw_stage(const gdws_plan_t *plan, int *stage);
 
 /*
  * gdws_pack_weights -- convert one weight set to the kernels' internal form

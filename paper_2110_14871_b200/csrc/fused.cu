@@ -50,7 +50,7 @@ struct alignas(64) FusedParams {
     int Dtot, Dpad_tot;            // output channels of the layer (row pitch of y), rows per chunk of the packed pointwise matrix
     int box_bytes, slot_bytes;
     int nhalf, unit_bytes, nacc, acc_cols;
-    int a_kmajor, dw_math, zout;
+    int a_kmajor, zout;
 };
 
 // Warp roles, in warpgroups of 4 so that registers can be moved between the roles (setmaxnreg):
@@ -890,7 +890,6 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     P.acc_cols = tmem_cols_for(Dloc);
     P.nacc = P.acc_cols <= 256 ? 2 : 1;
     P.a_kmajor = zout ? 1 : p->opt_a_layout;
-    P.dw_math = p->opt_dw_math;
     P.zout = zout ? 1 : 0;
     const size_t smem = t.smem;     // one block per SM (register file), so the TMEM columns are never oversubscribed
     const int grid = nsplit > 1 ? P.ntiles * nsplit : (P.ntiles < p->sm_count ? P.ntiles : p->sm_count);
@@ -920,8 +919,11 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
 
 gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t st)
 {
-    // GDWS_OPT_DW_MATH: 0 or 1 = GDW stage on the ALUs (the faster kernel on every benchmark layer), 2 = on the tensor cores
-    if (p->opt_dw_math == 2) return bf16_fused_tc(p, x, y, st);
+    // GDWS_OPT_DW_MATH: 1 = GDW stage on the ALUs, 2 = on the tensor cores, 0 = whichever measured faster for this kind of layer
+    if (gdw_stage_of(p) == 2) {
+        const gdws_status_t rc = bf16_fused_tc(p, x, y, st);
+        if (rc != GDWS_ERR_UNSUPPORTED || p->opt_dw_math == 2) return rc;     // chosen automatically but no tile fits: the ALU kernel
+    }
     return run_tiled(p, x, y->ptr, y->h, y->w, false, st);
 }
 

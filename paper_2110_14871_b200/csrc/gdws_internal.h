@@ -131,6 +131,16 @@ bool choose_tile(const gdws_plan_s *p, int n, int h, int w, Tile *t);
 
 inline size_t dtype_size(gdws_dtype_t d) { return d == GDWS_F32 ? 4 : 2; }
 
+// Where the fused bf16 kernel runs the GDW stage: 1 = ALUs, 2 = tensor cores.  With the option left at 0 the
+// tensor cores are taken where they measured faster on B200: their cost is k*k products per 16-channel window
+// whatever the multipliers, the ALU kernel's is proportional to G, and beyond 256 output channels the PW
+// accumulator leaves no room for a second GDW accumulator.
+inline int gdw_stage_of(const gdws_plan_s *p)
+{
+    if (p->opt_dw_math == 1 || p->opt_dw_math == 2) return p->opt_dw_math;
+    return (p->tc_ok && p->k == 3 && p->stride == 1 && p->Dpad <= 256 && p->G >= 4 * p->C) ? 2 : 1;
+}
+
 // SMs of the plan's device; a plan built without a device (host-side queries only) assumes a B200's 148.
 constexpr int kB200Sms = 148;
 inline int sm_count_of(const gdws_plan_s *p) { return p->sm_count > 0 ? p->sm_count : kB200Sms; }

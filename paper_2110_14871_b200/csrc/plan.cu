@@ -472,6 +472,13 @@ gdws_status_t gdws_set_workspace(gdws_plan_t *p, void *ws, size_t bytes)
     return GDWS_OK;
 }
 
+gdws_status_t gdws_plan_gdw_stage(const gdws_plan_t *p, int *stage)
+{
+    if (!p || !stage) return fail(GDWS_ERR_INVALID_ARG, "gdws_plan_gdw_stage: NULL argument");
+    *stage = gdw_stage_of(p);
+    return GDWS_OK;
+}
+
 int64_t gdws_launch_count(const gdws_plan_t *p) { return p ? p->launches : 0; }
 
 const char *gdws_last_error(void) { return gdws::g_err; }

@@ -28,7 +28,7 @@ EXPORTS = [
     "gdws_out_dim", "gdws_pack_weights", "gdws_workspace_bytes", "gdws_set_workspace", "gdws_forward",
     "gdws_depthwise", "gdws_pointwise", "gdws_forward_host", "gdws_status", "gdws_launch_count",
     "gdws_last_error", "gdws_version", "gdws_destroy", "gdws_forward_static", "gdws_static_scratch_bytes",
-    "gdws_measure_fma_rate", "gdws_measure_code_size", "gdws_selftest_wait",
+    "gdws_measure_fma_rate", "gdws_measure_code_size", "gdws_selftest_wait", "gdws_plan_gdw_stage",
 ]
 
 
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
     L.gdws_plan_tables.restype = ci
     L.gdws_plan_tile.argtypes = [vp, ci, ci, ci, pint, pint, pint, pi64]
     L.gdws_plan_tile.restype = ci
+    L.gdws_plan_gdw_stage.argtypes = [vp, pint]
+    L.gdws_plan_gdw_stage.restype = ci
     L.gdws_out_dim.argtypes = [ci, ci, ci, ci]
     L.gdws_out_dim.restype = ci
     L.gdws_pack_weights.argtypes = [vp, vp, vp, vp, ci, vp]
@@ -238,6 +240,12 @@ class Plan:
         _check(lib().gdws_plan_tile(self._h, n, h, w, ctypes.byref(TN), ctypes.byref(PH), ctypes.byref(PW),
                                     ctypes.byref(tiles)))
         return TN.value, PH.value, PW.value, tiles.value
+
+    def gdw_stage(self) -> int:
+        """gdws_plan_gdw_stage: 1 = the fused kernel runs the GDW stage on the ALUs, 2 = on the tensor cores."""
+        st = ctypes.c_int()
+        _check(lib().gdws_plan_gdw_stage(self._h, ctypes.byref(st)))
+        return st.value
 
     def workspace_bytes(self, dtype: int, n: int, h: int, w: int) -> int:
         return int(lib().gdws_workspace_bytes(self._h, dtype, n, h, w))

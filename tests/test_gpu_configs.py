@@ -103,16 +103,19 @@ def test_full_size_layer_sampled_images(cfg, layer):
     _check_sampled(spec, g, x, dw_w, pw_w, bias, y)
 
 
-# the other launch configurations at full size: GDW stage on the tensor cores, and the unfused pair
+# the other launch configurations at full size: GDW stage forced onto the ALUs / the tensor cores (the default
+# lets the library choose), and the unfused pair
 OTHER = [(1, 0), (2, 0), (4, 4)]
 
 
 @pytest.mark.parametrize("cfg,layer", OTHER)
-@pytest.mark.parametrize("variant", ["tensor_core_gdw", "unfused"])
+@pytest.mark.parametrize("variant", ["alu_gdw", "tensor_core_gdw", "unfused"])
 def test_full_size_other_paths(cfg, layer, variant):
     spec = gi.config_layers(cfg)[layer]
     g, x, dw_w, pw_w, bias, _ = _instance(spec)
-    if variant == "tensor_core_gdw":
+    if variant == "alu_gdw":
+        y = _layer_on_gpu(spec, g, x, dw_w, pw_w, bias, path=gdws.PATH_FUSED, dw_math=1, twice=True)
+    elif variant == "tensor_core_gdw":
         y = _layer_on_gpu(spec, g, x, dw_w, pw_w, bias, path=gdws.PATH_FUSED, dw_math=2, twice=True)
     else:
         y = _layer_on_gpu(spec, g, x, dw_w, pw_w, bias, path=gdws.PATH_UNFUSED, twice=True)

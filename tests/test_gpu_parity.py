@@ -92,7 +92,7 @@ BF16_SHAPES = [
 ]
 
 
-# dw_math: 0 or 1 = GDW stage on the ALUs (default); 2 = on the tensor cores (own tests below)
+# dw_math: 0 = the library chooses where the GDW stage runs, 1 = on the ALUs, 2 = on the tensor cores (own tests below)
 @pytest.mark.parametrize("path,a_layout,dw_math", [(gdws.PATH_UNFUSED, 0, 0), (gdws.PATH_FUSED, 0, 0), (gdws.PATH_FUSED, 1, 1)])
 @pytest.mark.parametrize("shape", BF16_SHAPES)
 def test_bf16_forward_matches_reference(shape, path, a_layout, dw_math):
