@@ -67,7 +67,11 @@ def layer_numbers(spec: gi.LayerSpec, G: int):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (key: config, layer, path, GDW stage).  An entry is removed when its kernel changes.
-TRAFFIC_BYTES_PER_LAUNCH = {}
+TRAFFIC_BYTES_PER_LAUNCH = {
+    (1, 0, "fused", 2): 9199104,      # x + weights; y (8.39 MB) stays in L2 within the captured launch
+    (2, 0, "fused", 1): 25806848,     # x + weights; y (25.7 MB) stays in L2
+    (3, 0, "fused", 2): 93391872,     # x (67.1 MB) + the part of y that left L2
+}
 
 
 def layer_roofline_us(macs, nbytes, peaks, sustained=False):
@@ -504,7 +508,7 @@ def run_ours(args, spec):
         "ms_per_step": sec_per_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": spec.dtype, "data": "synthetic", "config": cfg,
         "effective_tmacs": world * macs / sec_per_step / 1e12,
-        "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps * repeats,
         "clocks": clocks, "parity_max_rel_err": parity, "context": context,
     }
     print(json.dumps(out), flush=True)
