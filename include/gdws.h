@@ -80,12 +80,16 @@ typedef enum {
     GDWS_OPT_A_LAYOUT = 3, /* bf16 fused path, shared-memory layout of the intermediate
                               tile handed to the tensor cores: 0 = pixel-contiguous
                               (default), 1 = channel-contiguous                            */
-    GDWS_OPT_DW_MATH = 4   /* bf16 fused path, where the GDW stage runs: 1 = on the ALUs (fp32
+    GDWS_OPT_DW_MATH = 4,  /* bf16 fused path, where the GDW stage runs: 1 = on the ALUs (fp32
                               multiply-adds); 2 = on the tensor cores as k*k block-sparse
                               products per 16-channel window (fp32 accumulation), for stride 1
                               and k <= 5, else GDWS_ERR_UNSUPPORTED; 0 (default) = the library
                               chooses (see gdws_plan_gdw_stage).  Both give the same result
                               up to summation order                                         */
+    GDWS_OPT_OUT_DTYPE = 5 /* bf16 plans: 0 (default) = y has the dtype of x; 1 = y is fp32
+                              (GDWS_F32, NHWC): bias and ReLU are applied to the fp32 sums of
+                              the PW stage and stored without the rounding to bf16.  Every
+                              forward call of the plan then expects such a y               */
 } gdws_option_t;
 
 typedef enum {

@@ -34,8 +34,10 @@ gdws_status_t check_pair(const gdws_plan_s *p, const gdws_tensor_t *x, const gdw
     if (x->c != p->C) return fail(GDWS_ERR_INVALID_ARG, "x->c=%d but the plan has C=%d", x->c, p->C);
     if (y->c != p->D) return fail(GDWS_ERR_INVALID_ARG, "y->c=%d but the plan has D=%d", y->c, p->D);
     if (x->n != y->n) return fail(GDWS_ERR_INVALID_ARG, "batch mismatch: x->n=%d y->n=%d", x->n, y->n);
-    if (x->dtype != y->dtype || x->layout != y->layout)
-        return fail(GDWS_ERR_INVALID_ARG, "x and y must share dtype and layout");
+    const gdws_dtype_t want = (x->dtype == GDWS_BF16 && p->opt_out_f32) ? GDWS_F32 : x->dtype;
+    if (y->dtype != want)
+        return fail(GDWS_ERR_INVALID_ARG, "y must be %s for this plan and x", want == GDWS_F32 ? "fp32" : "bf16 (GDWS_OPT_OUT_DTYPE is 0)");
+    if (x->layout != y->layout) return fail(GDWS_ERR_INVALID_ARG, "x and y must share the layout");
     const int Ho = gdws_out_dim(x->h, p->k, p->stride, p->pad), Wo = gdws_out_dim(x->w, p->k, p->stride, p->pad);
     if (Ho < 1 || Wo < 1) return fail(GDWS_ERR_INVALID_ARG, "input %dx%d is smaller than the filter", x->h, x->w);
     if (y->h != Ho || y->w != Wo)
@@ -168,7 +170,7 @@ gdws_status_t gdws_pointwise(gdws_plan_t *p, const void *z, const void *pw_w, co
     st = prepare(p);
     if (st != GDWS_OK) return st;
     cudaStream_t cs = (cudaStream_t)stream;
-    if (y->dtype == GDWS_F32) {
+    if (y->dtype == GDWS_F32 && !p->opt_out_f32) {
         if (!pw_w || !aligned16(pw_w)) return fail(GDWS_ERR_INVALID_ARG, "fp32 plans need pw_w (16-byte aligned)");
         return f32_pointwise(p, (const float *)z, (const float *)pw_w, bias, y, cs);
     }

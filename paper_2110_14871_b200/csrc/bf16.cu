@@ -261,7 +261,7 @@ __global__ void __launch_bounds__(kPwThreads, 1) pw_bf16_tc_kernel(const __grid_
                 uint32_t acc[16];
                 tmem_ld16(t_base + (uint32_t)d0, acc);
                 tmem_ld_wait();
-                if (p < P.npix) store_row16(acc, P.bias, d0, P.D, P.relu, P.y + (size_t)p * P.D);
+                if (p < P.npix) store_row16(acc, P.bias, d0, P.D, P.relu, P.y, (size_t)p * P.D);
             }
             tc_fence_before();
             __syncwarp();
@@ -299,7 +299,7 @@ gdws_status_t bf16_pointwise(gdws_plan_s *p, const void *z, gdws_tensor_t *y, cu
         if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     }
     P.pw_img = p->d_pw_img; P.bias = p->d_bias; P.y = (uint16_t *)y->ptr; P.status = p->d_status;
-    P.npix = npix; P.ntiles = (int)tiles; P.nchunks = p->nchunks; P.D = p->D; P.Dpad = p->Dpad; P.relu = p->opt_relu;
+    P.npix = npix; P.ntiles = (int)tiles; P.nchunks = p->nchunks; P.D = p->D; P.Dpad = p->Dpad; P.relu = (p->opt_relu ? kOutRelu : 0) | (y->dtype == GDWS_F32 ? kOutF32 : 0);
     P.stage_bytes = 16384 + p->Dpad * kChunk * 2;
     P.ns = (kMaxSmem - 1024) / P.stage_bytes;
     if (P.ns > kPwMaxStages) P.ns = kPwMaxStages;

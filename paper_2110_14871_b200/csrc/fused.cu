@@ -350,7 +350,7 @@ __device__ __forceinline__ void dw_generic(const FusedParams &P, uint32_t xs, in
 
 // Epilogue of one thread's accumulator row with direct stores: the 16-column granules first, first + step, ...
 // go from TMEM through bias / ReLU / bf16 rounding to y.
-__device__ __forceinline__ void epilogue_row(const FusedParams &P, uint32_t t_base, uint32_t bias_s, uint16_t *yrow, bool live,
+__device__ __forceinline__ void epilogue_row(const FusedParams &P, uint32_t t_base, uint32_t bias_s, size_t yrow, bool live,
                                              int first, int step)
 {
     const int ngran = P.Dpad >> 4;
@@ -360,10 +360,14 @@ __device__ __forceinline__ void epilogue_row(const FusedParams &P, uint32_t t_ba
         tmem_ld_wait();
         if (live) {
             float bv[16];
-            uint32_t o[8];
             bias16_shared(bias_s + (uint32_t)j * 64, bv);
-            finish_row16(acc, bv, P.relu, o);
-            store_packed16(o, j * 16, P.D, yrow);
+            if (P.relu & kOutF32) {          // fp32 output asked for: the sums are not rounded to bf16
+                finish_store_row16_f32(acc, bv, P.relu & kOutRelu, j * 16, P.D, reinterpret_cast<float *>(P.y) + yrow);
+            } else {
+                uint32_t o[8];
+                finish_row16(acc, bv, P.relu & kOutRelu, o);
+                store_packed16(o, j * 16, P.D, P.y + yrow);
+            }
         }
     }
 }
@@ -629,7 +633,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
             const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
             const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
-            uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.Dtot + part * P.Dpad;
+            const size_t yrow = (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.Dtot + part * P.Dpad;   // element index of the row's first channel
             if (ZOUT) {
                 // this thread's pixel row of every finished stage goes to z (row r of the stage: 128 bytes, swizzled)
                 for (int q = 0; q < P.nchunks; ++q, ++wq) {
@@ -641,7 +645,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                     for (int c = 0; c < 8; ++c) v[c] = lds128(row_s + (uint32_t)((c ^ (r & 7)) << 4));
                     warp_arrive(bar_afree + 8 * sa);
                     if (live) {
-                        uint4 *dst = reinterpret_cast<uint4 *>(yrow + (size_t)q * kChunk);
+                        uint4 *dst = reinterpret_cast<uint4 *>(P.y + yrow + (size_t)q * kChunk);
 #pragma unroll
                         for (int c = 0; c < 8; ++c) dst[c] = v[c];
                     }
@@ -670,7 +674,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                         tmem_ld_wait();
                         float bv[16];
                         bias16_shared(bias_s + (uint32_t)(cb * 64 + h4 * 16) * 4, bv);
-                        finish_row16(acc, bv, P.relu, o);
+                        finish_row16(acc, bv, P.relu & kOutRelu, o);
                         sts128(row_s + (uint32_t)(((2 * h4) ^ (r & 7)) << 4), make_uint4(o[0], o[1], o[2], o[3]));
                         sts128(row_s + (uint32_t)(((2 * h4 + 1) ^ (r & 7)) << 4), make_uint4(o[4], o[5], o[6], o[7]));
                     }
@@ -773,7 +777,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
         const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
         const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
-        uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.Dtot + part * P.Dpad;
+        const size_t yrow = (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.Dtot + part * P.Dpad;
         const int buf = tl % P.nacc;
         warp_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
         tc_fence_after();
@@ -826,7 +830,7 @@ static gdws_status_t launch_fast(const FusedParams &P, int device, int grid, siz
     }
 }
 
-static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out, int Ho, int Wo, bool zout, cudaStream_t st)
+static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out, int Ho, int Wo, bool zout, bool out_f32, cudaStream_t st)
 {
     if (!zout && p->Dpad > 512) return fail(GDWS_ERR_UNSUPPORTED, "bf16 fused kernel supports D <= 512 (got %d)", p->D);
     if (p->D % 8 || p->C % 8)
@@ -856,7 +860,7 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     }
     // The staged epilogue pays when it overlaps the next tile's main loop; a block with a single tile would
     // only wait for its one staging buffer between the column blocks.
-    const bool tma_out = !zout && t.ostage && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && t.tiles() > p->sm_count;
+    const bool tma_out = !zout && !out_f32 && t.ostage && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && t.tiles() > p->sm_count;
     if (tma_out) {
         // y as a rank-4 tensor, innermost first: channels, width, height, batch
         const cuuint64_t dims[4] = {(cuuint64_t)p->D, (cuuint64_t)Wo, (cuuint64_t)Ho, (cuuint64_t)x->n};
@@ -879,7 +883,7 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     P.nsplit = nsplit; P.Dtot = zout ? p->Gpad : p->D; P.Dpad_tot = p->Dpad;
     P.N = x->n; P.H = x->h; P.W = x->w; P.C = p->C; P.Ho = Ho; P.Wo = Wo; P.D = zout ? p->Gpad : (nsplit > 1 ? Dloc : p->D); P.Dpad = Dloc;
     P.G = p->G; P.nchunks = p->nchunks; P.stride = p->stride; P.pad = p->pad;
-    P.relu = p->opt_relu;
+    P.relu = (p->opt_relu ? kOutRelu : 0) | (out_f32 ? kOutF32 : 0);
     P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
     P.IH = t.IH; P.IW = t.IW; P.ps = t.cbox * 2; P.nslots = t.nslots; P.nwslots = t.nwslots; P.nboxes = p->nboxes; P.nsb = t.nsb; P.wstride = p->wstride;
     P.spg_shift = t.spg == 2 ? 1 : 0;
@@ -924,7 +928,7 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
         const gdws_status_t rc = bf16_fused_tc(p, x, y, st);
         if (rc != GDWS_ERR_UNSUPPORTED || p->opt_dw_math == 2) return rc;     // chosen automatically but no tile fits: the ALU kernel
     }
-    return run_tiled(p, x, y->ptr, y->h, y->w, false, st);
+    return run_tiled(p, x, y->ptr, y->h, y->w, false, y->dtype == GDWS_F32, st);
 }
 
 // The unfused GDW stage with the tiled pipeline (TMA-staged input, register-blocked depthwise warps,
@@ -933,7 +937,7 @@ gdws_status_t bf16_fused(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *
 gdws_status_t bf16_depthwise_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cudaStream_t st)
 {
     const int Ho = gdws_out_dim(x->h, p->k, p->stride, p->pad), Wo = gdws_out_dim(x->w, p->k, p->stride, p->pad);
-    return run_tiled(p, x, z, Ho, Wo, true, st);
+    return run_tiled(p, x, z, Ho, Wo, true, false, st);
 }
 
 }  // namespace gdws

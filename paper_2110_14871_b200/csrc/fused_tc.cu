@@ -420,7 +420,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
             const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
             const bool live = n < P.N && ho < P.Ho && wo < P.Wo;
-            uint16_t *yrow = P.y + (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D + part * P.Dloc;
+            const size_t yrow = (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D + part * P.Dloc;   // element index of the row's first channel
             const int dvalid = P.D - part * P.Dloc < P.Dloc ? P.D - part * P.Dloc : P.Dloc;
             const int buf = it % P.nacc;
             tc_warp_wait(bar_accfull + 8 * buf, (uint32_t)(it / P.nacc) & 1u, &abort_flag, P.status, kStatusWaitMma);
@@ -442,7 +442,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                         tmem_ld_wait();
                         float bv[16];
                         bias16_shared(bias_part + (uint32_t)(cb * 64 + h4 * 16) * 4, bv);
-                        finish_row16(acc, bv, P.relu, o);
+                        finish_row16(acc, bv, P.relu & kOutRelu, o);
                         sts128(row_s + (uint32_t)(((2 * h4) ^ (r & 7)) << 4), make_uint4(o[0], o[1], o[2], o[3]));
                         sts128(row_s + (uint32_t)(((2 * h4 + 1) ^ (r & 7)) << 4), make_uint4(o[4], o[5], o[6], o[7]));
                     }
@@ -465,10 +465,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     tmem_ld_wait();
                     if (live && j * 16 < dvalid) {
                         float bv[16];
-                        uint32_t o[8];
                         bias16_shared(bias_part + (uint32_t)j * 64, bv);
-                        finish_row16(acc, bv, P.relu, o);
-                        store_packed16(o, j * 16, dvalid, yrow);
+                        if (P.relu & kOutF32) {      // fp32 output asked for: the sums are not rounded to bf16
+                            finish_store_row16_f32(acc, bv, P.relu & kOutRelu, j * 16, dvalid, reinterpret_cast<float *>(P.y) + yrow);
+                        } else {
+                            uint32_t o[8];
+                            finish_row16(acc, bv, P.relu & kOutRelu, o);
+                            store_packed16(o, j * 16, dvalid, P.y + yrow);
+                        }
                     }
                 }
                 tc_fence_before();
@@ -652,7 +656,7 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     P.wslab_bytes = (uint32_t)Dloc * 32u;
     P.xslot_bytes = (uint32_t)((g.xbox + 255) / 256 * 256);
     // Shared memory: output staging (optional) | B operand buffers | z slabs | weight slabs | input boxes | tables
-    const bool can_stage = p->D % 64 == 0 && Dloc % 64 == 0 && ((uintptr_t)y->ptr & 15) == 0 && nitems > p->sm_count;
+    const bool can_stage = y->dtype != GDWS_F32 && p->D % 64 == 0 && Dloc % 64 == 0 && ((uintptr_t)y->ptr & 15) == 0 && nitems > p->sm_count;
     const size_t tables = (size_t)nchunks * sizeof(TcChunk) + (size_t)p->tc_nparts * Dloc * 4 + kTcMaxNB * 256 + 256;
     double best_score = -1;
     int b_ost = 0, b_nx = 0, b_nb = 0, b_nz = 0, b_nw = 0;
@@ -730,7 +734,7 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     P.y = (uint16_t *)y->ptr; P.filt = p->d_tc_filt; P.pw = p->d_tc_pw; P.bias = p->d_bias; P.chunks = p->d_tc_chunks;
     P.status = p->d_status;
     P.N = x->n; P.Ho = Ho; P.Wo = Wo; P.D = p->D; P.Dloc = Dloc; P.Dpad_tot = p->tc_nparts * Dloc; P.nparts = p->tc_nparts;
-    P.nchunks = nchunks; P.pad = p->pad; P.relu = p->opt_relu;
+    P.nchunks = nchunks; P.pad = p->pad; P.relu = (p->opt_relu ? kOutRelu : 0) | (y->dtype == GDWS_F32 ? kOutF32 : 0);
     P.TN = g.TN; P.PH = g.PH; P.PW = g.PW; P.tiles_h = g.tiles_h; P.tiles_w = g.tiles_w; P.nitems = (int)nitems;
     P.nacc = Dloc <= 128 ? 2 : 1;
     P.rec_hw = p->tc_rec_hw; P.nslabs_total = p->tc_nslabs;

@@ -89,6 +89,7 @@ struct gdws_plan_s {
     int opt_tile = 0;
     int opt_a_layout = 0;
     int opt_dw_math = 0;
+    int opt_out_f32 = 0;           // bf16 plans: y is fp32
 
     // device side (allocated by ensure_device)
     int device = -1;

@@ -414,6 +414,9 @@ gdws_status_t gdws_plan_set_option(gdws_plan_t *p, int key, int value)
     case GDWS_OPT_DW_MATH:
         if (value < 0 || value > 2) return fail(GDWS_ERR_INVALID_ARG, "dw_math must be 0, 1 or 2");
         p->opt_dw_math = value; return GDWS_OK;
+    case GDWS_OPT_OUT_DTYPE:
+        if (value != 0 && value != 1) return fail(GDWS_ERR_INVALID_ARG, "out_dtype must be 0 (as x) or 1 (fp32)");
+        p->opt_out_f32 = value; return GDWS_OK;
     default:
         return fail(GDWS_ERR_INVALID_ARG, "unknown option %d", key);
     }

@@ -293,6 +293,24 @@ __device__ __forceinline__ void finish_row16(const uint32_t (&acc)[16], const fl
         o[j] = pack_bf16x2(lo, hi);
     }
 }
+// The same 16 columns kept as fp32 (bias, optional ReLU) and stored to an fp32 row: channels d0 .. d0+15 below D,
+// in 16-byte pieces (D is a multiple of 8 for these kernels, the row 16-byte aligned).
+__device__ __forceinline__ void finish_store_row16_f32(const uint32_t (&acc)[16], const float (&bv)[16], int relu, int d0, int D,
+                                                       float *__restrict__ yrow)
+{
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        float4 v;
+        v.x = __uint_as_float(acc[4 * q]) + bv[4 * q];
+        v.y = __uint_as_float(acc[4 * q + 1]) + bv[4 * q + 1];
+        v.z = __uint_as_float(acc[4 * q + 2]) + bv[4 * q + 2];
+        v.w = __uint_as_float(acc[4 * q + 3]) + bv[4 * q + 3];
+        if (relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
+        if (d0 + 4 * q + 4 <= D) *reinterpret_cast<float4 *>(yrow + d0 + 4 * q) = v;
+    }
+}
+// Flags carried in the kernels' `relu` parameter.
+enum : int { kOutRelu = 1, kOutF32 = 2 };
 // Stores a row's 16 finished channels d0 .. d0+15 (those below D) to yrow.
 __device__ __forceinline__ void store_packed16(const uint32_t (&o)[8], int d0, int D, uint16_t *__restrict__ yrow)
 {
@@ -306,14 +324,19 @@ __device__ __forceinline__ void store_packed16(const uint32_t (&o)[8], int d0, i
         if (d0 + 16 <= D) *reinterpret_cast<uint4 *>(dst + 8) = make_uint4(o[4], o[5], o[6], o[7]);
     }
 }
+// `y` is the output tensor's base, `row` the element index of the row's first channel; flags: kOutRelu, kOutF32.
 __device__ __forceinline__ void store_row16(const uint32_t (&acc)[16], const float *__restrict__ bias, int d0, int D,
-                                            int relu, uint16_t *__restrict__ yrow)
+                                            int flags, void *__restrict__ y, size_t row)
 {
     float bv[16];
-    uint32_t o[8];
     bias16_global(bias + d0, bv);
-    finish_row16(acc, bv, relu, o);
-    store_packed16(o, d0, D, yrow);
+    if (flags & kOutF32) {
+        finish_store_row16_f32(acc, bv, flags & kOutRelu, d0, D, reinterpret_cast<float *>(y) + row);
+    } else {
+        uint32_t o[8];
+        finish_row16(acc, bv, flags & kOutRelu, o);
+        store_packed16(o, d0, D, reinterpret_cast<uint16_t *>(y) + row);
+    }
 }
 
 // Issue the MMAs of one 64-wide K chunk (4 steps of K=16; output channels beyond 256 take a

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libgdws.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_ARCH, ERR_WORKSPACE = range(8)
 F32, BF16 = 0, 1
 NCHW, NHWC = 0, 1
-OPT_PATH, OPT_RELU, OPT_TILE, OPT_A_LAYOUT, OPT_DW_MATH = range(5)
+OPT_PATH, OPT_RELU, OPT_TILE, OPT_A_LAYOUT, OPT_DW_MATH, OPT_OUT_DTYPE = range(6)
 PATH_AUTO, PATH_FUSED, PATH_UNFUSED = 0, 1, 2
 
 EXPORTS = [

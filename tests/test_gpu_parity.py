@@ -291,3 +291,34 @@ def test_code_size_cliff_is_where_the_kernels_assume_it():
     small = gdws.measure_code_size(128, 512)
     large = gdws.measure_code_size(1024, 512)
     assert small > 0.7 and large < 0.65 * small, (small, large)
+
+
+@pytest.mark.parametrize("variant", ["alu", "tensor_cores", "unfused"])
+def test_fp32_output_of_a_bf16_plan(variant):
+    """GDWS_OPT_OUT_DTYPE = 1: y keeps the fp32 sums of the PW stage (bias, ReLU applied, no rounding to bf16), so it
+    is at least as close to the reference as the bf16 output, and equal to it after rounding."""
+    spec = small_spec("t", 3, 32, 40, 12, 9, 3, 1, 1, ("uniform", 1, 9), "bf16", "NHWC", relu=True, seed=91)
+    data = gi.make_layer(spec)
+    ref, _ = run_oracle(data)
+    path = gdws.PATH_UNFUSED if variant == "unfused" else gdws.PATH_FUSED
+    dw_math = 2 if variant == "tensor_cores" else 1
+    want16 = run_gpu(data, path=path, dw_math=dw_math)
+    plan = make_plan(data, path=path, dw_math=dw_math)
+    plan.set_option(gdws.OPT_OUT_DTYPE, 1)
+    x, dw, pw = (to_device(a, "bf16") for a in (data.x, data.dw_w, data.pw_w))
+    b = torch.from_numpy(data.bias).cuda()
+    if path == gdws.PATH_UNFUSED:
+        ws = torch.empty(plan.workspace_bytes(gdws.BF16, spec.N, spec.H, spec.W), dtype=torch.uint8, device="cuda")
+        plan.set_workspace(ws)
+    y = torch.full((spec.N, spec.Ho, spec.Wo, spec.D), float("nan"), dtype=torch.float32, device="cuda")
+    plan.forward(x, y, "NHWC", dw, pw, b)
+    torch.cuda.synchronize()
+    plan.status()
+    got = y.cpu().numpy().astype(np.float64)
+    assert rel_err(got, ref) <= TOL["bf16"]
+    assert rel_err(got, ref) <= rel_err(want16, ref) + 1e-6
+    assert np.array_equal(y.to(torch.bfloat16).float().cpu().numpy().astype(np.float64), want16)
+    y16 = torch.empty((spec.N, spec.Ho, spec.Wo, spec.D), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(gdws.GdwsError):
+        plan.forward(x, y16, "NHWC", dw, pw, b)        # the plan now expects an fp32 y
+    plan.destroy()
