@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
 {
     extern __shared__ uint8_t smem_raw[];
     // dwready[4] | zfull[2] (2 unused) | pwready[4] pwdone[4] | bfree[4] xfree[4] | accfull[2] accfree[2]
-    __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4 + 1];
+    __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4 + 2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -147,6 +147,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         for (int i = 0; i < kTcMaxNB; ++i) mbar_init(bar_bfree + 8 * i, 1);
         for (int i = 0; i < kTcMaxNX; ++i) mbar_init(bar_xfree + 8 * i, 1);
         mbar_init(bar_drain, 1);
+        mbar_init(bar_drain + 8, 1);
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512u);
@@ -186,10 +187,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         const uint32_t b_lo0 = ((b_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t xstep = P.xslot_bytes >> 4, bstep = P.bbuf_bytes >> 4, pstep = P.bplane >> 4;
         const uint32_t rstep = P.tap_row_step >> 4, cstep = P.tap_col_step >> 4;
-        const uint32_t idesc_pw = make_idesc(P.Dloc, false);
-        const uint32_t z_lo0 = ((z_s & 0x3FFFFu) >> 4) | (1u << 16);
-        const uint32_t w_lo0 = ((w_s & 0x3FFFFu) >> 4) | (1u << 16);
-        const uint32_t wstep = P.wslab_bytes >> 4;
         // The loop below is this warp's whole working set of instructions and is kept near a hundred of them (it has to
         // stay in the small instruction cache next to the scheduler while the other warps of the block come and go):
         // tap offsets live in registers, ring positions advance by a compare per slab, waits are calls when they miss.
@@ -202,63 +199,75 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 tap_b[ur * K + v] = (uint32_t)(ur * K + v) * pstep;
             }
         uint32_t xslot = 0, bslot = 0, a_lo = a_lo0, b_lo = b_lo0;
-        uint32_t zh = 0, wh = 0, z_lo = z_lo0, w_lo = w_lo0, buf = 0, accpar = 1;
         int q = 0;                  // chunk index of unit u within its work item
-        int qp = 0, itp = 0;        // the same for unit u - 1, and its work item
-        for (int u = 0; u <= total; ++u) {
-            if (u < total) {
-                const int npad = tab[q].npad, flags = tab[q].flags;
-                mbar_wait_call(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
-                tc_fence_after();
-                if (elect_one()) {
-                    const uint32_t idesc = make_idesc(npad, false);
-                    const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
+        for (int u = 0; u < total; ++u) {
+            const int npad = tab[q].npad, flags = tab[q].flags;
+            mbar_wait_call(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
+            // accumulator u & 1 held chunk u - 2: the converters have read it once they announce that chunk's slabs
+            if (u >= 2) mbar_wait_call(bar_pwready + 8 * ((u - 2) & 3), (uint32_t)((u - 2) >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
+            tc_fence_after();
+            if (elect_one()) {
+                const uint32_t idesc = make_idesc(npad, false);
+                const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
 #pragma unroll
-                    for (int i = 0; i < K * K; ++i)
-                        umma_bf16_words(d_z, a_lo + tap_a[i], a_hi, b_lo + tap_b[i], p_hi, idesc, i != 0);
-                    umma_commit(bar_zfull + 8 * (u & 1));
-                }
-                __syncwarp();
-                b_lo += bstep;
-                if (++bslot == (uint32_t)P.nb) { bslot = 0; b_lo = b_lo0; }
-                if (flags & 2) {
-                    a_lo += xstep;
-                    if (++xslot == (uint32_t)P.nx) { xslot = 0; a_lo = a_lo0; }
-                }
-                if (++q == P.nchunks) q = 0;
+                for (int i = 0; i < K * K; ++i)
+                    umma_bf16_words(d_z, a_lo + tap_a[i], a_hi, b_lo + tap_b[i], p_hi, idesc, i != 0);
+                umma_commit(bar_zfull + 8 * (u & 1));
             }
-            if (u > 0) {
-                const int v = u - 1;
-                const int ns = tab[qp].npad >> 4;
-                if (qp == 0 && itp >= P.nacc) mbar_wait_call(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
-                mbar_wait_call(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
-                tc_fence_after();
-                const bool leader = elect_one();
-                const uint32_t d_y = tmem + buf * 128u;
-#pragma unroll 1
-                for (int s = 0; s < ns; ++s) {           // every lane keeps the ring positions, the leader issues
-                    if (leader) umma_bf16_words(d_y, z_lo, p_hi, w_lo, p_hi, idesc_pw, (uint32_t)(qp | s));
-                    z_lo += kTcSlab >> 4;
-                    if (++zh == (uint32_t)P.nz) { zh = 0; z_lo = z_lo0; }
-                    w_lo += wstep;
-                    if (++wh == (uint32_t)P.nw) { wh = 0; w_lo = w_lo0; }
-                }
-                if (leader) {
-                    umma_commit(bar_pwdone + 8 * (v & 3));
-                    if (qp == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
-                }
-                __syncwarp();
-                if (++qp == P.nchunks) {
-                    qp = 0; ++itp;
-                    if (++buf == (uint32_t)P.nacc) { buf = 0; accpar ^= 1; }
-                }
+            __syncwarp();
+            b_lo += bstep;
+            if (++bslot == (uint32_t)P.nb) { bslot = 0; b_lo = b_lo0; }
+            if (flags & 2) {
+                a_lo += xstep;
+                if (++xslot == (uint32_t)P.nx) { xslot = 0; a_lo = a_lo0; }
             }
+            if (++q == P.nchunks) q = 0;
         }
-        // Teardown: one more commit covers every product issued before it (after an abort, products may have been issued
+        // Teardown: one more commit covers every product this thread issued (after an abort, products may have been issued
         // on operands that were not there; they must have ended all the same); its wait is bounded and ignores the abort flag.
-        if (lane == 0) {
+        if (elect_one()) {
             umma_commit(bar_drain);
             mbar_wait_drain(bar_drain, 0);
+        }
+        __syncwarp();
+    } else if (warp == 3) {
+        // ---------------- PW issue ----------------
+        // A second issuing warp: while it waits, commits and keeps its ring positions, warp 0 issues the next chunk's GDW
+        // products, and the other way round.  The two streams of products go to different accumulators and may interleave.
+        const uint32_t idesc_pw = make_idesc(P.Dloc, false);
+        const uint32_t z_lo0 = ((z_s & 0x3FFFFu) >> 4) | (1u << 16);
+        const uint32_t w_lo0 = ((w_s & 0x3FFFFu) >> 4) | (1u << 16);
+        const uint32_t wstep = P.wslab_bytes >> 4;
+        uint32_t zh = 0, wh = 0, z_lo = z_lo0, w_lo = w_lo0, buf = 0, accpar = 1;
+        int qp = 0, itp = 0;
+        for (int v = 0; v < total; ++v) {
+            const int ns = tab[qp].npad >> 4;
+            if (qp == 0 && itp >= P.nacc) mbar_wait_call(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
+            mbar_wait_call(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
+            tc_fence_after();
+            const bool leader = elect_one();
+            const uint32_t d_y = tmem + buf * 128u;
+#pragma unroll 1
+            for (int s = 0; s < ns; ++s) {           // every lane keeps the ring positions, the leader issues
+                if (leader) umma_bf16_words(d_y, z_lo, p_hi, w_lo, p_hi, idesc_pw, (uint32_t)(qp | s));
+                z_lo += kTcSlab >> 4;
+                if (++zh == (uint32_t)P.nz) { zh = 0; z_lo = z_lo0; }
+                w_lo += wstep;
+                if (++wh == (uint32_t)P.nw) { wh = 0; w_lo = w_lo0; }
+            }
+            if (leader) {
+                umma_commit(bar_pwdone + 8 * (v & 3));
+                if (qp == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
+            }
+            __syncwarp();
+            if (++qp == P.nchunks) {
+                qp = 0; ++itp;
+                if (++buf == (uint32_t)P.nacc) { buf = 0; accpar ^= 1; }
+            }
+        }
+        if (elect_one()) {
+            umma_commit(bar_drain + 8);
+            mbar_wait_drain(bar_drain + 8, 0);
         }
         __syncwarp();
     } else if (warp == 1) {

@@ -11,6 +11,8 @@ the same entry point, so the shared array holds NaNs wherever the target layer d
 stale element read by the second layer would show.  Across the calls the device's free memory and
 torch's allocation count must not move.  A layer whose intermediate exceeds the built-in array is
 refused without a launch; overlapping x and y are refused as gdws_forward refuses them."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -57,6 +59,8 @@ def test_forward_static_matches_forward_twice(dtype, layout):
     if dtype == "bf16":
         plan.pack_weights(dw, pw, b)          # the allocation-free call then takes no weight arguments
     torch.cuda.synchronize()
+    gc.collect()                  # tensors of earlier tests that only the cycle collector frees must not go in between
+    gc.disable()
     free_before, _ = torch.cuda.mem_get_info()
     count_before = torch.cuda.memory_stats().get("allocation.all.allocated", 0)
     held_before = torch.cuda.memory_allocated()
@@ -69,7 +73,9 @@ def test_forward_static_matches_forward_twice(dtype, layout):
     free_after, _ = torch.cuda.mem_get_info()
     assert free_after == free_before, "device memory in use changed across gdws_forward_static"
     assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == count_before
-    assert torch.cuda.memory_allocated() == held_before
+    held_after = torch.cuda.memory_allocated()
+    gc.enable()
+    assert held_after == held_before
     for call in range(2):
         got = ys[call].float().cpu().numpy().astype(np.float64)
         assert rel_err(got, want) <= TOL[dtype], call
