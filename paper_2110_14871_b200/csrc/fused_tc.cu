@@ -70,25 +70,12 @@ struct alignas(64) TcParams {
     int ostage, rec_hw, nslabs_total, bias_len;
 };
 
-// Bounded wait of every role but the MMA warp: each poll lets the hardware suspend the thread until the phase
-// completes (or 16 us pass), so that waiting warps issue next to nothing.  The MMA warp is a single
-// instruction stream whose shared-memory latency sets the pace of the whole pipeline; polls of a dozen other
-// warps in front of it in the shared-memory queue slowed it down several times.
+// Bounded wait of every role but the issuing warps: each poll lets the hardware suspend the thread until the phase
+// completes (or 16 us pass), so that waiting warps issue next to nothing.  The polling loop is a call (one copy of it in
+// the kernel; inlined and unrolled at every site it was a third of the kernel's code), the first poll is inline.
 __device__ __forceinline__ void tc_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
 {
-    if (mbar_try_wait(bar, parity)) return;
-    if (*abort_flag) return;
-    for (uint32_t it = 0; it < (1u << 16); ++it) {     // bounded: about a second
-        if (mbar_try_wait_suspend(bar, parity, 16384u)) return;
-        if (*abort_flag) return;
-    }
-    *abort_flag = 1;
-    atomicOr(status, code);
-}
-__device__ __forceinline__ void tc_warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
-{
-    if ((threadIdx.x & 31) == 0) tc_wait(bar, parity, abort_flag, status, code);
-    __syncwarp();
+    if (!mbar_try_wait(bar, parity)) mbar_wait_relaxed_slow(bar, parity, 16384u, abort_flag, status, code);
 }
 // The same with the polling loop as a call: for the warps whose per-chunk code has to stay small.
 __device__ __forceinline__ void tc_warp_wait_call(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
@@ -200,6 +187,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             }
         uint32_t xslot = 0, bslot = 0, a_lo = a_lo0, b_lo = b_lo0;
         int q = 0;                  // chunk index of unit u within its work item
+#pragma unroll 1
         for (int u = 0; u < total; ++u) {
             const int npad = tab[q].npad, flags = tab[q].flags;
             mbar_wait_call(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
@@ -240,6 +228,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         const uint32_t wstep = P.wslab_bytes >> 4;
         uint32_t zh = 0, wh = 0, z_lo = z_lo0, w_lo = w_lo0, buf = 0, accpar = 1;
         int qp = 0, itp = 0;
+#pragma unroll 1
         for (int v = 0; v < total; ++v) {
             const int ns = tab[qp].npad >> 4;
             if (qp == 0 && itp >= P.nacc) mbar_wait_call(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
@@ -276,6 +265,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             int box = 0, u = 0;
             uint32_t xslot = 0;
             bool stop = false;
+#pragma unroll 1
             for (int it = 0; it < my_items && !stop; ++it) {
                 const int item = (int)blockIdx.x + it * (int)gridDim.x;
                 int tile = item / P.nparts;
@@ -283,6 +273,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 tile -= bn * tiles_hw;
                 const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
                 const int n0 = bn * P.TN, hi0 = bh * P.PH - P.pad, wi0 = bw * P.PW - P.pad;
+#pragma unroll 1
                 for (int q = 0; q < P.nchunks; ++q, ++u) {
                     const int cbase = tab[q].cbase, flags = tab[q].flags;
                     const uint32_t bar = bar_dwready + 8 * (u & 3);
@@ -294,6 +285,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                         tc_wait(bar_xfree + 8 * xslot, (uint32_t)((box / P.nx) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
                     mbar_expect_tx(bar, (uint32_t)P.xbox_bytes);
                     const uint32_t dst = x_s + xslot * P.xslot_bytes;
+#pragma unroll 1
                     for (int l = 0; l < P.nloads; ++l)
                         tma_load_4d(dst + P.load_off[l], &P.tmap_x, cbase, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, bar);
                     ++box;
@@ -314,9 +306,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             SlabRing ring;
             ring.free_slabs = P.nw;
             int q = 0, it = 0, issued = 0;
+#pragma unroll 1
             for (int v = 0; v < total; ++v) {
                 const TcChunk ch = tab[q];
                 const int ns = ch.npad >> 4;
+#pragma unroll 1
                 while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
                     const int o = ring.oldest;
                     tc_wait(bar_pwdone + 8 * (o & 3), (uint32_t)(o >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
@@ -358,8 +352,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         ring.free_slabs = P.nz;
         uint32_t bslot = 0, xslot = 0;
         int q = 0, qo = 0;                                   // chunk index of unit v and of the ring's oldest unit
+#pragma unroll 1
         for (int v = 0; v < total; ++v) {
             const int ns = tab[q].npad >> 4, flags = tab[q].flags;
+#pragma unroll 1
             while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
                 const int o = ring.oldest;
                 tc_warp_wait_call(bar_pwdone + 8 * (o & 3), (uint32_t)(o >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
@@ -420,6 +416,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         const int rem = r - tn * hw;
         const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
         const bool issuer = warp == kTcEpiWarp0 && lane == 0;
+#pragma unroll 1
         for (int it = 0; it < my_items; ++it) {
             const int item = (int)blockIdx.x + it * (int)gridDim.x;
             int tile = item / P.nparts;
@@ -432,7 +429,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             const size_t yrow = (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D + part * P.Dloc;   // element index of the row's first channel
             const int dvalid = P.D - part * P.Dloc < P.Dloc ? P.D - part * P.Dloc : P.Dloc;
             const int buf = it % P.nacc;
-            tc_warp_wait(bar_accfull + 8 * buf, (uint32_t)(it / P.nacc) & 1u, &abort_flag, P.status, kStatusWaitMma);
+            tc_warp_wait_call(bar_accfull + 8 * buf, (uint32_t)(it / P.nacc) & 1u, &abort_flag, P.status, kStatusWaitMma);
             tc_fence_after();
             const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * 128);
             const uint32_t bias_part = bias_s + (uint32_t)(part * P.Dloc) * 4u;
@@ -441,6 +438,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 // (64, PW, PH, TN) box of y; 16-byte pieces swizzled by row), stored by TMA, which clips the box.
                 const uint32_t row_s = o_s + (uint32_t)r * 128;
                 const int nblk = P.Dloc >> 6;
+#pragma unroll 1
                 for (int cb = 0; cb < nblk; ++cb) {
                     if (issuer) bulk_wait_read_all();
                     named_bar_sync(1, 128);
@@ -468,6 +466,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 }
             } else {
                 const int ngran = P.Dloc >> 4;
+#pragma unroll 1
                 for (int j = 0; j < ngran; ++j) {
                     uint32_t acc[16];
                     tmem_ld16(t_base + (uint32_t)(j * 16), acc);
@@ -513,6 +512,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         if (total > 0) load_rec(tab[0], nxt);
         uint32_t bslot = 0, bpar = 0;      // B buffer of unit v, and the parity of the "free" phase it waits for
         int q = 0;
+#pragma unroll 1
         for (int v = 0; v < total; ++v) {
 #pragma unroll
             for (int j = 0; j < RW; ++j) rec[j] = nxt[j];
