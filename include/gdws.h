@@ -282,9 +282,11 @@ GDWS_API gdws_status_t gdws_measure_fma_rate(int kind, double *macs_per_clk_per_
 /*
  * gdws_measure_code_size -- diagnostic: instructions per clock and warp scheduler that `threads` threads per SM
  * (128, 256 or 512) sustain on independent fp32 multiply-adds in a loop whose body is `body_instructions` long
- * (64, 128, 160, 256, 512 or 1024; 16 bytes each).  Bodies beyond about 2 KB no longer fit the instruction cache
- * next to a scheduler; the rate then is that of instruction fetch.  This sizes the kernels' hot loops.  (No
- * counterpart in the paper.)  Allocates a few KB, runs for about a millisecond, synchronises.
+ * (128, 512, 1024, 2048, 3072, 4096, 6144 or 8192; 16 bytes each, the loop is not unrolled).  Measured on B200: up to
+ * 2048 instructions (32 KB) 0.7 to 0.9 per clock and scheduler; from 3072 (48 KB) on 0.31 with one warp per scheduler,
+ * 0.70 with two, 0.45 to 0.50 with four: code that all warps walk through has to stay below some 32 KB per SM, else it
+ * runs at the speed of instruction fetch.  (No counterpart in the paper.)  Allocates a few KB, runs for about a
+ * millisecond, synchronises.
  */
 GDWS_API gdws_status_t gdws_measure_code_size(int body_instructions, int threads, double *instructions_per_clk_per_scheduler);
 

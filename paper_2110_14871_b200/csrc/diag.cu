@@ -53,8 +53,9 @@ __global__ void __launch_bounds__(1024, 1) fma_rate_kernel(float *sink, long lon
     if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
 }
 
-// The same independent fp32 multiply-adds with a loop body of BODY instructions (16 bytes each): shows where straight-line
-// code stops fitting the instruction cache next to a scheduler and runs at the speed of instruction fetch instead.
+// The same independent fp32 multiply-adds with a loop body of BODY instructions (16 bytes each; the loop itself is kept
+// from being unrolled, so BODY * 16 bytes is what the warps walk through): shows where straight-line code stops
+// fitting the SM's instruction caches and runs at the speed of instruction fetch instead.
 template <int BODY>
 __global__ void __launch_bounds__(512, 1) code_size_kernel(float *sink, long long *cycles, int total_fma, float seed)
 {
@@ -68,6 +69,7 @@ __global__ void __launch_bounds__(512, 1) code_size_kernel(float *sink, long lon
     __syncthreads();
     const int iters = total_fma / BODY;
     const long long t0 = clock64();
+#pragma unroll 1
     for (int it = 0; it < iters; ++it) {
 #pragma unroll
         for (int b = 0; b < BODY / 32; ++b)
@@ -174,17 +176,19 @@ gdws_status_t gdws_measure_code_size(int body_instructions, int threads, double 
     e = cudaMalloc((void **)&sink, 4096);
     if (e == cudaSuccess) e = cudaMalloc((void **)&cyc, sizeof(long long) * (size_t)sms);
     if (e != cudaSuccess) { cudaFree(sink); return cuda_fail(e, "cudaMalloc"); }
-    const int total = 1 << 19;
+    const int total = 3 << 18;      // a multiple of every body size
     bool known = true;
     for (int pass = 0; pass < 2 && known; ++pass) {
-        const int n = pass == 0 ? 1 << 14 : total;
+        const int n = pass == 0 ? 3 << 13 : total;
         switch (body_instructions) {
-        case 64: code_size_kernel<64><<<sms, threads>>>(sink, cyc, n, 1.f); break;
         case 128: code_size_kernel<128><<<sms, threads>>>(sink, cyc, n, 1.f); break;
-        case 160: code_size_kernel<160><<<sms, threads>>>(sink, cyc, n, 1.f); break;
-        case 256: code_size_kernel<256><<<sms, threads>>>(sink, cyc, n, 1.f); break;
         case 512: code_size_kernel<512><<<sms, threads>>>(sink, cyc, n, 1.f); break;
         case 1024: code_size_kernel<1024><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 2048: code_size_kernel<2048><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 3072: code_size_kernel<3072><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 4096: code_size_kernel<4096><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 6144: code_size_kernel<6144><<<sms, threads>>>(sink, cyc, n, 1.f); break;
+        case 8192: code_size_kernel<8192><<<sms, threads>>>(sink, cyc, n, 1.f); break;
         default: known = false; break;
         }
     }
@@ -199,7 +203,7 @@ gdws_status_t gdws_measure_code_size(int body_instructions, int threads, double 
     }
     cudaFree(sink);
     cudaFree(cyc);
-    if (!known) return fail(GDWS_ERR_INVALID_ARG, "gdws_measure_code_size: body must be 64, 128, 160, 256, 512 or 1024 instructions");
+    if (!known) return fail(GDWS_ERR_INVALID_ARG, "gdws_measure_code_size: body must be 128, 512, 1024, 2048, 3072, 4096, 6144 or 8192 instructions");
     if (e != cudaSuccess) return cuda_fail(e, "gdws_measure_code_size");
     if (instructions_per_clk_per_scheduler)
         *instructions_per_clk_per_scheduler = worst > 0 ? (double)total * (threads / 32) / 4.0 / (double)worst : 0.0;

@@ -14,8 +14,8 @@
 //
 // One persistent block of 20 warps per SM walks over work items (tile of 128 output pixels x block of up to
 // 256 output channels).  Roles, coupled by mbarriers only:
-//   warp 0             issues every tcgen05.mma (one elected lane): for chunk u the k*k GDW products, then the
-//                      PW products of chunk u-1 (whose z is being converted meanwhile);
+//   warp 0             issues the k*k GDW products of every chunk (one elected lane);
+//   warp 3             issues the PW products of every chunk, once its z slabs and weights are in place;
 //   warp 1 (one lane)  fetches the input boxes by TMA (x as a rank-4 tensor: C, W, H, N; 16 channels per box);
 //   warp 2 (one lane)  streams the packed pointwise weights (bulk copies into a ring of 16-channel slabs);
 //   warps 4-11         converter: TMEM z -> bf16 -> ring of 16-channel operand slabs (two warps per lane quarter);
@@ -137,17 +137,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         mbar_init(bar_drain + 8, 1);
         fence_mbar_init();
     }
+    // The kernel that follows in the stream (launched with programmatic serialisation, as this one is) may start its
+    // blocks as SMs become free; it reads nothing from global memory before its own grid_dependency_wait below.
+    grid_launch_dependents();
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512u);
     {
-        const uint4 *src = reinterpret_cast<const uint4 *>(P.chunks);
-        uint4 *dst = reinterpret_cast<uint4 *>(tab);
-        for (int i = tid; i < P.nchunks * 2; i += kTcThreads) dst[i] = __ldg(src + i);
-        for (int d = tid; d < P.Dpad_tot; d += kTcThreads) bias_sm[d] = d < P.bias_len ? __ldg(P.bias + d) : 0.f;
         for (int i = tid; i < P.nb * 128; i += kTcThreads) bold[i] = 0xFFFFu;
         const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
         const uint32_t nb16 = (uint32_t)P.nb * P.bbuf_bytes / 16u;
         for (uint32_t i = tid; i < nb16; i += kTcThreads) sts128(b_s + i * 16u, zero);
         fence_proxy_async();
+        // Everything above touches this block's shared and tensor memory only.  From here on global memory is read and
+        // written: the kernel before this one in the stream (which may have produced x or the packed weights, or may
+        // still be reading what this one overwrites) has to be complete.
+        grid_dependency_wait();
+        const uint4 *src = reinterpret_cast<const uint4 *>(P.chunks);
+        uint4 *dst = reinterpret_cast<uint4 *>(tab);
+        for (int i = tid; i < P.nchunks * 2; i += kTcThreads) dst[i] = __ldg(src + i);
+        for (int d = tid; d < P.Dpad_tot; d += kTcThreads) bias_sm[d] = d < P.bias_len ? __ldg(P.bias + d) : 0.f;
     }
     tc_fence_before();
     __syncthreads();
@@ -159,24 +166,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const int tiles_hw = P.tiles_h * P.tiles_w;
     const uint32_t p_hi = (256u >> 4) | (1u << 14) | kTcSw32;   // descriptor high word: 8-row groups 256 bytes apart, version 1, 32-byte swizzle
 
-    // The issue warp is a single instruction stream that paces the pipeline: a satisfied mbarrier wait costs it some
-    // 140 cycles and a tcgen05.commit some 80, against 24 per tcgen05.mma (measured), while the tensor-core work of a
-    // chunk is a few hundred cycles.  Hence one wait and one commit per chunk and stage, and descriptors advanced as
-    // 32-bit words.  Both stages are issued by the same warp: products into different accumulators issued alternately
-    // (by two warps) ran several times slower than the same products issued stage by stage.
+    // An issuing warp is a single instruction stream: a satisfied mbarrier wait costs it some 140 cycles and a
+    // tcgen05.commit some 80, against 24 per tcgen05.mma (measured), while the tensor-core work of a chunk is a few
+    // hundred cycles.  Hence one wait and one commit per chunk and stage, descriptors advanced as 32-bit words, and
+    // one warp per stage: while one waits, commits and keeps its positions, the other issues.
     if (warp == 0) {
-        // ---------------- MMA issue ----------------
-        // Unit u: the k*k GDW products of chunk u into accumulator u & 1, then the PW products of chunk u-1, whose z
-        // the converter rounds meanwhile.  Accumulator u & 1 is free again once the converter has announced the slabs
-        // of chunk u-2 (it reads TMEM before that), which this warp waited for before the PW products of chunk u-2.
+        // ---------------- GDW issue ----------------
+        // Unit u: the k*k GDW products of chunk u into accumulator u & 1, which is free again once the converter has
+        // announced the slabs of chunk u-2 (it reads TMEM before that).
         const uint32_t a_hi = ((P.a_sbo >> 4) & 0x3FFFu) | (1u << 14) | kTcSw32;
         const uint32_t a_lo0 = ((x_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t b_lo0 = ((b_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t xstep = P.xslot_bytes >> 4, bstep = P.bbuf_bytes >> 4, pstep = P.bplane >> 4;
         const uint32_t rstep = P.tap_row_step >> 4, cstep = P.tap_col_step >> 4;
-        // The loop below is this warp's whole working set of instructions and is kept near a hundred of them (it has to
-        // stay in the small instruction cache next to the scheduler while the other warps of the block come and go):
-        // tap offsets live in registers, ring positions advance by a compare per slab, waits are calls when they miss.
+        // This warp is a single dependent instruction stream (a dozen cycles per instruction), so its loop is kept
+        // near a hundred instructions: tap offsets live in registers, waits are calls when they miss.
         uint32_t tap_a[K * K], tap_b[K * K];
 #pragma unroll
         for (int ur = 0; ur < K; ++ur)
@@ -342,8 +346,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         // Two warps per TMEM lane quarter; each takes every other 16-column granule of the chunk (at most 4), reads
         // them with one wait, rounds and stores them.  Warp 4's first lane also releases, on behalf of the GDW issue
         // warp, the B buffer and (after a window's last chunk) the input box that the chunk's products have read.
-        // The per-chunk code is a short loop over pairs of granules (it shares the scheduler's small instruction cache
-        // with the issue, builder and epilogue code of the same quarter), and its waits are calls when they miss.
+        // The per-chunk code is a short loop over pairs of granules, and its waits are calls when they miss.
         const int lg = warp & 3, half = (warp - 4) >> 2;
         const uint32_t r = (uint32_t)(lg * 32 + lane);
         const uint32_t sw = ((r >> 2) & 1u) << 4;           // 32-byte swizzle: address bit 4 ^= bit 7
@@ -759,7 +762,14 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
             if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_tc_kernel)");                         \
             attr_set[p->device & 63] = true;                                                                            \
         }                                                                                                               \
-        fused_tc_kernel<KK><<<grid, kTcThreads, smem, st>>>(P);                                                         \
+        cudaLaunchConfig_t cfg = {};                                                                                    \
+        cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(kTcThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st; \
+        cudaLaunchAttribute attr[1];                                                                                    \
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                                \
+        attr[0].val.programmaticStreamSerializationAllowed = 1;                                                         \
+        cfg.attrs = attr; cfg.numAttrs = 1;                                                                             \
+        e = cudaLaunchKernelEx(&cfg, fused_tc_kernel<KK>, P);                                                           \
+        if (e != cudaSuccess) return cuda_fail(e, "fused_tc_kernel launch");                                            \
     } while (0)
     switch (k) {
     case 1: GDWS_TC_LAUNCH(1); break;

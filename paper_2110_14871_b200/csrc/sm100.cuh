@@ -54,16 +54,22 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
+// Programmatic dependent launch.  grid_launch_dependents: the next kernel in the stream, if it was launched with
+// programmatic stream serialisation, may be scheduled once every block of this grid has executed this (or exited).
+// grid_dependency_wait: returns once the kernel before this one in the stream has completed and its writes are visible
+// (at once when this kernel was not launched with the attribute).  A kernel must execute it, in every thread that
+// touches global memory afterwards, before its first global access.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 // Bounded wait.  When the limit runs out (about a second) the thread records `code` in the
 // status word and raises the block's abort flag; from then on every wait in the block returns
 // at once, so that all threads still walk the same control flow, reach the common teardown
 // (barriers stay matched, TMEM is freed) and the kernel ends.  The first few thousand polls
 // are back to back (waits in the pipeline are short and a sleeping waiter wakes up late).
 constexpr uint32_t kSpinLimit = 1u << 22;
-// The waiting loops are kept out of line on purpose: a kernel's hot loops have to fit the small instruction cache
-// next to each scheduler (about 2 KB; measured: code that does not fit runs at the speed of instruction fetch, a
-// third of an instruction per cycle for a lone warp), and an inlined loop with its bookkeeping is some forty
-// instructions per wait.  Inline is only the first poll, which succeeds in the common case.
+// The waiting loops are kept out of line on purpose: inlined (and unrolled by the compiler) at every site they were a
+// third of a kernel's code, and code that the warps of an SM walk through runs at the speed of instruction fetch once it
+// exceeds some 32 KB (measured: gdws_measure_code_size).  Inline is only the first poll, which succeeds in the common case.
 static __device__ __noinline__ void mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t limit, volatile int *abort_flag, int *status, int code)
 {
     if (*abort_flag) return;
