@@ -95,6 +95,8 @@ struct DwShape {
 __global__ void gdw_bf16_kernel(DwShape s, const uint16_t *__restrict__ x, const float *__restrict__ dw,
                                 const int32_t *__restrict__ chan, uint16_t *__restrict__ z)
 {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int groups = s.Gpad / 8;
     const long long total = (long long)s.N * s.Ho * s.Wo * groups;
     for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total;
@@ -148,9 +150,9 @@ gdws_status_t bf16_depthwise(gdws_plan_s *p, const gdws_tensor_t *x, void *z, cu
     const long long total = (long long)s.N * s.Ho * s.Wo * (s.Gpad / 8);
     long long blocks = (total + 255) / 256;
     if (blocks > (long long)sm_count_of(p) * 32) blocks = (long long)sm_count_of(p) * 32;
-    gdw_bf16_kernel<<<(int)blocks, 256, 0, st>>>(s, (const uint16_t *)x->ptr, p->d_dw, p->d_chan, (uint16_t *)z);
+    cudaError_t e = launch_overlapped(gdw_bf16_kernel, (unsigned)blocks, 256u, 0, st, s, (const uint16_t *)x->ptr, (const float *)p->d_dw,
+                                      (const int32_t *)p->d_chan, (uint16_t *)z);
     p->launches++;
-    cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "gdw_bf16_kernel launch");
 }
 
@@ -197,10 +199,12 @@ __global__ void __launch_bounds__(kPwThreads, 1) pw_bf16_tc_kernel(const __grid_
         fence_mbar_init();
     }
     __syncwarp();
+    grid_launch_dependents();
     if (warp == 1) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    grid_dependency_wait();      // z comes from the kernel before this one in the stream
     const uint32_t tmem = tmem_slot;
     const int my_tiles = (P.ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
 
@@ -317,9 +321,8 @@ gdws_status_t bf16_pointwise(gdws_plan_s *p, const void *z, gdws_tensor_t *y, cu
         attr_set[p->device & 63] = true;
     }
     const int grid = (int)(tiles < p->sm_count ? tiles : p->sm_count);
-    pw_bf16_tc_kernel<<<grid, kPwThreads, smem, st>>>(P);
+    e = launch_overlapped(pw_bf16_tc_kernel, (unsigned)grid, kPwThreads, smem, st, P);
     p->launches++;
-    e = cudaGetLastError();
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "pw_bf16_tc_kernel launch");
 }
 

@@ -415,6 +415,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     const uint32_t w_s = x_s + (uint32_t)P.nslots * P.slot_bytes;         // ring of nwslots filter blocks
     int4 *meta_tab = reinterpret_cast<int4 *>(base + (w_s - a_s) + (size_t)P.nwslots * wblock);
 
+    grid_launch_dependents();      // the next kernel in the stream may start its prologue as SMs become free
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < 4; ++i) {
@@ -436,6 +437,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         fence_mbar_init();
     }
     if (!ZOUT && warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
+    // up to here only this block's shared and tensor memory were touched; the kernel before this one in the stream has
+    // to be complete before global memory is read or written
+    grid_dependency_wait();
     for (int q = tid; q < P.nchunks; q += kFusedThreads) meta_tab[q] = __ldg(P.chunk_meta + q);
     // a copy of the bias next to the chunk table: the epilogue reads it per 16 columns, with the accumulator in hand
     float *bias_sm = reinterpret_cast<float *>(meta_tab + P.nchunks);
@@ -803,8 +807,7 @@ static gdws_status_t launch_one(const FusedParams &P, int device, int grid, size
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_bf16_kernel)");
         attr_set[device & 63] = true;
     }
-    fused_bf16_kernel<K, MODE, S, PS, VAR><<<grid, kFusedThreads, smem, st>>>(P);
-    e = cudaGetLastError();
+    e = launch_overlapped(fused_bf16_kernel<K, MODE, S, PS, VAR>, (unsigned)grid, kFusedThreads, smem, st, P);
     return e == cudaSuccess ? GDWS_OK : cuda_fail(e, "fused_bf16_kernel launch");
 }
 

@@ -762,13 +762,7 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
             if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fused_tc_kernel)");                         \
             attr_set[p->device & 63] = true;                                                                            \
         }                                                                                                               \
-        cudaLaunchConfig_t cfg = {};                                                                                    \
-        cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(kTcThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st; \
-        cudaLaunchAttribute attr[1];                                                                                    \
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                                \
-        attr[0].val.programmaticStreamSerializationAllowed = 1;                                                         \
-        cfg.attrs = attr; cfg.numAttrs = 1;                                                                             \
-        e = cudaLaunchKernelEx(&cfg, fused_tc_kernel<KK>, P);                                                           \
+        e = launch_overlapped(fused_tc_kernel<KK>, (unsigned)grid, kTcThreads, smem, st, P);                              \
         if (e != cudaSuccess) return cuda_fail(e, "fused_tc_kernel launch");                                            \
     } while (0)
     switch (k) {

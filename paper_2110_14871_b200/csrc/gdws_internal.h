@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "gdws.h"
@@ -124,6 +125,21 @@ gdws_status_t fail(gdws_status_t st, const char *fmt, ...);
 gdws_status_t cuda_fail(cudaError_t e, const char *what);
 gdws_status_t ensure_device(gdws_plan_s *p);   // allocate device tables on the current device
 gdws_status_t check_arch();
+
+// Launch with programmatic stream serialisation: the kernel may be scheduled while the kernel before it in the stream
+// is still running (once all blocks of that one have executed griddepcontrol.launch_dependents, which the library's
+// kernels do first thing).  Such a kernel touches global memory only after its own griddepcontrol.wait.
+template <class... KArgs, class... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 // x and y of a forward call against the plan: pointers, alignment, extents, dtype/layout pair, no overlap
 gdws_status_t check_pair(const gdws_plan_s *p, const gdws_tensor_t *x, const gdws_tensor_t *y);
 // static_ws.cu: looks up (once per device, the device being current) the address of the built-in scratch array
