@@ -14,19 +14,24 @@
 //
 // One persistent block of 20 warps per SM walks over work items (tile of 128 output pixels x block of up to
 // 256 output channels).  Roles, coupled by mbarriers only:
-//   warp 0             issues the k*k GDW products of every chunk (one elected lane);
+//   warp 0             issues the k*k GDW products of every chunk (one elected lane) and, with commits of its own,
+//                      hands back the B buffer and the input box they have read;
 //   warp 3             issues the PW products of every chunk, once its z slabs and weights are in place;
 //   warp 1 (one lane)  fetches the input boxes by TMA (x as a rank-4 tensor: C, W, H, N; 16 channels per box);
-//   warp 2 (one lane)  streams the packed pointwise weights (bulk copies into a ring of 16-channel slabs);
-//   warps 4-11         converter: TMEM z -> bf16 -> ring of 16-channel operand slabs (two warps per lane quarter);
+//   warp 2 (one lane)  streams the packed pointwise weights (one bulk copy per chunk into a ring of 16-channel slabs);
+//   warps 4-11         converter: TMEM z -> bf16 -> 16-channel operand slabs; two groups of four warps (one per TMEM
+//                      lane quarter) that take alternate chunks;
 //   warps 12-15        epilogue: TMEM y -> bias, ReLU, bf16 -> global memory (TMA store or direct);
 //   warps 16-19        builder: one thread per intermediate channel of the chunk scatters its k*k taps into B
 //                      operand planes that are otherwise zero, and clears what it wrote when the buffer comes back.
+// A chunk's slabs are contiguous in the two rings (a chunk that does not fit behind its predecessor starts over at
+// slab 0), at places that are the same for every work item and come from a table computed at launch.
 // All operands are K-major with 32-byte rows and the 32-byte swizzle (address bit 4 ^= bit 7), 8-row groups
 // `stride byte offset` apart.  Every wait is bounded (see mbar_wait, tc_wait).
 #include <string.h>
 
 #include <algorithm>
+#include <vector>
 
 #include "sm100.cuh"
 
@@ -34,13 +39,12 @@ namespace gdws {
 
 static_assert(sizeof(TcChunk) == 32, "chunk table entries are copied as two 16-byte words");
 
-constexpr int kTcConvWarps = 8;        // converter warps 4 .. 11 (two per TMEM lane quarter)
-constexpr int kTcEpiWarp0 = 4 + kTcConvWarps, kTcBuildWarp0 = kTcEpiWarp0 + 4;
-constexpr int kTcThreads = (kTcBuildWarp0 + 4) * 32;
-static_assert(kTcEpiWarp0 % 4 == 0, "a warp reads the TMEM lanes of quarter warp % 4");
+constexpr int kTcConvWarp0 = 4, kTcConvWarps = 8;    // converter warps 4 .. 11: two groups of four (one warp per TMEM lane quarter)
+constexpr int kTcEpiWarp0 = kTcConvWarp0 + kTcConvWarps, kTcBuildWarp0 = kTcEpiWarp0 + 4, kTcBuildWarps = 4;
+constexpr int kTcThreads = (kTcBuildWarp0 + kTcBuildWarps) * 32;
 constexpr int kTcNU = 4;              // chunks in flight per ring (barriers per ring)
 static_assert(kTcNU == 4, "unit parity is taken from bit 2 of the unit index");
-constexpr int kTcMaxNB = 4;           // B operand buffers of the GDW stage (one chunk each: k*k planes)
+constexpr int kTcMaxNB = 4;           // B operand buffers of the GDW stage (one chunk each: k*k planes), up to two per chunk parity
 constexpr int kTcMaxNX = 4;           // input box slots
 constexpr int kTcMaxTaps = 25;
 constexpr int kTcZCol = 256;          // TMEM columns 256..511: two GDW accumulators of up to 128 columns
@@ -68,6 +72,10 @@ struct alignas(64) TcParams {
     uint32_t bbuf_bytes, bplane, xslot_bytes, wslab_bytes;
     uint32_t off_b, off_z, off_w, off_x, off_tab;    // from the 1024-aligned base; the output staging comes first
     int ostage, rec_hw, nslabs_total, bias_len;
+    // Per chunk of the work item, where its slabs sit in the two rings and which older chunk must have left them:
+    // bits 0-7 first z slab, 8-15 first weight slab, 16-18 / 19-21 how many units back the PW products must be done
+    // before the z slabs / the weight slabs are overwritten (0: no wait).  A chunk's slabs are contiguous (no wrap).
+    uint32_t ring[kTcMaxChunks];
 };
 
 // Bounded wait of every role but the issuing warps: each poll lets the hardware suspend the thread until the phase
@@ -99,7 +107,7 @@ template <int K>
 __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_constant__ TcParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    // dwready[4] | zfull[2] (2 unused) | pwready[4] pwdone[4] | bfree[4] xfree[4] | accfull[2] accfree[2]
+    // dwready[4] | zfull[2] (2 unused) | pwready[4] pwdone[4] | bfree[4] xfree[4] | accfull[2] accfree[2] | drain[2]
     __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4 + 2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -107,20 +115,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t base_s = smem_u32(base);
     const uint32_t o_s = base_s, b_s = base_s + P.off_b, z_s = base_s + P.off_z, w_s = base_s + P.off_w, x_s = base_s + P.off_x;
-    // dwready: the B operands (4 builder warps) and the input box (the loader's arrive, with the box's bytes when the
-    // chunk opens a window) of a chunk are in place.  zfull: its GDW products are done.  pwready: the chunk's z slabs
-    // (8 converter warps) and its pointwise weights (the loader's arrive with their bytes) are in place.  pwdone: its PW products are done.  bfree / xfree: arrived by the
-    // converter once the GDW products that read a B buffer / the last ones that read a box are done.
+    // dwready: the B operands (the 4 builder warps of the chunk's parity) and the input box (the loader's arrive, with the
+    // box's bytes when the chunk opens a window) of a chunk are in place.  zfull[h]: the GDW products of a chunk of parity h
+    // are done.  pwready: the chunk's z slabs (the 4 converter warps of its parity) and its pointwise weights (the loader's
+    // arrive with their bytes) are in place.  pwdone: its PW products are done.  bfree: arrived by a converter once the
+    // GDW products that read a B buffer are done.  xfree: two arrivals per window, after the GDW products of its last
+    // chunk and of the chunk before it (issued by the other warp) are done.
     const uint32_t bar_dwready = smem_u32(&bars[0]);
     const uint32_t bar_zfull = bar_dwready + 32;
     const uint32_t bar_pwready = bar_zfull + 32, bar_pwdone = bar_pwready + 8 * kTcNU;
     const uint32_t bar_bfree = bar_pwdone + 8 * kTcNU, bar_xfree = bar_bfree + 8 * kTcMaxNB;
     const uint32_t bar_accfull = bar_xfree + 8 * kTcMaxNX, bar_accfree = bar_accfull + 16;
-    const uint32_t bar_drain = bar_accfull + 32;       // the issue warp's last commit, awaited before TMEM is freed
+    const uint32_t bar_drain = bar_accfull + 32;       // the issuing warps' last commits, awaited before TMEM is freed
     volatile int *const vabort = &abort_flag;
     TcChunk *tab = reinterpret_cast<TcChunk *>(base + P.off_tab);
     float *bias_sm = reinterpret_cast<float *>(tab + P.nchunks);
-    uint16_t *bold = reinterpret_cast<uint16_t *>(bias_sm + P.Dpad_tot);     // [nb][128]: what each builder thread wrote last
+    uint16_t *bold = reinterpret_cast<uint16_t *>(bias_sm + P.Dpad_tot);     // [2 * nb][128]: what each builder thread wrote last
     const uint32_t bias_s = smem_u32(bias_sm);
 
     if (tid == 0) {
@@ -130,11 +140,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             mbar_init(bar_zfull + 8 * i, 1);
             mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4);
         }
-        for (int i = 0; i < kTcNU; ++i) { mbar_init(bar_pwready + 8 * i, kTcConvWarps + 1); mbar_init(bar_pwdone + 8 * i, 1); }
+        for (int i = 0; i < kTcNU; ++i) { mbar_init(bar_pwready + 8 * i, kTcConvWarps / 2 + 1); mbar_init(bar_pwdone + 8 * i, 1); }
         for (int i = 0; i < kTcMaxNB; ++i) mbar_init(bar_bfree + 8 * i, 1);
         for (int i = 0; i < kTcMaxNX; ++i) mbar_init(bar_xfree + 8 * i, 1);
-        mbar_init(bar_drain, 1);
-        mbar_init(bar_drain + 8, 1);
+        for (int i = 0; i < 2; ++i) mbar_init(bar_drain + 8 * i, 1);
         fence_mbar_init();
     }
     // The kernel that follows in the stream (launched with programmatic serialisation, as this one is) may start its
@@ -153,7 +162,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         grid_dependency_wait();
         const uint4 *src = reinterpret_cast<const uint4 *>(P.chunks);
         uint4 *dst = reinterpret_cast<uint4 *>(tab);
-        for (int i = tid; i < P.nchunks * 2; i += kTcThreads) dst[i] = __ldg(src + i);
+        for (int i = tid; i < P.nchunks * 2; i += kTcThreads) {
+            uint4 w4 = __ldg(src + i);
+            if (i & 1) w4.z = P.ring[i >> 1];        // second half of the entry: slab0, flags, places in the rings, (unused)
+            dst[i] = w4;
+        }
         for (int d = tid; d < P.Dpad_tot; d += kTcThreads) bias_sm[d] = d < P.bias_len ? __ldg(P.bias + d) : 0.f;
     }
     tc_fence_before();
@@ -166,21 +179,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const int tiles_hw = P.tiles_h * P.tiles_w;
     const uint32_t p_hi = (256u >> 4) | (1u << 14) | kTcSw32;   // descriptor high word: 8-row groups 256 bytes apart, version 1, 32-byte swizzle
 
-    // An issuing warp is a single instruction stream: a satisfied mbarrier wait costs it some 140 cycles and a
-    // tcgen05.commit some 80, against 24 per tcgen05.mma (measured), while the tensor-core work of a chunk is a few
-    // hundred cycles.  Hence one wait and one commit per chunk and stage, descriptors advanced as 32-bit words, and
-    // one warp per stage: while one waits, commits and keeps its positions, the other issues.
+    // A warp runs a dozen cycles per instruction on this control-heavy code (every step waits for the one before), so the
+    // code each role runs per chunk is kept short: slab positions come from a table instead of ring bookkeeping, the
+    // issuing warps release the buffers their products have read with commits of their own, and the converters, whose
+    // per-chunk work is the longest, take alternate chunks in two groups.
     if (warp == 0) {
         // ---------------- GDW issue ----------------
-        // Unit u: the k*k GDW products of chunk u into accumulator u & 1, which is free again once the converter has
-        // announced the slabs of chunk u-2 (it reads TMEM before that).
+        // Unit u: the k*k GDW products of chunk u into accumulator u & 1, which is free again once the converters have
+        // announced the slabs of chunk u - 2 (they read TMEM before that).  Three commits: the accumulator is full, the
+        // B buffer may be rebuilt, and (after a window's last chunk) the input box may be overwritten.
         const uint32_t a_hi = ((P.a_sbo >> 4) & 0x3FFFu) | (1u << 14) | kTcSw32;
         const uint32_t a_lo0 = ((x_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t b_lo0 = ((b_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t xstep = P.xslot_bytes >> 4, bstep = P.bbuf_bytes >> 4, pstep = P.bplane >> 4;
         const uint32_t rstep = P.tap_row_step >> 4, cstep = P.tap_col_step >> 4;
-        // This warp is a single dependent instruction stream (a dozen cycles per instruction), so its loop is kept
-        // near a hundred instructions: tap offsets live in registers, waits are calls when they miss.
         uint32_t tap_a[K * K], tap_b[K * K];
 #pragma unroll
         for (int ur = 0; ur < K; ++ur)
@@ -195,7 +207,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         for (int u = 0; u < total; ++u) {
             const int npad = tab[q].npad, flags = tab[q].flags;
             mbar_wait_call(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
-            // accumulator u & 1 held chunk u - 2: the converters have read it once they announce that chunk's slabs
             if (u >= 2) mbar_wait_call(bar_pwready + 8 * ((u - 2) & 3), (uint32_t)((u - 2) >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
             tc_fence_after();
             if (elect_one()) {
@@ -205,6 +216,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 for (int i = 0; i < K * K; ++i)
                     umma_bf16_words(d_z, a_lo + tap_a[i], a_hi, b_lo + tap_b[i], p_hi, idesc, i != 0);
                 umma_commit(bar_zfull + 8 * (u & 1));
+                umma_commit(bar_bfree + 8 * bslot);
+                if (flags & 2) umma_commit(bar_xfree + 8 * xslot);
             }
             __syncwarp();
             b_lo += bstep;
@@ -223,32 +236,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         }
         __syncwarp();
     } else if (warp == 3) {
-        // ---------------- PW issue ----------------
-        // A second issuing warp: while it waits, commits and keeps its ring positions, warp 0 issues the next chunk's GDW
-        // products, and the other way round.  The two streams of products go to different accumulators and may interleave.
+        // ---------------- PW issue, every chunk in order ----------------
         const uint32_t idesc_pw = make_idesc(P.Dloc, false);
         const uint32_t z_lo0 = ((z_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t w_lo0 = ((w_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t wstep = P.wslab_bytes >> 4;
-        uint32_t zh = 0, wh = 0, z_lo = z_lo0, w_lo = w_lo0, buf = 0, accpar = 1;
+        uint32_t buf = 0, accpar = 1;
         int qp = 0, itp = 0;
 #pragma unroll 1
         for (int v = 0; v < total; ++v) {
             const int ns = tab[qp].npad >> 4;
+            const uint32_t ring = (uint32_t)tab[qp].reserved0;
             if (qp == 0 && itp >= P.nacc) mbar_wait_call(bar_accfree + 8 * buf, accpar, &abort_flag, P.status, kStatusWaitStage);
             mbar_wait_call(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
             tc_fence_after();
-            const bool leader = elect_one();
-            const uint32_t d_y = tmem + buf * 128u;
-#pragma unroll 1
-            for (int s = 0; s < ns; ++s) {           // every lane keeps the ring positions, the leader issues
-                if (leader) umma_bf16_words(d_y, z_lo, p_hi, w_lo, p_hi, idesc_pw, (uint32_t)(qp | s));
-                z_lo += kTcSlab >> 4;
-                if (++zh == (uint32_t)P.nz) { zh = 0; z_lo = z_lo0; }
-                w_lo += wstep;
-                if (++wh == (uint32_t)P.nw) { wh = 0; w_lo = w_lo0; }
-            }
-            if (leader) {
+            if (elect_one()) {
+                const uint32_t d_y = tmem + buf * 128u;
+                const uint32_t z_lo = z_lo0 + (ring & 0xFFu) * (uint32_t)(kTcSlab >> 4);
+                const uint32_t w_lo = w_lo0 + ((ring >> 8) & 0xFFu) * wstep;
+#pragma unroll
+                for (int s = 0; s < 8; ++s)          // a chunk has at most 8 slabs
+                    if (s < ns) umma_bf16_words(d_y, z_lo + (uint32_t)s * (uint32_t)(kTcSlab >> 4), p_hi, w_lo + (uint32_t)s * wstep, p_hi, idesc_pw,
+                                                (uint32_t)(qp | s));
                 umma_commit(bar_pwdone + 8 * (v & 3));
                 if (qp == P.nchunks - 1) umma_commit(bar_accfull + 8 * buf);
             }
@@ -307,31 +316,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     } else if (warp == 2) {
         if (lane == 0) {
             // ---------------- pointwise-weight loader ----------------
-            SlabRing ring;
-            ring.free_slabs = P.nw;
             int q = 0, it = 0, issued = 0;
 #pragma unroll 1
             for (int v = 0; v < total; ++v) {
-                const TcChunk ch = tab[q];
-                const int ns = ch.npad >> 4;
-#pragma unroll 1
-                while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
-                    const int o = ring.oldest;
-                    tc_wait(bar_pwdone + 8 * (o & 3), (uint32_t)(o >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
-                    ring.free_slabs += tab[o % P.nchunks].npad >> 4;
-                    ++ring.oldest;
-                }
+                const int ns = tab[q].npad >> 4, slab0 = tab[q].slab0;
+                const uint32_t ring = (uint32_t)tab[q].reserved0;
+                // the chunk's place in the ring was last used wdep units ago (1 .. 4, which also keeps the four pwready
+                // barriers apart): the PW products of that chunk must be done
+                const int wdep = (int)((ring >> 19) & 7u);
+                if (v >= wdep) tc_wait(bar_pwdone + 8 * ((v - wdep) & 3), (uint32_t)((v - wdep) >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
                 if (*vabort) break;                            // a wait ran out somewhere: no new copies
                 issued = v + 1;
-                const int part = ((int)blockIdx.x + it * (int)gridDim.x) % P.nparts;
+                const int part = P.nparts == 1 ? 0 : ((int)blockIdx.x + it * (int)gridDim.x) % P.nparts;
                 const uint32_t bar = bar_pwready + 8 * (v & 3);
                 mbar_expect_tx(bar, (uint32_t)ns * P.wslab_bytes);
-                const uint16_t *src = P.pw + ((size_t)part * P.nslabs_total + ch.slab0) * 16 * P.Dloc;
-                const int first = ns < P.nw - ring.head ? ns : P.nw - ring.head;
-                bulk_g2s(w_s + (uint32_t)ring.head * P.wslab_bytes, src, (uint32_t)first * P.wslab_bytes, bar);
-                if (first < ns) bulk_g2s(w_s, src + (size_t)first * 16 * P.Dloc, (uint32_t)(ns - first) * P.wslab_bytes, bar);
-                ring.head = (ring.head + ns) % P.nw;
-                ring.free_slabs -= ns;
+                const uint16_t *src = P.pw + ((size_t)part * P.nslabs_total + slab0) * 16 * P.Dloc;
+                bulk_g2s(w_s + ((ring >> 8) & 0xFFu) * P.wslab_bytes, src, (uint32_t)ns * P.wslab_bytes, bar);
                 if (++q == P.nchunks) { q = 0; ++it; }
             }
             // Teardown: the last phase armed on each pwready barrier completes when its weights have landed and the
@@ -341,73 +341,59 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 mbar_wait_drain(bar_pwready + 8 * (v & 3), (uint32_t)(v >> 2) & 1u);
             }
         }
-    } else if (warp >= 4 && warp < 4 + kTcConvWarps) {
+    } else if (warp >= kTcConvWarp0 && warp < kTcConvWarp0 + kTcConvWarps) {
         // ---------------- converter: z (fp32, TMEM) -> bf16 operand slabs ----------------
-        // Two warps per TMEM lane quarter; each takes every other 16-column granule of the chunk (at most 4), reads
-        // them with one wait, rounds and stores them.  Warp 4's first lane also releases, on behalf of the GDW issue
-        // warp, the B buffer and (after a window's last chunk) the input box that the chunk's products have read.
-        // The per-chunk code is a short loop over pairs of granules, and its waits are calls when they miss.
-        const int lg = warp & 3, half = (warp - 4) >> 2;
+        // Group grp (four warps, one per TMEM lane quarter) takes the chunks of parity grp: it reads the chunk's
+        // accumulator granule by granule (16 columns; the next granule's load is in flight while one is rounded and
+        // stored) and writes the slabs the table names.
+        const int lg = warp & 3, grp = (warp - kTcConvWarp0) >> 2;
         const uint32_t r = (uint32_t)(lg * 32 + lane);
         const uint32_t sw = ((r >> 2) & 1u) << 4;           // 32-byte swizzle: address bit 4 ^= bit 7
         const uint32_t row_s = z_s + r * 32u;
-        SlabRing ring;
-        ring.free_slabs = P.nz;
-        uint32_t bslot = 0, xslot = 0;
-        int q = 0, qo = 0;                                   // chunk index of unit v and of the ring's oldest unit
+        const uint32_t taddr = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(kTcZCol + 128 * grp);
+        int q = 0;
+        auto round_store = [&](const uint32_t (&acc)[16], uint32_t addr) {
+            uint4 lo, hi;
+            lo.x = pack_bf16x2(__uint_as_float(acc[0]), __uint_as_float(acc[1]));
+            lo.y = pack_bf16x2(__uint_as_float(acc[2]), __uint_as_float(acc[3]));
+            lo.z = pack_bf16x2(__uint_as_float(acc[4]), __uint_as_float(acc[5]));
+            lo.w = pack_bf16x2(__uint_as_float(acc[6]), __uint_as_float(acc[7]));
+            hi.x = pack_bf16x2(__uint_as_float(acc[8]), __uint_as_float(acc[9]));
+            hi.y = pack_bf16x2(__uint_as_float(acc[10]), __uint_as_float(acc[11]));
+            hi.z = pack_bf16x2(__uint_as_float(acc[12]), __uint_as_float(acc[13]));
+            hi.w = pack_bf16x2(__uint_as_float(acc[14]), __uint_as_float(acc[15]));
+            sts128(addr + sw, lo);                 // channels 0 .. 7 of the slab for this pixel
+            sts128(addr + (sw ^ 16u), hi);         // channels 8 .. 15
+        };
 #pragma unroll 1
         for (int v = 0; v < total; ++v) {
-            const int ns = tab[q].npad >> 4, flags = tab[q].flags;
+            const int ns = tab[q].npad >> 4;
+            if ((v & 1) == grp) {
+                const uint32_t ring = (uint32_t)tab[q].reserved0;
+                const int zdep = (int)((ring >> 16) & 7u);
+                if (zdep && v >= zdep)
+                    tc_warp_wait_call(bar_pwdone + 8 * ((v - zdep) & 3), (uint32_t)((v - zdep) >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                tc_warp_wait_call(bar_zfull + 8 * grp, (uint32_t)(v >> 1) & 1u, &abort_flag, P.status, kStatusWaitMma);
+                tc_fence_after();
+                uint32_t addr = row_s + (ring & 0xFFu) * (uint32_t)kTcSlab;
+                uint32_t acc0[16], acc1[16];
+                tmem_ld16(taddr, acc0);
 #pragma unroll 1
-            while ((ring.free_slabs < ns || v - ring.oldest >= kTcNU) && ring.oldest < v) {
-                const int o = ring.oldest;
-                tc_warp_wait_call(bar_pwdone + 8 * (o & 3), (uint32_t)(o >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
-                ring.free_slabs += tab[qo].npad >> 4;
-                if (++qo == P.nchunks) qo = 0;
-                ++ring.oldest;
-            }
-            tc_warp_wait_call(bar_zfull + 8 * (v & 1), (uint32_t)(v >> 1) & 1u, &abort_flag, P.status, kStatusWaitMma);
-            if (warp == 4 && lane == 0) {
-                mbar_arrive(bar_bfree + 8 * bslot);
-                if (flags & 2) mbar_arrive(bar_xfree + 8 * xslot);
-            }
-            if (++bslot == (uint32_t)P.nb) bslot = 0;
-            if (flags & 2) { if (++xslot == (uint32_t)P.nx) xslot = 0; }
-            tc_fence_after();
-            const uint32_t taddr = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(kTcZCol + 128 * (v & 1));
-#pragma unroll 1
-            for (int g = half; g < ns; g += 4) {             // this warp's granules g and g + 2 with one wait
-                uint32_t acc[2][16];
-                const bool two = g + 2 < ns;
-                tmem_ld16(taddr + (uint32_t)(g * 16), acc[0]);
-                if (two) tmem_ld16(taddr + (uint32_t)((g + 2) * 16), acc[1]);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    if (j == 0 || two) {
-                        uint4 lo, hi;
-                        lo.x = pack_bf16x2(__uint_as_float(acc[j][0]), __uint_as_float(acc[j][1]));
-                        lo.y = pack_bf16x2(__uint_as_float(acc[j][2]), __uint_as_float(acc[j][3]));
-                        lo.z = pack_bf16x2(__uint_as_float(acc[j][4]), __uint_as_float(acc[j][5]));
-                        lo.w = pack_bf16x2(__uint_as_float(acc[j][6]), __uint_as_float(acc[j][7]));
-                        hi.x = pack_bf16x2(__uint_as_float(acc[j][8]), __uint_as_float(acc[j][9]));
-                        hi.y = pack_bf16x2(__uint_as_float(acc[j][10]), __uint_as_float(acc[j][11]));
-                        hi.z = pack_bf16x2(__uint_as_float(acc[j][12]), __uint_as_float(acc[j][13]));
-                        hi.w = pack_bf16x2(__uint_as_float(acc[j][14]), __uint_as_float(acc[j][15]));
-                        int slab = ring.head + g + 2 * j;
-                        if (slab >= P.nz) slab -= P.nz;
-                        const uint32_t addr = row_s + (uint32_t)slab * kTcSlab;
-                        sts128(addr + sw, lo);                 // channels 0 .. 7 of the slab for this pixel
-                        sts128(addr + (sw ^ 16u), hi);         // channels 8 .. 15
+                for (int g = 0; g < ns; g += 2) {
+                    tmem_ld_wait();
+                    if (g + 1 < ns) tmem_ld16(taddr + (uint32_t)((g + 1) * 16), acc1);
+                    round_store(acc0, addr);
+                    if (g + 1 < ns) {
+                        tmem_ld_wait();
+                        if (g + 2 < ns) tmem_ld16(taddr + (uint32_t)((g + 2) * 16), acc0);
+                        round_store(acc1, addr + (uint32_t)kTcSlab);
                     }
+                    addr += 2u * (uint32_t)kTcSlab;
                 }
+                fence_proxy_async();
+                tc_fence_before();
+                tc_warp_arrive(bar_pwready + 8 * (v & 3));
             }
-            fence_proxy_async();
-            tc_fence_before();
-            tc_warp_arrive(bar_pwready + 8 * (v & 3));
-            ring.head += ns;
-            if (ring.head >= P.nz) ring.head -= P.nz;
-            ring.free_slabs -= ns;
             if (++q == P.nchunks) q = 0;
         }
     } else if (warp >= kTcEpiWarp0 && warp < kTcEpiWarp0 + 4) {
@@ -641,6 +627,33 @@ bool tc_geometry(const gdws_plan_s *p, int n, int Ho, int Wo, TcGeom *out)
     return found;
 }
 
+// Places of the chunks' slabs in a ring of `cap` slabs, the same for every work item: a chunk's slabs are contiguous,
+// and a chunk that does not fit behind its predecessor starts over at slab 0.  dep[q] = how many units before chunk q
+// the last chunk that used any of its slabs ran (in steady state, work item after work item), at most 4: the four
+// barriers of a ring are reused every four units, so a producer never runs further ahead than that anyway.
+bool tc_ring_places(const std::vector<TcChunk> &chunks, int cap, std::vector<int> *pos, std::vector<int> *dep)
+{
+    const int n = (int)chunks.size();
+    pos->assign(n, 0);
+    dep->assign(n, 4);
+    int head = 0;
+    for (int q = 0; q < n; ++q) {
+        const int ns = chunks[q].npad / 16;
+        if (ns > cap) return false;
+        if (head + ns > cap) head = 0;
+        (*pos)[q] = head;
+        head += ns;
+    }
+    std::vector<int> last(cap, -1000000);
+    for (int v = 0; v < 3 * n; ++v) {
+        const int q = v % n, ns = chunks[q].npad / 16;
+        int newest = -1000000;
+        for (int s2 = (*pos)[q]; s2 < (*pos)[q] + ns; ++s2) { newest = std::max(newest, last[s2]); last[s2] = v; }
+        if (v >= 2 * n) (*dep)[q] = std::max(1, std::min(4, v - newest));
+    }
+    return true;
+}
+
 }  // namespace
 
 gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t st)
@@ -681,15 +694,22 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
                     if (fixed + (size_t)m * P.wslab_bytes > (size_t)kMaxSmem) continue;
                     int nw = (int)(((size_t)kMaxSmem - fixed) / P.wslab_bytes);
                     if (nw > 3 * m) nw = 3 * m;
-                    // First two chunks of z slabs (the converter writes one while the PW products of the one before are
-                    // pending: with less, conversion and PW products of consecutive chunks serialise -- seen in a cycle
-                    // trace), then two chunks of weights, then the rest.
+                    // First two chunks of z slabs (one is converted while the PW products of the one before are pending)
+                    // and of weights, then a second B buffer per parity (a chunk's operands are built while the products
+                    // of the chunk before it run), then the rest.
                     const double score = 10.0 * std::min(nz, 2 * m) / m + 6.0 * std::min(nw, 2 * m) / m + 1.0 * std::min(nw, 3 * m) / m +
                                          0.5 * nz / m + 0.8 * ost + 0.6 * nb + 0.3 * nx;
                     if (score > best_score) { best_score = score; b_ost = ost; b_nx = nx; b_nb = nb; b_nz = nz; b_nw = nw; }
                 }
     if (best_score < 0) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: shared memory does not fit this layer");
     P.ostage = b_ost ? 16384 : 0; P.nx = b_nx; P.nb = b_nb; P.nz = b_nz; P.nw = b_nw;
+    {
+        std::vector<int> zpos, zdep, wpos, wdep;
+        if (!tc_ring_places(p->tc_chunks, P.nz, &zpos, &zdep) || !tc_ring_places(p->tc_chunks, P.nw, &wpos, &wdep))
+            return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: a chunk does not fit the slab rings");
+        for (int q = 0; q < nchunks; ++q)
+            P.ring[q] = (uint32_t)zpos[q] | ((uint32_t)wpos[q] << 8) | ((uint32_t)zdep[q] << 16) | ((uint32_t)wdep[q] << 19);
+    }
     P.off_b = (uint32_t)P.ostage;
     P.off_z = P.off_b + (uint32_t)P.nb * P.bbuf_bytes;
     P.off_w = P.off_z + (uint32_t)P.nz * kTcSlab;
