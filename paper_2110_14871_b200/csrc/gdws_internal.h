@@ -155,7 +155,9 @@ inline size_t dtype_size(gdws_dtype_t d) { return d == GDWS_F32 ? 4 : 2; }
 inline int gdw_stage_of(const gdws_plan_s *p)
 {
     if (p->opt_dw_math == 1 || p->opt_dw_math == 2) return p->opt_dw_math;
-    return (p->tc_ok && p->k == 3 && p->stride == 1 && p->Dpad <= 256 && p->G >= 4 * p->C) ? 2 : 1;
+    if (!(p->tc_ok && p->k == 3 && p->stride == 1 && p->Dpad <= 256)) return 1;
+    // average multiplier of at least 4, or of at least 2.7 when the PW products are small (at most 128 output channels)
+    return (p->G >= 4 * p->C || (p->Dpad <= 128 && 10 * (long long)p->G >= 27 * (long long)p->C)) ? 2 : 1;
 }
 
 // SMs of the plan's device; a plan built without a device (host-side queries only) assumes a B200's 148.
