@@ -53,7 +53,9 @@ constexpr int kTcSlab = 4096;         // bytes of one z slab: 128 pixels x 16 ch
 constexpr int kTcMaxChunks = 256;
 
 struct alignas(64) TcParams {
-    CUtensorMap tmap_x;          // x as (C, W, H, N) bf16, box (16, IW, rows, TN), 32-byte swizzle
+    CUtensorMap tmap_xp[4];      // x as (C, W, H, N) bf16, box (16, IW, rows, TN), 32-byte swizzle; with stride 2 one map per
+                                 // parity of the input row and column (index 2 * row parity + column parity), each a dense
+                                 // (C, W/2, H/2, N) view of every other row and column
     CUtensorMap tmap_y;          // y as (D, Wo, Ho, N) bf16, box (64, PW, PH, TN), 128-byte swizzle (when ostage != 0)
     uint16_t *y;
     const uint16_t *filt;
@@ -64,9 +66,9 @@ struct alignas(64) TcParams {
     int N, Ho, Wo, D, Dloc, Dpad_tot, nparts, nchunks, pad, relu;
     int TN, PH, PW, tiles_h, tiles_w, nitems;
     int nloads, xbox_bytes;
-    int load_dw[kTcMaxTaps], load_dh[kTcMaxTaps];
+    int load_dw[kTcMaxTaps], load_dh[kTcMaxTaps], load_map[kTcMaxTaps];   // per copy of the box: start relative to the tile's first output pixel, which map
     uint32_t load_off[kTcMaxTaps];
-    uint32_t tap_row_step, tap_col_step;   // the A operand of tap (u, v) starts u * row_step + v * col_step bytes into the box
+    uint32_t tap_off[kTcMaxTaps];          // the A operand of tap (u, v) starts this many bytes into the box slot
     uint32_t a_sbo;              // GDW A operand: bytes between 8-pixel groups
     int nb, nx, nz, nw, nacc;
     uint32_t bbuf_bytes, bplane, xslot_bytes, wslab_bytes;
@@ -192,13 +194,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         const uint32_t a_lo0 = ((x_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t b_lo0 = ((b_s & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t xstep = P.xslot_bytes >> 4, bstep = P.bbuf_bytes >> 4, pstep = P.bplane >> 4;
-        const uint32_t rstep = P.tap_row_step >> 4, cstep = P.tap_col_step >> 4;
         uint32_t tap_a[K * K], tap_b[K * K];
 #pragma unroll
         for (int ur = 0; ur < K; ++ur)
 #pragma unroll
             for (int v = 0; v < K; ++v) {
-                tap_a[ur * K + v] = (uint32_t)ur * rstep + (uint32_t)v * cstep;
+                tap_a[ur * K + v] = P.tap_off[ur * K + v] >> 4;
                 tap_b[ur * K + v] = (uint32_t)(ur * K + v) * pstep;
             }
         uint32_t xslot = 0, bslot = 0, a_lo = a_lo0, b_lo = b_lo0;
@@ -285,7 +286,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 const int bn = tile / tiles_hw;
                 tile -= bn * tiles_hw;
                 const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
-                const int n0 = bn * P.TN, hi0 = bh * P.PH - P.pad, wi0 = bw * P.PW - P.pad;
+                const int n0 = bn * P.TN, hi0 = bh * P.PH, wi0 = bw * P.PW;     // the copies' offsets carry the padding
 #pragma unroll 1
                 for (int q = 0; q < P.nchunks; ++q, ++u) {
                     const int cbase = tab[q].cbase, flags = tab[q].flags;
@@ -300,7 +301,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     const uint32_t dst = x_s + xslot * P.xslot_bytes;
 #pragma unroll 1
                     for (int l = 0; l < P.nloads; ++l)
-                        tma_load_4d(dst + P.load_off[l], &P.tmap_x, cbase, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, bar);
+                        tma_load_4d(dst + P.load_off[l], &P.tmap_xp[P.load_map[l]], cbase, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, bar);
                     ++box;
                     if (++xslot == (uint32_t)P.nx) xslot = 0;
                 }
@@ -594,27 +595,58 @@ void tc_pack(gdws_plan_s *p, const void *dw_w, const void *pw_w, int is_bf16, cu
 // ------------------------------------------------------------------------------------------
 namespace {
 
+// Input row h = stride * ho + u - pad of filter row u (columns alike).  With stride 2 the input is read through four
+// dense views, one per parity of row and column (every other row, every other column): in the view of parity par
+// filter row u reads row ho + off of the view, which turns the strided access into a unit-stride one.
+struct TcTaps {
+    int par[5] = {}, off[5] = {};          // per filter row (the filter is square and padded alike: same for columns)
+    int omin[2] = {}, omax[2] = {};        // per parity: smallest and largest offset
+    bool used[2] = {};
+    int ext = 0;                           // halo of a copy: the largest omax - omin
+    int npar = 0;
+};
+
+TcTaps tc_taps(int k, int stride, int pad)
+{
+    TcTaps t;
+    for (int par = 0; par < 2; ++par) { t.omin[par] = 1 << 20; t.omax[par] = -(1 << 20); }
+    for (int u = 0; u < k; ++u) {
+        const int i = u - pad;
+        const int par = ((i % stride) + stride) % stride;
+        t.par[u] = par; t.off[u] = (i - par) / stride;
+        t.used[par] = true;
+        t.omin[par] = std::min(t.omin[par], t.off[u]); t.omax[par] = std::max(t.omax[par], t.off[u]);
+    }
+    for (int par = 0; par < 2; ++par)
+        if (t.used[par]) { t.ext = std::max(t.ext, t.omax[par] - t.omin[par]); ++t.npar; }
+    return t;
+}
+
 struct TcGeom {
-    int layout = 0;              // 1: one box with halo rows (one image per tile), 2: one copy per filter row,
-                                 // 3: one copy per tap (maps at most 4 wide)
-    int TN = 0, PH = 0, PW = 0, IW = 0;
+    int layout = 0;              // 1: boxes with halo rows (one image per tile; one box per parity pair), 2: one copy per
+                                 // filter row and column parity, 3: one copy per tap (maps at most 4 wide)
+    int TN = 0, PH = 0, PW = 0, IW = 0, IH = 0;
     int tiles_n = 0, tiles_h = 0, tiles_w = 0;
-    int nloads = 0, xbox = 0;
+    int nloads = 0, xbox = 0, copy = 0;     // copies per box, bytes of a box, bytes of one copy (in shared memory: a multiple of 256)
     int64_t tiles() const { return (int64_t)tiles_n * tiles_h * tiles_w; }
 };
 
 bool tc_geometry(const gdws_plan_s *p, int n, int Ho, int Wo, TcGeom *out)
 {
     const int k = p->k;
+    const TcTaps t = tc_taps(k, p->stride, p->pad);
     double best = 1e300;
     bool found = false;
     auto consider = [&](int layout, int TN, int PH, int PW) {
         TcGeom g;
         g.layout = layout; g.TN = TN; g.PH = PH; g.PW = PW;
         g.tiles_n = (n + TN - 1) / TN; g.tiles_h = (Ho + PH - 1) / PH; g.tiles_w = (Wo + PW - 1) / PW;
-        g.IW = layout == 3 ? 4 : PW + k - 1;
-        g.nloads = layout == 1 ? 1 : (layout == 2 ? k : k * k);
-        g.xbox = layout == 1 ? 2 * (PH + k - 1) * g.IW * 16 : (layout == 2 ? k * 2 * 16 * g.IW * 16 : k * k * 4096);
+        g.IW = layout == 3 ? 4 : PW + t.ext;
+        g.IH = layout == 1 ? PH + t.ext : PH;
+        g.nloads = layout == 1 ? t.npar * t.npar : (layout == 2 ? k * t.npar : k * k);
+        g.copy = (TN * g.IH * g.IW * 32 + 255) / 256 * 256;
+        g.xbox = g.nloads * g.copy;
+        if (g.nloads > kTcMaxTaps) return;
         const double cost = (double)g.tiles() * (1.0 + 0.02 * (g.nloads - 1));
         if (cost < best) { best = cost; *out = g; found = true; }
     };
@@ -658,7 +690,7 @@ bool tc_ring_places(const std::vector<TcChunk> &chunks, int cap, std::vector<int
 
 gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_t *y, cudaStream_t st)
 {
-    if (!p->tc_ok) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: layer not covered (stride 1, k <= 5, C and D multiples of 8)");
+    if (!p->tc_ok) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: layer not covered (stride 1 or 2, k <= 5, C and D multiples of 8)");
     const int nchunks = (int)p->tc_chunks.size();
     if (nchunks > kTcMaxChunks) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: %d chunks (at most %d)", nchunks, kTcMaxChunks);
     if (p->sm_count <= 0) {
@@ -719,17 +751,25 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     if (smem < (size_t)kMaxSmem / 2 + 4096) smem = (size_t)kMaxSmem / 2 + 4096;   // one block per SM: it owns all of TMEM
     if (smem > (size_t)kMaxSmem) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: shared memory plan exceeds the limit");
 
-    {   // x as a rank-4 tensor, innermost first: channels, width, height, batch; a box holds 16 channels (32 bytes) per pixel
-        const cuuint64_t dims[4] = {(cuuint64_t)p->C, (cuuint64_t)x->w, (cuuint64_t)x->h, (cuuint64_t)x->n};
-        const cuuint64_t strides[3] = {(cuuint64_t)p->C * 2, (cuuint64_t)x->w * p->C * 2, (cuuint64_t)x->h * x->w * p->C * 2};
-        cuuint32_t box[4] = {16, (cuuint32_t)g.IW, 0, (cuuint32_t)g.TN};
-        box[2] = (cuuint32_t)(g.layout == 1 ? g.PH + k - 1 : g.PH);
-        const cuuint32_t estr[4] = {1, 1, 1, 1};
-        const CUresult r = encode(&P.tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, x->ptr, dims, strides, box, estr,
-                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
-                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled (x) failed with code %d", (int)r);
-    }
+    const int sd = p->stride;
+    const TcTaps taps = tc_taps(k, sd, p->pad);
+    for (int hp = 0; hp < sd; ++hp)
+        for (int wp = 0; wp < sd; ++wp) {
+            if (!taps.used[hp] || !taps.used[wp]) continue;
+            // x as a rank-4 tensor, innermost first: channels, width, height, batch; a box holds 16 channels (32 bytes) per
+            // pixel.  With stride 2: the rows of parity hp and the columns of parity wp only.
+            const int Wp = (x->w - wp + sd - 1) / sd, Hp = (x->h - hp + sd - 1) / sd;
+            if (Wp <= 0 || Hp <= 0) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: input too small for stride %d", sd);
+            const cuuint64_t dims[4] = {(cuuint64_t)p->C, (cuuint64_t)Wp, (cuuint64_t)Hp, (cuuint64_t)x->n};
+            const cuuint64_t strides[3] = {(cuuint64_t)sd * p->C * 2, (cuuint64_t)sd * x->w * p->C * 2, (cuuint64_t)x->h * x->w * p->C * 2};
+            const cuuint32_t box[4] = {16, (cuuint32_t)g.IW, (cuuint32_t)g.IH, (cuuint32_t)g.TN};
+            const cuuint32_t estr[4] = {1, 1, 1, 1};
+            void *base = (uint8_t *)x->ptr + ((size_t)hp * x->w + wp) * p->C * 2;
+            const CUresult r = encode(&P.tmap_xp[hp * 2 + wp], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr,
+                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
+                                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled (x) failed with code %d", (int)r);
+        }
     if (P.ostage) {
         const cuuint64_t dims[4] = {(cuuint64_t)p->D, (cuuint64_t)Wo, (cuuint64_t)Ho, (cuuint64_t)x->n};
         const cuuint64_t strides[3] = {(cuuint64_t)p->D * 2, (cuuint64_t)Wo * p->D * 2, (cuuint64_t)Ho * Wo * p->D * 2};
@@ -740,29 +780,58 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
                                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(GDWS_ERR_CUDA, "cuTensorMapEncodeTiled (y) failed with code %d", (int)r);
     } else {
-        P.tmap_y = P.tmap_x;
+        P.tmap_y = P.tmap_xp[taps.used[0] ? 0 : 3];
     }
     // Where each copy of the box goes, and where the A operand of tap (u, v) starts.
     const uint32_t px = 32;      // bytes of one staged pixel (16 channels)
+    int nl = 0;
     if (g.layout == 1) {
-        P.nloads = 1; P.load_dw[0] = 0; P.load_dh[0] = 0; P.load_off[0] = 0;
-        P.a_sbo = 8u * (uint32_t)g.IW * px / 8u;
-        P.tap_row_step = (uint32_t)g.IW * px; P.tap_col_step = px;
-    } else if (g.layout == 2) {
-        const uint32_t copy = 16u * (uint32_t)g.IW * px;
-        P.nloads = k;
-        for (int u = 0; u < k; ++u) { P.load_dw[u] = 0; P.load_dh[u] = u; P.load_off[u] = (uint32_t)u * copy; }
+        int idx[2][2] = {{-1, -1}, {-1, -1}};
+        for (int hp = 0; hp < sd; ++hp)
+            for (int wp = 0; wp < sd; ++wp) {
+                if (!taps.used[hp] || !taps.used[wp]) continue;
+                idx[hp][wp] = nl;
+                P.load_map[nl] = hp * 2 + wp; P.load_dh[nl] = taps.omin[hp]; P.load_dw[nl] = taps.omin[wp];
+                P.load_off[nl] = (uint32_t)nl * (uint32_t)g.copy;
+                ++nl;
+            }
+        for (int u = 0; u < k; ++u)
+            for (int v = 0; v < k; ++v) {
+                const int hp = taps.par[u], wp = taps.par[v];
+                P.tap_off[u * k + v] = P.load_off[idx[hp][wp]] +
+                                       (uint32_t)((taps.off[u] - taps.omin[hp]) * g.IW + (taps.off[v] - taps.omin[wp])) * px;
+            }
         P.a_sbo = (uint32_t)g.IW * px;
-        P.tap_row_step = copy; P.tap_col_step = px;
+    } else if (g.layout == 2) {
+        int idx[5][2];
+        for (int u = 0; u < k; ++u)
+            for (int wp = 0; wp < sd; ++wp) {
+                if (!taps.used[wp]) continue;
+                idx[u][wp] = nl;
+                P.load_map[nl] = taps.par[u] * 2 + wp; P.load_dh[nl] = taps.off[u]; P.load_dw[nl] = taps.omin[wp];
+                P.load_off[nl] = (uint32_t)nl * (uint32_t)g.copy;
+                ++nl;
+            }
+        for (int u = 0; u < k; ++u)
+            for (int v = 0; v < k; ++v) {
+                const int wp = taps.par[v];
+                P.tap_off[u * k + v] = P.load_off[idx[u][wp]] + (uint32_t)(taps.off[v] - taps.omin[wp]) * px;
+            }
+        P.a_sbo = (uint32_t)g.IW * px;
     } else {
-        P.nloads = k * k;
-        for (int u = 0; u < k; ++u) for (int v = 0; v < k; ++v) {
-            P.load_dw[u * k + v] = v; P.load_dh[u * k + v] = u; P.load_off[u * k + v] = (uint32_t)(u * k + v) * 4096u;
-        }
-        P.tap_row_step = (uint32_t)k * 4096u; P.tap_col_step = 4096u;
+        for (int u = 0; u < k; ++u)
+            for (int v = 0; v < k; ++v) {
+                P.load_map[nl] = taps.par[u] * 2 + taps.par[v]; P.load_dh[nl] = taps.off[u]; P.load_dw[nl] = taps.off[v];
+                P.load_off[nl] = (uint32_t)nl * (uint32_t)g.copy;
+                P.tap_off[u * k + v] = P.load_off[nl];
+                ++nl;
+            }
         P.a_sbo = 256u;
     }
-    P.xbox_bytes = g.xbox;
+    if (nl != g.nloads) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: internal error in the box plan");
+    P.nloads = nl;
+    // bytes that arrive per box: every copy delivers its full box (positions outside the image are zero-filled)
+    P.xbox_bytes = nl * g.TN * g.IH * g.IW * 32;
     P.y = (uint16_t *)y->ptr; P.filt = p->d_tc_filt; P.pw = p->d_tc_pw; P.bias = p->d_bias; P.chunks = p->d_tc_chunks;
     P.status = p->d_status;
     P.N = x->n; P.Ho = Ho; P.Wo = Wo; P.D = p->D; P.Dloc = Dloc; P.Dpad_tot = p->tc_nparts * Dloc; P.nparts = p->tc_nparts;

@@ -150,12 +150,13 @@ inline size_t dtype_size(gdws_dtype_t d) { return d == GDWS_F32 ? 4 : 2; }
 
 // Where the fused bf16 kernel runs the GDW stage: 1 = ALUs, 2 = tensor cores.  With the option left at 0 the
 // tensor cores are taken where they measured faster on B200: their cost is k*k products per 16-channel window
-// whatever the multipliers, the ALU kernel's is proportional to G, and beyond 256 output channels the PW
-// accumulator leaves no room for a second GDW accumulator.
+// whatever the multipliers, the ALU kernel's is proportional to G (and its stride-2 code reuses less of each input
+// row), and beyond 256 output channels the tensor-core kernel computes the GDW stage once per 256 of them.
 inline int gdw_stage_of(const gdws_plan_s *p)
 {
     if (p->opt_dw_math == 1 || p->opt_dw_math == 2) return p->opt_dw_math;
-    if (!(p->tc_ok && p->k == 3 && p->stride == 1 && p->Dpad <= 256)) return 1;
+    if (!(p->tc_ok && p->k == 3 && p->stride <= 2)) return 1;
+    if (p->stride == 1 && p->Dpad > 256) return 1;     // measured equal or slower there; with stride 2 faster at D = 512 too
     // average multiplier of at least 4, or of at least 2.7 when the PW products are small (at most 128 output channels)
     return (p->G >= 4 * p->C || (p->Dpad <= 128 && 10 * (long long)p->G >= 27 * (long long)p->C)) ? 2 : 1;
 }

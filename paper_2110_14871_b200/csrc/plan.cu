@@ -137,7 +137,7 @@ static int round_up(int a, int b) { return (a + b - 1) / b * b; }
 static void build_tc_chunks(gdws_plan_s *p)
 {
     p->tc_ok = false;
-    if (p->stride != 1 || p->k > 5 || p->C % 8 || p->D % 8 || p->Dpad > 1024) return;
+    if (p->stride > 2 || p->k > 5 || p->C % 8 || p->D % 8 || p->Dpad > 1024) return;
     p->tc_nparts = (p->Dpad + 255) / 256;
     p->tc_dloc = round_up((p->Dpad + p->tc_nparts - 1) / p->tc_nparts, 16);
     const int nmax = tc_nmax(p->k, p->tc_dloc);

@@ -133,6 +133,14 @@ TC_SHAPES = [
     (4, 16, 128, 3, 3, 3, 1, 1, ("uniform", 1, 9)),
     (2, 16, 32, 6, 20, 3, 1, 0, ("uniform", 1, 9)),
     (1, 16, 16, 9, 9, 3, 1, 1, ("const", 12)),              # g_c > k*k is legal (Lemma 1 caps the rank, not the count)
+    # stride 2: the input is read through one dense view per parity of row and column
+    (2, 16, 16, 8, 8, 3, 2, 1, ("uniform", 1, 9)),          # 4 x 4 output maps: one copy per tap
+    (3, 32, 64, 17, 15, 3, 2, 1, ("uniform", 1, 9)),        # odd input sizes: the views differ in size
+    (1, 16, 32, 32, 32, 3, 2, 1, ("uniform", 1, 9)),        # one image per tile, four boxes with halo
+    (5, 16, 24, 16, 16, 3, 2, 1, ("uniform", 0, 9)),        # 8 x 8 output maps: two images per tile
+    (2, 24, 40, 19, 23, 5, 2, 2, ("uniform", 1, 25)),
+    (2, 16, 16, 12, 12, 1, 2, 0, ("uniform", 1, 1)),        # k = 1: only the even rows and columns are read
+    (1, 64, 272, 28, 28, 3, 2, 1, ("heavy",)),
 ]
 
 
@@ -147,14 +155,14 @@ def test_bf16_tensor_core_gdw_matches_reference(shape):
     assert err <= 1e-2, err
 
 
-def test_tensor_core_gdw_agrees_with_alu_gdw_and_refuses_stride_2():
+def test_tensor_core_gdw_agrees_with_alu_gdw_and_refuses_stride_3():
     spec = small_spec("t", 6, 32, 48, 16, 16, seed=77)
     data = gi.make_layer(spec)
     a = run_gpu(data, path=gdws.PATH_FUSED, dw_math=2)
     b = run_gpu(data, path=gdws.PATH_FUSED, dw_math=1)
     # both round z to bf16 once and accumulate in fp32; only the summation order differs
     assert rel_err(a, b) <= 4e-3
-    data2 = gi.make_layer(small_spec("t", 2, 16, 16, 8, 8, 3, 2, 1, seed=78))
+    data2 = gi.make_layer(small_spec("t", 2, 16, 16, 9, 9, 3, 3, 1, seed=78))
     with pytest.raises(gdws.GdwsError) as e:
         run_gpu(data2, path=gdws.PATH_FUSED, dw_math=2)
     assert e.value.status == gdws.ERR_UNSUPPORTED
