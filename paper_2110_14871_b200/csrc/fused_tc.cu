@@ -11,6 +11,8 @@
 // rounded to bf16 and written as the K-major A operand of the pointwise stage (Property 1: W_P is M x G), whose
 // products accumulate in a second TMEM region over all windows of the tile.  The ALUs only round z, scatter the
 // filter taps into the B operands and run the epilogue; they execute no multiply of the GDW stage.
+// With stride 2 the box is staged from four dense views of x (one per parity of input row and column), in each of which
+// a tap is again a unit-stride shift; which copy a tap reads and where its operand starts come from tables.
 //
 // One persistent block of 20 warps per SM walks over work items (tile of 128 output pixels x block of up to
 // 256 output channels).  Roles, coupled by mbarriers only:
