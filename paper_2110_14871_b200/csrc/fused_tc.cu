@@ -80,6 +80,7 @@ struct alignas(64) TcParams {
     // bits 0-7 first z slab, 8-15 first weight slab, 16-18 / 19-21 how many units back the PW products must be done
     // before the z slabs / the weight slabs are overwritten (0: no wait).  A chunk's slabs are contiguous (no wrap).
     uint32_t ring[kTcMaxChunks];
+    uint8_t order[kTcMaxChunks];   // the chunk the block takes i-th within a work item (an index into `chunks`)
 };
 
 // Bounded wait of every role but the issuing warps: each poll lets the hardware suspend the thread until the phase
@@ -167,7 +168,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         const uint4 *src = reinterpret_cast<const uint4 *>(P.chunks);
         uint4 *dst = reinterpret_cast<uint4 *>(tab);
         for (int i = tid; i < P.nchunks * 2; i += kTcThreads) {
-            uint4 w4 = __ldg(src + i);
+            uint4 w4 = __ldg(src + 2 * (int)P.order[i >> 1] + (i & 1));
             if (i & 1) w4.z = P.ring[i >> 1];        // second half of the entry: slab0, flags, places in the rings, (unused)
             dst[i] = w4;
         }
@@ -665,14 +666,14 @@ bool tc_geometry(const gdws_plan_s *p, int n, int Ho, int Wo, TcGeom *out)
 // and a chunk that does not fit behind its predecessor starts over at slab 0.  dep[q] = how many units before chunk q
 // the last chunk that used any of its slabs ran (in steady state, work item after work item), at most 4: the four
 // barriers of a ring are reused every four units, so a producer never runs further ahead than that anyway.
-bool tc_ring_places(const std::vector<TcChunk> &chunks, int cap, std::vector<int> *pos, std::vector<int> *dep)
+bool tc_ring_places(const std::vector<int> &slabs, int cap, std::vector<int> *pos, std::vector<int> *dep)
 {
-    const int n = (int)chunks.size();
+    const int n = (int)slabs.size();
     pos->assign(n, 0);
     dep->assign(n, 4);
     int head = 0;
     for (int q = 0; q < n; ++q) {
-        const int ns = chunks[q].npad / 16;
+        const int ns = slabs[q];
         if (ns > cap) return false;
         if (head + ns > cap) head = 0;
         (*pos)[q] = head;
@@ -680,12 +681,61 @@ bool tc_ring_places(const std::vector<TcChunk> &chunks, int cap, std::vector<int
     }
     std::vector<int> last(cap, -1000000);
     for (int v = 0; v < 3 * n; ++v) {
-        const int q = v % n, ns = chunks[q].npad / 16;
+        const int q = v % n, ns = slabs[q];
         int newest = -1000000;
         for (int s2 = (*pos)[q]; s2 < (*pos)[q] + ns; ++s2) { newest = std::max(newest, last[s2]); last[s2] = v; }
         if (v >= 2 * n) (*dep)[q] = std::max(1, std::min(4, v - newest));
     }
     return true;
+}
+
+// The windows of a work item may be taken in any order (their contributions to y add up), and the order decides how
+// well consecutive chunks share the two slab rings: a chunk whose slabs are still held by the chunk right before it
+// waits for that one's PW products, and with them the weight copy or the conversion loses its head start.  A few
+// orders (as planned, large and small windows alternating, sorted, some shuffles) are laid out; the one with the
+// fewest such waits wins, the planned order on a tie.  Chunks of one window stay together.
+void tc_choose_order(const std::vector<TcChunk> &chunks, int nz, int nw, std::vector<int> *order)
+{
+    std::vector<std::vector<int>> windows;
+    for (int i = 0; i < (int)chunks.size(); ++i) {
+        if (chunks[i].flags & 1) windows.emplace_back();
+        windows.back().push_back(i);
+    }
+    const int nwin = (int)windows.size();
+    auto slabs_of = [&](int w) { int t = 0; for (int i : windows[w]) t += chunks[i].npad / 16; return t; };
+    std::vector<int> base(nwin), sorted(nwin);
+    for (int w = 0; w < nwin; ++w) base[w] = sorted[w] = w;
+    std::stable_sort(sorted.begin(), sorted.end(), [&](int a, int b) { return slabs_of(a) > slabs_of(b); });
+    std::vector<std::vector<int>> cands;
+    cands.push_back(base);
+    {
+        std::vector<int> alt;
+        for (int lo = 0, hi = nwin, turn = 0; lo < hi; ++turn) alt.push_back((turn & 1) ? sorted[--hi] : sorted[lo++]);
+        cands.push_back(alt);
+    }
+    cands.push_back(sorted);
+    cands.push_back(std::vector<int>(sorted.rbegin(), sorted.rend()));
+    uint32_t rng = 0x9E3779B9u ^ (uint32_t)chunks.size() * 2654435761u;
+    for (int t = 0; t < 24; ++t) {
+        std::vector<int> sh = base;
+        for (int i = nwin - 1; i > 0; --i) {
+            rng = rng * 1664525u + 1013904223u;
+            std::swap(sh[i], sh[(rng >> 8) % (uint32_t)(i + 1)]);
+        }
+        cands.push_back(sh);
+    }
+    double best = 1e300;
+    for (const std::vector<int> &cand : cands) {
+        std::vector<int> seq, slabs;
+        for (int w : cand) for (int i : windows[w]) { seq.push_back(i); slabs.push_back(chunks[i].npad / 16); }
+        std::vector<int> zp, zd, wp, wd;
+        if (!tc_ring_places(slabs, nz, &zp, &zd) || !tc_ring_places(slabs, nw, &wp, &wd)) continue;
+        double cost = 0;
+        for (size_t u = 0; u < seq.size(); ++u)
+            cost += (zd[u] == 1 ? 1.0 : 0.0) + (wd[u] == 1 ? 1.0 : 0.0);
+        if (cost < best - 1e-9) { best = cost; *order = seq; }
+    }
+    if (order->empty()) for (int i = 0; i < (int)chunks.size(); ++i) order->push_back(i);
 }
 
 }  // namespace
@@ -738,11 +788,21 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     if (best_score < 0) return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: shared memory does not fit this layer");
     P.ostage = b_ost ? 16384 : 0; P.nx = b_nx; P.nb = b_nb; P.nz = b_nz; P.nw = b_nw;
     {
-        std::vector<int> zpos, zdep, wpos, wdep;
-        if (!tc_ring_places(p->tc_chunks, P.nz, &zpos, &zdep) || !tc_ring_places(p->tc_chunks, P.nw, &wpos, &wdep))
-            return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: a chunk does not fit the slab rings");
-        for (int q = 0; q < nchunks; ++q)
-            P.ring[q] = (uint32_t)zpos[q] | ((uint32_t)wpos[q] << 8) | ((uint32_t)zdep[q] << 16) | ((uint32_t)wdep[q] << 19);
+        if (p->tc_lay_nz != P.nz || p->tc_lay_nw != P.nw || (int)p->tc_lay_order.size() != nchunks) {
+            std::vector<int> order, slabs, zpos, zdep, wpos, wdep;
+            tc_choose_order(p->tc_chunks, P.nz, P.nw, &order);
+            for (int i : order) slabs.push_back(p->tc_chunks[i].npad / 16);
+            if (!tc_ring_places(slabs, P.nz, &zpos, &zdep) || !tc_ring_places(slabs, P.nw, &wpos, &wdep))
+                return fail(GDWS_ERR_UNSUPPORTED, "tensor-core GDW path: a chunk does not fit the slab rings");
+            p->tc_lay_order.resize(nchunks); p->tc_lay_ring.resize(nchunks);
+            for (int q = 0; q < nchunks; ++q) {
+                p->tc_lay_order[q] = (uint8_t)order[q];
+                p->tc_lay_ring[q] = (uint32_t)zpos[q] | ((uint32_t)wpos[q] << 8) | ((uint32_t)zdep[q] << 16) | ((uint32_t)wdep[q] << 19);
+            }
+            p->tc_lay_nz = P.nz; p->tc_lay_nw = P.nw;
+        }
+        memcpy(P.order, p->tc_lay_order.data(), (size_t)nchunks);
+        memcpy(P.ring, p->tc_lay_ring.data(), (size_t)nchunks * 4);
     }
     P.off_b = (uint32_t)P.ostage;
     P.off_z = P.off_b + (uint32_t)P.nb * P.bbuf_bytes;

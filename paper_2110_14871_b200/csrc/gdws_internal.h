@@ -80,6 +80,11 @@ struct gdws_plan_s {
     // Tensor-core GDW path (fused_tc.cu): chunk list, output-channel split, packed sizes.
     bool tc_ok = false;              // the layer is one the path covers (stride 1, k <= 5, ...)
     std::vector<gdws::TcChunk> tc_chunks;
+    // last layout of the tensor-core path's slab rings (chunk order within a work item, places and waits), kept per
+    // ring sizes: working it out tries a few dozen orders
+    int tc_lay_nz = 0, tc_lay_nw = 0;
+    std::vector<uint8_t> tc_lay_order;
+    std::vector<uint32_t> tc_lay_ring;
     int tc_nslabs = 0;               // sum of npad / 16 over the chunks
     int tc_maxslabs = 0;             // largest npad / 16 of one chunk
     int tc_nparts = 1, tc_dloc = 0;  // blocks per tile along D, output channels per block (multiple of 16, <= 256)
