@@ -69,8 +69,8 @@ def layer_numbers(spec: gi.LayerSpec, G: int):
 # summarised under profiles/ (key: config, layer, path, GDW stage).  An entry is removed when its kernel changes.
 TRAFFIC_BYTES_PER_LAUNCH = {
     (1, 0, "fused", 2): 9182976,      # x + weights; y (8.39 MB) stays in L2 within the captured launch
-    (2, 0, "fused", 1): 25802240,     # x + weights; y (25.7 MB) stays in L2
-    (3, 0, "fused", 2): 93988864,     # x (67.1 MB) + the part of y that left L2
+    (2, 0, "fused", 1): 25810944,     # x + weights; y (25.7 MB) stays in L2
+    (3, 0, "fused", 2): 92575232,     # x (67.1 MB) + the part of y that left L2
 }
 
 
