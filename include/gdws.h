@@ -154,8 +154,8 @@ GDWS_API int gdws_out_dim(int in, int k, int stride, int pad);
  * Definition) with the current GDWS_OPT_DW_MATH: *stage = 1 (ALUs) or 2 (tensor cores).  With the option
  * at 0 the choice follows the measured cost of the two kernels: the tensor-core form costs k*k products
  * per window of 16 input channels whatever their g_c, the ALU form costs in proportion to sum g_c; the
- * tensor cores are taken for k = 3, stride 1 (with at most 256 output channels) or 2, and an average g_c
- * of at least 4 (at least 2.7 with at most 128 output channels).  Host only; errors: GDWS_ERR_INVALID_ARG.
+ * tensor cores are taken for k = 3 or 5, stride 1 (with at most 256 output channels) or 2, and an average
+ * g_c of at least 4 (at least 2.7 with at most 128 output channels).  Host only; errors: GDWS_ERR_INVALID_ARG.
  */
 GDWS_API gdws_status_t gdws_plan_gdw_stage(const gdws_plan_t *plan, int *stage);
 

@@ -108,12 +108,17 @@ struct SlabRing {
     int head = 0, free_slabs = 0, oldest = 0;
 };
 
+// Filters of more than 9 taps: a B buffer holds the operands of up to 9 taps at a time (8 for k = 4), and a chunk's GDW
+// products are issued group by group as the groups' operands arrive, all into the same accumulator.
+__host__ __device__ constexpr int tc_taps_per_build(int k) { return k * k <= 9 ? k * k : (k == 4 ? 8 : 9); }
+
 template <int K>
 __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_constant__ TcParams P)
 {
+    constexpr int TPB = tc_taps_per_build(K), NBUILD = (K * K + TPB - 1) / TPB;   // taps per B buffer, buffers per chunk
     extern __shared__ uint8_t smem_raw[];
-    // dwready[4] | zfull[2] (2 unused) | pwready[4] pwdone[4] | bfree[4] xfree[4] | accfull[2] accfree[2] | drain[2]
-    __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4 + 2];
+    // dwready[4] | zfull[2] (2 unused) | pwready[4] pwdone[4] | bfree[4] xfree[4] | accfull[2] accfree[2] | drain[2] | 2 unused | bready[4]
+    __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4 + 4 + kTcMaxNB];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -132,6 +137,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     const uint32_t bar_bfree = bar_pwdone + 8 * kTcNU, bar_xfree = bar_bfree + 8 * kTcMaxNB;
     const uint32_t bar_accfull = bar_xfree + 8 * kTcMaxNX, bar_accfree = bar_accfull + 16;
     const uint32_t bar_drain = bar_accfull + 32;       // the issuing warps' last commits, awaited before TMEM is freed
+    const uint32_t bar_bready = bar_drain + 32;        // (filters of more than 9 taps) the operands of a group of taps are in a B buffer
     volatile int *const vabort = &abort_flag;
     TcChunk *tab = reinterpret_cast<TcChunk *>(base + P.off_tab);
     float *bias_sm = reinterpret_cast<float *>(tab + P.nchunks);
@@ -140,7 +146,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
 
     if (tid == 0) {
         abort_flag = 0;
-        for (int i = 0; i < 4; ++i) mbar_init(bar_dwready + 8 * i, 5);
+        // with one B buffer per chunk the builder warps count towards dwready; else they have barriers of their own
+        for (int i = 0; i < 4; ++i) mbar_init(bar_dwready + 8 * i, NBUILD == 1 ? 5 : 1);
+        for (int i = 0; i < kTcMaxNB; ++i) mbar_init(bar_bready + 8 * i, 4);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_zfull + 8 * i, 1);
             mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4);
@@ -203,9 +211,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
 #pragma unroll
             for (int v = 0; v < K; ++v) {
                 tap_a[ur * K + v] = P.tap_off[ur * K + v] >> 4;
-                tap_b[ur * K + v] = (uint32_t)(ur * K + v) * pstep;
+                tap_b[ur * K + v] = (uint32_t)((ur * K + v) % TPB) * pstep;
             }
-        uint32_t xslot = 0, bslot = 0, a_lo = a_lo0, b_lo = b_lo0;
+        uint32_t xslot = 0, bslot = 0, buse = 0, a_lo = a_lo0, b_lo = b_lo0;
+        (void)buse;
         int q = 0;                  // chunk index of unit u within its work item
 #pragma unroll 1
         for (int u = 0; u < total; ++u) {
@@ -213,19 +222,44 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             mbar_wait_call(bar_dwready + 8 * (u & 3), (uint32_t)(u >> 2) & 1u, &abort_flag, P.status, kStatusWaitOperand);
             if (u >= 2) mbar_wait_call(bar_pwready + 8 * ((u - 2) & 3), (uint32_t)((u - 2) >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
             tc_fence_after();
-            if (elect_one()) {
+            if constexpr (NBUILD == 1) {
+                if (elect_one()) {
+                    const uint32_t idesc = make_idesc(npad, false);
+                    const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
+#pragma unroll
+                    for (int i = 0; i < K * K; ++i)
+                        umma_bf16_words(d_z, a_lo + tap_a[i], a_hi, b_lo + tap_b[i], p_hi, idesc, i != 0);
+                    umma_commit(bar_zfull + 8 * (u & 1));
+                    umma_commit(bar_bfree + 8 * bslot);
+                    if (flags & 2) umma_commit(bar_xfree + 8 * xslot);
+                }
+                __syncwarp();
+                b_lo += bstep;
+                if (++bslot == (uint32_t)P.nb) { bslot = 0; b_lo = b_lo0; }
+            } else {
                 const uint32_t idesc = make_idesc(npad, false);
                 const uint32_t d_z = tmem + (uint32_t)(kTcZCol + 128 * (u & 1));
 #pragma unroll
-                for (int i = 0; i < K * K; ++i)
-                    umma_bf16_words(d_z, a_lo + tap_a[i], a_hi, b_lo + tap_b[i], p_hi, idesc, i != 0);
-                umma_commit(bar_zfull + 8 * (u & 1));
-                umma_commit(bar_bfree + 8 * bslot);
-                if (flags & 2) umma_commit(bar_xfree + 8 * xslot);
+                for (int r = 0; r < NBUILD; ++r) {
+                    // the operands of tap group r: buffer bslot, for the buse-th time
+                    mbar_wait_call(bar_bready + 8 * bslot, buse & 1u, &abort_flag, P.status, kStatusWaitOperand);
+                    tc_fence_after();
+                    if (elect_one()) {
+#pragma unroll
+                        for (int j = 0; j < TPB; ++j)
+                            if (r * TPB + j < K * K)
+                                umma_bf16_words(d_z, a_lo + tap_a[r * TPB + j], a_hi, b_lo + tap_b[r * TPB + j], p_hi, idesc, (r | j) != 0);
+                        umma_commit(bar_bfree + 8 * bslot);
+                        if (r == NBUILD - 1) {
+                            umma_commit(bar_zfull + 8 * (u & 1));
+                            if (flags & 2) umma_commit(bar_xfree + 8 * xslot);
+                        }
+                    }
+                    __syncwarp();
+                    b_lo += bstep;
+                    if (++bslot == (uint32_t)P.nb) { bslot = 0; b_lo = b_lo0; ++buse; }
+                }
             }
-            __syncwarp();
-            b_lo += bstep;
-            if (++bslot == (uint32_t)P.nb) { bslot = 0; b_lo = b_lo0; }
             if (flags & 2) {
                 a_lo += xstep;
                 if (++xslot == (uint32_t)P.nx) { xslot = 0; a_lo = a_lo0; }
@@ -294,8 +328,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 for (int q = 0; q < P.nchunks; ++q, ++u) {
                     const int cbase = tab[q].cbase, flags = tab[q].flags;
                     const uint32_t bar = bar_dwready + 8 * (u & 3);
-                    // this barrier's last phase (chunk u - 4) must be complete before anything counts towards chunk u
-                    if (u >= 4) tc_wait(bar, (uint32_t)((u >> 2) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                    // This barrier's last phase (chunk u - 4) must be complete, and seen by the issuing warp, before anything
+                    // counts towards chunk u.  Where the builder warps count towards it too, they keep this thread within
+                    // four chunks of the issuing warp (they wait for its commits); where they do not (filters of more than
+                    // 9 taps), this thread waits until chunk u - 4 has been converted, which is after its products were issued.
+                    if (u >= 4) {
+                        if constexpr (NBUILD == 1) tc_wait(bar, (uint32_t)((u >> 2) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                        else tc_wait(bar_pwready + 8 * (u & 3), (uint32_t)((u >> 2) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                    }
                     if (*vabort) { stop = true; break; }       // a wait ran out somewhere: no new copies
                     if (!(flags & 1)) { mbar_arrive(bar); continue; }
                     if (box >= P.nx)
@@ -503,7 +543,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             }
         };
         if (total > 0) load_rec(tab[0], nxt);
-        uint32_t bslot = 0, bpar = 0;      // B buffer of unit v, and the parity of the "free" phase it waits for
+        uint32_t bslot = 0, bpar = 0, buse = 0;      // B buffer in turn, the parity of the "free" phase it waits for / how often it was used
+        (void)bpar; (void)buse;
         int q = 0;
 #pragma unroll 1
         for (int v = 0; v < total; ++v) {
@@ -514,23 +555,49 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             const uint32_t cw = rec[0] & 0xFFFFu;
             const bool valid = cw != 0xFFFFu;
             const uint32_t off = rowoff + ((((cw >> 3) & 1u) ^ rowsw) << 4) + (cw & 7u) * 2u;
-            if (v >= P.nb) tc_warp_wait_call(bar_bfree + 8 * bslot, bpar, &abort_flag, P.status, kStatusWaitStage);
-            const uint32_t bb = b_s + bslot * P.bbuf_bytes;
-            const uint32_t old = bold[bslot * 128 + t];
-            if (old != 0xFFFFu) {
-                uint32_t a = bb + old;
+            if constexpr (NBUILD == 1) {
+                if (v >= P.nb) tc_warp_wait_call(bar_bfree + 8 * bslot, bpar, &abort_flag, P.status, kStatusWaitStage);
+                const uint32_t bb = b_s + bslot * P.bbuf_bytes;
+                const uint32_t old = bold[bslot * 128 + t];
+                if (old != 0xFFFFu) {
+                    uint32_t a = bb + old;
 #pragma unroll 1
-                for (int j = 0; j < K * K; ++j, a += P.bplane) sts16(a, (uint16_t)0);
-            }
-            if (valid) {
+                    for (int j = 0; j < K * K; ++j, a += P.bplane) sts16(a, (uint16_t)0);
+                }
+                if (valid) {
 #pragma unroll
-                for (int j = 0; j < K * K; ++j)     // 16-bit word 1 + j of the record holds tap j
-                    sts16(bb + (uint32_t)j * P.bplane + off, (uint16_t)(rec[(1 + j) >> 1] >> (16 * ((1 + j) & 1))));
+                    for (int j = 0; j < K * K; ++j)     // 16-bit word 1 + j of the record holds tap j
+                        sts16(bb + (uint32_t)j * P.bplane + off, (uint16_t)(rec[(1 + j) >> 1] >> (16 * ((1 + j) & 1))));
+                }
+                bold[bslot * 128 + t] = (uint16_t)(valid ? off : 0xFFFFu);
+                fence_proxy_async();
+                tc_warp_arrive(bar_dwready + 8 * (v & 3));
+                if (++bslot == (uint32_t)P.nb) { bslot = 0; if (v >= P.nb) bpar ^= 1u; }
+            } else {
+                // up to TPB taps per buffer: NBUILD buffers per chunk, each announced on its own barrier
+#pragma unroll
+                for (int r = 0; r < NBUILD; ++r) {
+                    if (buse) tc_warp_wait_call(bar_bfree + 8 * bslot, (buse - 1u) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                    const uint32_t bb = b_s + bslot * P.bbuf_bytes;
+                    const uint32_t old = bold[bslot * 128 + t];
+                    if (old != 0xFFFFu) {
+                        uint32_t a = bb + old;
+#pragma unroll 1
+                        for (int j = 0; j < TPB; ++j, a += P.bplane) sts16(a, (uint16_t)0);
+                    }
+                    if (valid) {
+#pragma unroll
+                        for (int j = 0; j < TPB; ++j) {
+                            const int h = 1 + r * TPB + j;          // 16-bit word h of the record holds tap h - 1
+                            if (h <= K * K) sts16(bb + (uint32_t)j * P.bplane + off, (uint16_t)(rec[h >> 1] >> (16 * (h & 1))));
+                        }
+                    }
+                    bold[bslot * 128 + t] = (uint16_t)(valid ? off : 0xFFFFu);
+                    fence_proxy_async();
+                    tc_warp_arrive(bar_bready + 8 * bslot);
+                    if (++bslot == (uint32_t)P.nb) { bslot = 0; ++buse; }
+                }
             }
-            bold[bslot * 128 + t] = (uint16_t)(valid ? off : 0xFFFFu);
-            fence_proxy_async();
-            tc_warp_arrive(bar_dwready + 8 * (v & 3));
-            if (++bslot == (uint32_t)P.nb) { bslot = 0; if (v >= P.nb) bpar ^= 1u; }
         }
     }
     tc_fence_before();
@@ -761,7 +828,7 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     memset(&P, 0, sizeof(P));
     const int Dloc = p->tc_dloc, m = p->tc_maxslabs;
     // a B operand plane holds one 32-byte row per intermediate channel of the layer's largest chunk
-    P.bplane = (uint32_t)m * 16u * 32u; P.bbuf_bytes = (uint32_t)(k * k) * P.bplane;
+    P.bplane = (uint32_t)m * 16u * 32u; P.bbuf_bytes = (uint32_t)tc_taps_per_build(k) * P.bplane;
     P.wslab_bytes = (uint32_t)Dloc * 32u;
     P.xslot_bytes = (uint32_t)((g.xbox + 255) / 256 * 256);
     // Shared memory: output staging (optional) | B operand buffers | z slabs | weight slabs | input boxes | tables

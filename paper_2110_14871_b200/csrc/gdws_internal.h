@@ -37,9 +37,10 @@ struct TcChunk {
     int32_t reserved0, reserved1;
 };
 
-// Most intermediate channels one chunk of the tensor-core GDW path holds: its k*k B operands (32 bytes per
-// channel each) must fit shared memory twice, and two GDW accumulators must fit beside the PW accumulator in TMEM.
-inline int tc_nmax(int k, int dloc) { return k >= 4 ? 32 : (dloc > 128 ? 96 : 128); }
+// Most intermediate channels one chunk of the tensor-core GDW path holds: its B operands (32 bytes per channel and
+// tap; up to 9 taps per buffer) must fit shared memory twice, and two GDW
+// accumulators must fit beside the PW accumulator in TMEM.
+inline int tc_nmax(int k, int dloc) { (void)k; return dloc > 128 ? 96 : 128; }
 
 struct Tile {
     int TN = 0, PH = 0, PW = 0;      // images x rows x columns of output pixels per 128-row tile
@@ -160,7 +161,7 @@ inline size_t dtype_size(gdws_dtype_t d) { return d == GDWS_F32 ? 4 : 2; }
 inline int gdw_stage_of(const gdws_plan_s *p)
 {
     if (p->opt_dw_math == 1 || p->opt_dw_math == 2) return p->opt_dw_math;
-    if (!(p->tc_ok && p->k == 3 && p->stride <= 2)) return 1;
+    if (!(p->tc_ok && (p->k == 3 || p->k == 5) && p->stride <= 2)) return 1;
     if (p->stride == 1 && p->Dpad > 256) return 1;     // measured equal or slower there; with stride 2 faster at D = 512 too
     // average multiplier of at least 4, or of at least 2.7 when the PW products are small (at most 128 output channels)
     return (p->G >= 4 * p->C || (p->Dpad <= 128 && 10 * (long long)p->G >= 27 * (long long)p->C)) ? 2 : 1;

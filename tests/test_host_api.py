@@ -113,7 +113,7 @@ def test_fused_tiles_cover_the_benchmark_layers(cfg):
 
 
 def test_gdw_stage_choice_follows_the_documented_rule():
-    """Tensor cores for k = 3, stride 1 or 2, at most 256 output channels and an average multiplier of at least 4
+    """Tensor cores for k = 3 or 5, stride 1 or 2, at most 256 output channels and an average multiplier of at least 4
     (2.7 with at most 128 output channels); the option overrides the choice."""
     def stage(C, D, k, stride, g, opt=0):
         plan = gdws.Plan(C, D, k, stride, k // 2, np.full(C, g, dtype=np.int32))
@@ -127,5 +127,5 @@ def test_gdw_stage_choice_follows_the_documented_rule():
     assert stage(64, 512, 3, 1, 5) == 1         # no room for two GDW accumulators beside 512 output columns
     assert stage(64, 64, 3, 2, 5) == 2 and stage(64, 64, 3, 3, 5) == 1     # strides 1 and 2 are covered by the tensor-core form
     assert stage(64, 512, 3, 2, 5) == 2         # with stride 2 also beyond 256 output channels
-    assert stage(64, 64, 5, 1, 12) == 1
+    assert stage(64, 64, 5, 1, 12) == 2 and stage(64, 64, 4, 1, 12) == 1
     assert stage(64, 64, 3, 1, 2, opt=2) == 2 and stage(64, 64, 3, 1, 5, opt=1) == 1
