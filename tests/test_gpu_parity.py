@@ -141,6 +141,10 @@ TC_SHAPES = [
     (2, 24, 40, 19, 23, 5, 2, 2, ("uniform", 1, 25)),
     (2, 16, 16, 12, 12, 1, 2, 0, ("uniform", 1, 1)),        # k = 1: only the even rows and columns are read
     (1, 64, 272, 28, 28, 3, 2, 1, ("heavy",)),
+    # more than 9 taps: the B operands go through the buffers in groups of taps
+    (2, 16, 32, 12, 12, 4, 1, 1, ("uniform", 1, 16)),
+    (3, 32, 48, 13, 13, 4, 2, 1, ("uniform", 1, 16)),
+    (80, 32, 32, 16, 16, 5, 1, 2, ("uniform", 1, 25)),      # more tiles than SMs, windows of three chunks
 ]
 
 
