@@ -108,9 +108,9 @@ struct SlabRing {
     int head = 0, free_slabs = 0, oldest = 0;
 };
 
-// Filters of more than 9 taps: a B buffer holds the operands of up to 9 taps at a time (8 for k = 4), and a chunk's GDW
+// Filters of more than 9 taps: a B buffer holds the operands of up to 13 taps at a time (8 for k = 4), and a chunk's GDW
 // products are issued group by group as the groups' operands arrive, all into the same accumulator.
-__host__ __device__ constexpr int tc_taps_per_build(int k) { return k * k <= 9 ? k * k : (k == 4 ? 8 : 9); }
+__host__ __device__ constexpr int tc_taps_per_build(int k) { return k * k <= 9 ? k * k : (k == 4 ? 8 : 13); }
 
 template <int K>
 __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_constant__ TcParams P)
