@@ -73,6 +73,7 @@ struct alignas(64) TcParams {
     uint32_t tap_off[kTcMaxTaps];          // the A operand of tap (u, v) starts this many bytes into the box slot
     uint32_t a_sbo;              // GDW A operand: bytes between 8-pixel groups
     int nb, nx, nz, nw, nacc;
+    int nbw;                     // builder warps that have rows to fill (32 rows each; the layer's largest chunk decides)
     uint32_t bbuf_bytes, bplane, xslot_bytes, wslab_bytes;
     uint32_t off_b, off_z, off_w, off_x, off_tab;    // from the 1024-aligned base; the output staging comes first
     int ostage, rec_hw, nslabs_total, bias_len;
@@ -125,12 +126,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     uint8_t *base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t base_s = smem_u32(base);
     const uint32_t o_s = base_s, b_s = base_s + P.off_b, z_s = base_s + P.off_z, w_s = base_s + P.off_w, x_s = base_s + P.off_x;
-    // dwready: the B operands (the 4 builder warps of the chunk's parity) and the input box (the loader's arrive, with the
+    // dwready: the B operands (the builder warps that have rows to fill) and the input box (the loader's arrive, with the
     // box's bytes when the chunk opens a window) of a chunk are in place.  zfull[h]: the GDW products of a chunk of parity h
     // are done.  pwready: the chunk's z slabs (the 4 converter warps of its parity) and its pointwise weights (the loader's
-    // arrive with their bytes) are in place.  pwdone: its PW products are done.  bfree: arrived by a converter once the
-    // GDW products that read a B buffer are done.  xfree: two arrivals per window, after the GDW products of its last
-    // chunk and of the chunk before it (issued by the other warp) are done.
+    // arrive with their bytes) are in place.  pwdone: its PW products are done.  bfree / xfree: committed by the GDW
+    // issuing warp once the products that read a B buffer / the last ones that read a box are done.
     const uint32_t bar_dwready = smem_u32(&bars[0]);
     const uint32_t bar_zfull = bar_dwready + 32;
     const uint32_t bar_pwready = bar_zfull + 32, bar_pwdone = bar_pwready + 8 * kTcNU;
@@ -147,8 +147,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     if (tid == 0) {
         abort_flag = 0;
         // with one B buffer per chunk the builder warps count towards dwready; else they have barriers of their own
-        for (int i = 0; i < 4; ++i) mbar_init(bar_dwready + 8 * i, NBUILD == 1 ? 5 : 1);
-        for (int i = 0; i < kTcMaxNB; ++i) mbar_init(bar_bready + 8 * i, 4);
+        for (int i = 0; i < 4; ++i) mbar_init(bar_dwready + 8 * i, NBUILD == 1 ? 1 + P.nbw : 1);
+        for (int i = 0; i < kTcMaxNB; ++i) mbar_init(bar_bready + 8 * i, P.nbw);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_zfull + 8 * i, 1);
             mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4);
@@ -521,7 +521,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
             }
         }
         if (P.ostage && issuer) bulk_wait_all();
-    } else if (warp >= kTcBuildWarp0) {
+    } else if (warp >= kTcBuildWarp0 && warp < kTcBuildWarp0 + P.nbw) {
         // ---------------- builder: filter taps -> B operands of the GDW products ----------------
         // Thread t owns intermediate slot t of the current chunk.  The B operand of tap (ur, v) is a [n x 16]
         // K-major matrix whose row t has the tap's value in column `channel of slot t inside the window`.
@@ -969,6 +969,7 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     P.nacc = Dloc <= 128 ? 2 : 1;
     P.rec_hw = p->tc_rec_hw; P.nslabs_total = p->tc_nslabs;
     P.bias_len = p->Dpad;
+    P.nbw = std::min(kTcBuildWarps, (m * 16 + 31) / 32);
 
     const int grid = (int)(nitems < p->sm_count ? nitems : p->sm_count);
     cudaError_t e = cudaSuccess;
