@@ -144,20 +144,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
     uint16_t *bold = reinterpret_cast<uint16_t *>(bias_sm + P.Dpad_tot);     // [2 * nb][128]: what each builder thread wrote last
     const uint32_t bias_s = smem_u32(bias_sm);
 
-    if (tid == 0) {
-        abort_flag = 0;
-        // with one B buffer per chunk the builder warps count towards dwready; else they have barriers of their own
-        for (int i = 0; i < 4; ++i) mbar_init(bar_dwready + 8 * i, NBUILD == 1 ? 1 + P.nbw : 1);
-        for (int i = 0; i < kTcMaxNB; ++i) mbar_init(bar_bready + 8 * i, P.nbw);
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_zfull + 8 * i, 1);
-            mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accfree + 8 * i, 4);
+    // The chunk table was written when the plan was built (by a synchronous copy), not by a kernel: its loads may start
+    // at once and be in flight during the rest of the set-up (one 16-byte word per thread; at most 256 chunks).
+    static_assert(2 * kTcMaxChunks <= kTcThreads, "one table word per thread");
+    uint4 tabw = make_uint4(0u, 0u, 0u, 0u);
+    if (tid < P.nchunks * 2) {
+        tabw = __ldg(reinterpret_cast<const uint4 *>(P.chunks) + 2 * (int)P.order[tid >> 1] + (tid & 1));
+        if (tid & 1) tabw.z = P.ring[tid >> 1];      // second half of the entry: slab0, flags, places in the rings, (unused)
+    }
+    if (tid == 0) abort_flag = 0;
+    {
+        // One barrier per thread of warps 1 and 2 (warp 0 allocates tensor memory meanwhile).  Layout of bars[] as above;
+        // with one B buffer per chunk the builder warps count towards dwready, else they have barriers of their own.
+        constexpr int kBars = 4 + 4 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4 + 4 + kTcMaxNB;
+        const int b = tid - 32;
+        if (b >= 0 && b < kBars) {
+            uint32_t count = 1;                                                       // zfull, pwdone, bfree, xfree, accfull, drain
+            if (b < 4) count = NBUILD == 1 ? 1u + (uint32_t)P.nbw : 1u;               // dwready
+            else if (b >= 8 && b < 8 + kTcNU) count = kTcConvWarps / 2 + 1;           // pwready
+            else if (b >= 8 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 2 && b < 8 + 2 * kTcNU + kTcMaxNB + kTcMaxNX + 4) count = 4;   // accfree
+            else if (b >= kBars - kTcMaxNB) count = (uint32_t)P.nbw;                   // bready
+            mbar_init(bar_dwready + 8 * (uint32_t)b, count);
+            fence_mbar_init();
         }
-        for (int i = 0; i < kTcNU; ++i) { mbar_init(bar_pwready + 8 * i, kTcConvWarps / 2 + 1); mbar_init(bar_pwdone + 8 * i, 1); }
-        for (int i = 0; i < kTcMaxNB; ++i) mbar_init(bar_bfree + 8 * i, 1);
-        for (int i = 0; i < kTcMaxNX; ++i) mbar_init(bar_xfree + 8 * i, 1);
-        for (int i = 0; i < 2; ++i) mbar_init(bar_drain + 8 * i, 1);
-        fence_mbar_init();
     }
     // The kernel that follows in the stream (launched with programmatic serialisation, as this one is) may start its
     // blocks as SMs become free; it reads nothing from global memory before its own grid_dependency_wait below.
@@ -169,18 +178,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         const uint32_t nb16 = (uint32_t)P.nb * P.bbuf_bytes / 16u;
         for (uint32_t i = tid; i < nb16; i += kTcThreads) sts128(b_s + i * 16u, zero);
         fence_proxy_async();
-        // Everything above touches this block's shared and tensor memory only.  From here on global memory is read and
-        // written: the kernel before this one in the stream (which may have produced x or the packed weights, or may
-        // still be reading what this one overwrites) has to be complete.
+        if (tid < P.nchunks * 2) reinterpret_cast<uint4 *>(tab)[tid] = tabw;
+        // Everything above touches this block's shared and tensor memory and the plan's chunk table only.  From here on
+        // what other kernels write is read and written: the kernel before this one in the stream (which may have
+        // produced x or the packed weights, or may still be reading what this one overwrites) has to be complete.
         grid_dependency_wait();
-        const uint4 *src = reinterpret_cast<const uint4 *>(P.chunks);
-        uint4 *dst = reinterpret_cast<uint4 *>(tab);
-        for (int i = tid; i < P.nchunks * 2; i += kTcThreads) {
-            uint4 w4 = __ldg(src + 2 * (int)P.order[i >> 1] + (i & 1));
-            if (i & 1) w4.z = P.ring[i >> 1];        // second half of the entry: slab0, flags, places in the rings, (unused)
-            dst[i] = w4;
-        }
-        for (int d = tid; d < P.Dpad_tot; d += kTcThreads) bias_sm[d] = d < P.bias_len ? __ldg(P.bias + d) : 0.f;
     }
     tc_fence_before();
     __syncthreads();
@@ -449,6 +451,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         const int rem = r - tn * hw;
         const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
         const bool issuer = warp == kTcEpiWarp0 && lane == 0;
+        // the bias is first needed here: these warps copy it while the first tile is being computed
+        for (int d = r; d < P.Dpad_tot; d += 128) bias_sm[d] = d < P.bias_len ? __ldg(P.bias + d) : 0.f;
+        named_bar_sync(1, 128);
 #pragma unroll 1
         for (int it = 0; it < my_items; ++it) {
             const int item = (int)blockIdx.x + it * (int)gridDim.x;
