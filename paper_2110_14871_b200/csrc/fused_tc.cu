@@ -73,6 +73,7 @@ struct alignas(64) TcParams {
     uint32_t tap_off[kTcMaxTaps];          // the A operand of tap (u, v) starts this many bytes into the box slot
     uint32_t a_sbo;              // GDW A operand: bytes between 8-pixel groups
     int nb, nx, nz, nw, nacc;
+    uint32_t dv_parts[2], dv_thw[2], dv_tw[2];   // multiplier and shift for the divisions by nparts, tiles_h * tiles_w, tiles_w
     int nbw;                     // builder warps that have rows to fill (32 rows each; the layer's largest chunk decides)
     uint32_t bbuf_bytes, bplane, xslot_bytes, wslab_bytes;
     uint32_t off_b, off_z, off_w, off_x, off_tab;    // from the 1024-aligned base; the output staging comes first
@@ -108,6 +109,10 @@ __device__ __forceinline__ void tc_warp_arrive(uint32_t bar)
 struct SlabRing {
     int head = 0, free_slabs = 0, oldest = 0;
 };
+
+// n / d for n < 2^31 as a multiplication: md = (ceil(2^(31+s) / d), 31 + s) with s = ceil(log2 d) is exact in that range
+// (a division by a run-time value is some fifty instructions, and the work item's coordinates need three of them).
+__device__ __forceinline__ int tc_fdiv(int n, const uint32_t (&md)[2]) { return (int)(((uint64_t)(uint32_t)n * md[0]) >> md[1]); }
 
 // Filters of more than 9 taps: a B buffer holds the operands of up to 13 taps at a time (8 for k = 4), and a chunk's GDW
 // products are issued group by group as the groups' operands arrive, all into the same accumulator.
@@ -316,15 +321,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         if (lane == 0) {
             // ---------------- input loader ----------------
             int box = 0, u = 0;
-            uint32_t xslot = 0;
+            uint32_t xslot = 0, xuse = 0;      // slot of the next box, and how often that slot has been used
             bool stop = false;
 #pragma unroll 1
             for (int it = 0; it < my_items && !stop; ++it) {
                 const int item = (int)blockIdx.x + it * (int)gridDim.x;
-                int tile = item / P.nparts;
-                const int bn = tile / tiles_hw;
+                int tile = tc_fdiv(item, P.dv_parts);
+                const int bn = tc_fdiv(tile, P.dv_thw);
                 tile -= bn * tiles_hw;
-                const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+                const int bh = tc_fdiv(tile, P.dv_tw), bw = tile - bh * P.tiles_w;
                 const int n0 = bn * P.TN, hi0 = bh * P.PH, wi0 = bw * P.PW;     // the copies' offsets carry the padding
 #pragma unroll 1
                 for (int q = 0; q < P.nchunks; ++q, ++u) {
@@ -341,14 +346,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     if (*vabort) { stop = true; break; }       // a wait ran out somewhere: no new copies
                     if (!(flags & 1)) { mbar_arrive(bar); continue; }
                     if (box >= P.nx)
-                        tc_wait(bar_xfree + 8 * xslot, (uint32_t)((box / P.nx) - 1) & 1u, &abort_flag, P.status, kStatusWaitStage);
+                        tc_wait(bar_xfree + 8 * xslot, (xuse - 1u) & 1u, &abort_flag, P.status, kStatusWaitStage);
                     mbar_expect_tx(bar, (uint32_t)P.xbox_bytes);
                     const uint32_t dst = x_s + xslot * P.xslot_bytes;
 #pragma unroll 1
                     for (int l = 0; l < P.nloads; ++l)
                         tma_load_4d(dst + P.load_off[l], &P.tmap_xp[P.load_map[l]], cbase, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, bar);
                     ++box;
-                    if (++xslot == (uint32_t)P.nx) xslot = 0;
+                    if (++xslot == (uint32_t)P.nx) { xslot = 0; ++xuse; }
                 }
             }
             // Teardown: no box copy may be in flight when the block ends.  This thread arrived for units 0 .. u-1; the
@@ -373,7 +378,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 if (v >= wdep) tc_wait(bar_pwdone + 8 * ((v - wdep) & 3), (uint32_t)((v - wdep) >> 2) & 1u, &abort_flag, P.status, kStatusWaitStage);
                 if (*vabort) break;                            // a wait ran out somewhere: no new copies
                 issued = v + 1;
-                const int part = P.nparts == 1 ? 0 : ((int)blockIdx.x + it * (int)gridDim.x) % P.nparts;
+                const int item = (int)blockIdx.x + it * (int)gridDim.x;
+                const int part = P.nparts == 1 ? 0 : item - tc_fdiv(item, P.dv_parts) * P.nparts;
                 const uint32_t bar = bar_pwready + 8 * (v & 3);
                 mbar_expect_tx(bar, (uint32_t)ns * P.wslab_bytes);
                 const uint16_t *src = P.pw + ((size_t)part * P.nslabs_total + slab0) * 16 * P.Dloc;
@@ -454,20 +460,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         // the bias is first needed here: these warps copy it while the first tile is being computed
         for (int d = r; d < P.Dpad_tot; d += 128) bias_sm[d] = d < P.bias_len ? __ldg(P.bias + d) : 0.f;
         named_bar_sync(1, 128);
+        int buf = 0;
+        uint32_t accuse = 0;          // accumulator of the tile in turn, and how often it has been used
 #pragma unroll 1
         for (int it = 0; it < my_items; ++it) {
             const int item = (int)blockIdx.x + it * (int)gridDim.x;
-            int tile = item / P.nparts;
+            int tile = tc_fdiv(item, P.dv_parts);
             const int part = item - tile * P.nparts;
-            const int bn = tile / tiles_hw;
+            const int bn = tc_fdiv(tile, P.dv_thw);
             tile -= bn * tiles_hw;
-            const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+            const int bh = tc_fdiv(tile, P.dv_tw), bw = tile - bh * P.tiles_w;
             const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
             const bool live = n < P.N && ho < P.Ho && wo < P.Wo;
             const size_t yrow = (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.D + part * P.Dloc;   // element index of the row's first channel
             const int dvalid = P.D - part * P.Dloc < P.Dloc ? P.D - part * P.Dloc : P.Dloc;
-            const int buf = it % P.nacc;
-            tc_warp_wait_call(bar_accfull + 8 * buf, (uint32_t)(it / P.nacc) & 1u, &abort_flag, P.status, kStatusWaitMma);
+            tc_warp_wait_call(bar_accfull + 8 * buf, accuse & 1u, &abort_flag, P.status, kStatusWaitMma);
             tc_fence_after();
             const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * 128);
             const uint32_t bias_part = bias_s + (uint32_t)(part * P.Dloc) * 4u;
@@ -524,6 +531,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                 tc_fence_before();
                 tc_warp_arrive(bar_accfree + 8 * buf);
             }
+            if (++buf == P.nacc) { buf = 0; ++accuse; }
         }
         if (P.ostage && issuer) bulk_wait_all();
     } else if (warp >= kTcBuildWarp0 && warp < kTcBuildWarp0 + P.nbw) {
@@ -975,6 +983,13 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     P.rec_hw = p->tc_rec_hw; P.nslabs_total = p->tc_nslabs;
     P.bias_len = p->Dpad;
     P.nbw = std::min(kTcBuildWarps, (m * 16 + 31) / 32);
+    auto magic = [](int d, uint32_t (&md)[2]) {
+        int sh = 0;
+        while ((1 << sh) < d) ++sh;
+        md[0] = (uint32_t)((((uint64_t)1 << (31 + sh)) + (uint64_t)d - 1) / (uint64_t)d);
+        md[1] = (uint32_t)(31 + sh);
+    };
+    magic(p->tc_nparts, P.dv_parts); magic(g.tiles_h * g.tiles_w, P.dv_thw); magic(g.tiles_w, P.dv_tw);
 
     const int grid = (int)(nitems < p->sm_count ? nitems : p->sm_count);
     cudaError_t e = cudaSuccess;
