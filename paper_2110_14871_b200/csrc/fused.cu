@@ -43,6 +43,7 @@ struct alignas(64) FusedParams {
     int *status;
     int N, H, W, C, Ho, Wo, D, Dpad, G, nchunks, stride, pad, relu;
     int TN, PH, PW, tiles_h, tiles_w, ntiles;
+    uint32_t dv_thw[2], dv_tw[2];   // multiplier and shift for the divisions by tiles_h * tiles_w and by tiles_w
     int IH, IW, ps, nslots, nwslots, nboxes, nsb, wstride;
     int spg_shift;                 // log2 of the operand stages per depthwise group (0 or 1)
     int ostage;                    // bytes of output staging (0: the epilogue stores rows directly)
@@ -86,6 +87,10 @@ __device__ __forceinline__ void warp_arrive(uint32_t bar)
     __syncwarp();
     if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
 }
+
+// n / d for n < 2^31 as a multiplication: md = (ceil(2^(31+s) / d), 31 + s) with s = ceil(log2 d) is exact in that range
+// (a division by a run-time value is some fifty instructions; a tile's coordinates need two of them).
+__device__ __forceinline__ int fdiv31(int n, const uint32_t (&md)[2]) { return (int)(((uint64_t)(uint32_t)n * md[0]) >> md[1]); }
 
 template <int N> __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -482,11 +487,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             const uint32_t spg_mask = (1u << P.spg_shift) - 1u;
             uint32_t sb = 0, pb = 0;          // weight-ring slot and its phase parity
             uint32_t gq = 0;
-            for (int tl = 0; tl < my_tiles; ++tl) {
-                const int buf = tl % P.nacc;
+            int buf = 0;
+            uint32_t accuse = 0;              // accumulator of the tile in turn, and how often it has been used
+            for (int tl = 0; tl < my_tiles; ++tl, buf = (buf + 1 == P.nacc ? 0 : buf + 1), accuse += (buf == 0)) {
                 const uint32_t d_tmem = tmem + (uint32_t)(buf * P.acc_cols);
-                if (tl >= P.nacc)
-                    mbar_wait_call(bar_accfree + 8 * buf, ((tl / P.nacc) - 1) & 1, &abort_flag, P.status, kStatusWaitStage);
+                if (accuse)
+                    mbar_wait_call(bar_accfree + 8 * buf, (accuse - 1u) & 1u, &abort_flag, P.status, kStatusWaitStage);
                 for (int q = 0; q < P.nchunks; ++q, ++gq) {
                     // chunk gq is the (gq >> 1)-th chunk of group gq & 1, which cycles through its own stages
                     const uint32_t sa = ((gq & 1u) << P.spg_shift) + ((gq >> 1) & spg_mask);
@@ -562,9 +568,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
             bool stop = false;
             for (int tl = 0; tl < my_tiles && !stop; ++tl) {
                 int tile = bid + tl * nblocks;
-                const int bn = tile / tiles_hw;
+                const int bn = fdiv31(tile, P.dv_thw);
                 tile -= bn * tiles_hw;
-                const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+                const int bh = fdiv31(tile, P.dv_tw), bw = tile - bh * P.tiles_w;
                 const int n0 = bn * P.TN, hi0 = bh * P.PH * P.stride - P.pad, wi0 = bw * P.PW * P.stride - P.pad;
                 for (int q = 0; q < P.nchunks; ++q, ++gq) {
                     const int4 meta = meta_tab[q];
@@ -632,9 +638,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         int wq = 0;                                       // ZOUT: running index of the next finished chunk
         for (int tl = 0; tl < my_tiles; ++tl) {
             int tile = bid + tl * nblocks;
-            const int bn = tile / tiles_hw;
+            const int bn = fdiv31(tile, P.dv_thw);
             tile -= bn * tiles_hw;
-            const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+            const int bh = fdiv31(tile, P.dv_tw), bw = tile - bh * P.tiles_w;
             const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
             const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
             const size_t yrow = (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.Dtot + part * P.Dpad;   // element index of the row's first channel
@@ -656,8 +662,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
                 }
                 continue;
             }
-            const int buf = tl % P.nacc;
-            warp_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
+            const int buf = tl & (P.nacc - 1);            // one or two accumulators
+            warp_wait(bar_accfull + 8 * buf, (tl >> (P.nacc - 1)) & 1, &abort_flag, P.status, kStatusWaitMma);
             tc_fence_after();
             const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * P.acc_cols);
             if (P.ostage) {
@@ -776,14 +782,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
         const int rem = r - tn * hw;
         const int ph = rem / P.PW, pw_ = rem - (rem / P.PW) * P.PW;
         int tile = bid + tl * nblocks;
-        const int bn = tile / tiles_hw;
+        const int bn = fdiv31(tile, P.dv_thw);
         tile -= bn * tiles_hw;
-        const int bh = tile / P.tiles_w, bw = tile - bh * P.tiles_w;
+        const int bh = fdiv31(tile, P.dv_tw), bw = tile - bh * P.tiles_w;
         const int n = bn * P.TN + tn, ho = bh * P.PH + ph, wo = bw * P.PW + pw_;
         const bool live = tn < P.TN && n < P.N && ho < P.Ho && wo < P.Wo;
         const size_t yrow = (((size_t)n * P.Ho + ho) * P.Wo + wo) * P.Dtot + part * P.Dpad;
-        const int buf = tl % P.nacc;
-        warp_wait(bar_accfull + 8 * buf, (tl / P.nacc) & 1, &abort_flag, P.status, kStatusWaitMma);
+        const int buf = tl & (P.nacc - 1);            // one or two accumulators
+        warp_wait(bar_accfull + 8 * buf, (tl >> (P.nacc - 1)) & 1, &abort_flag, P.status, kStatusWaitMma);
         tc_fence_after();
         const uint32_t t_base = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(buf * P.acc_cols);
         epilogue_row(P, t_base, bias_s, yrow, live, 1 + ((warp - kDwWarp0) >> 2), kTailShare);
@@ -888,6 +894,15 @@ static gdws_status_t run_tiled(gdws_plan_s *p, const gdws_tensor_t *x, void *out
     P.G = p->G; P.nchunks = p->nchunks; P.stride = p->stride; P.pad = p->pad;
     P.relu = (p->opt_relu ? kOutRelu : 0) | (out_f32 ? kOutF32 : 0);
     P.TN = t.TN; P.PH = t.PH; P.PW = t.PW; P.tiles_h = t.tiles_h; P.tiles_w = t.tiles_w; P.ntiles = (int)t.tiles();
+    {
+        auto magic = [](int d, uint32_t (&md)[2]) {
+            int sh = 0;
+            while ((1 << sh) < d) ++sh;
+            md[0] = (uint32_t)((((uint64_t)1 << (31 + sh)) + (uint64_t)d - 1) / (uint64_t)d);
+            md[1] = (uint32_t)(31 + sh);
+        };
+        magic(t.tiles_h * t.tiles_w, P.dv_thw); magic(t.tiles_w, P.dv_tw);
+    }
     P.IH = t.IH; P.IW = t.IW; P.ps = t.cbox * 2; P.nslots = t.nslots; P.nwslots = t.nwslots; P.nboxes = p->nboxes; P.nsb = t.nsb; P.wstride = p->wstride;
     P.spg_shift = t.spg == 2 ? 1 : 0;
     P.ostage = tma_out ? t.ostage : 0;
