@@ -74,6 +74,7 @@ struct alignas(64) TcParams {
     uint32_t a_sbo;              // GDW A operand: bytes between 8-pixel groups
     int nb, nx, nz, nw, nacc;
     uint32_t dv_parts[2], dv_thw[2], dv_tw[2];   // multiplier and shift for the divisions by nparts, tiles_h * tiles_w, tiles_w
+    int first_cbase;             // first input channel of the window the block takes first
     int nbw;                     // builder warps that have rows to fill (32 rows each; the layer's largest chunk decides)
     uint32_t bbuf_bytes, bplane, xslot_bytes, wslab_bytes;
     uint32_t off_b, off_z, off_w, off_x, off_tab;    // from the 1024-aligned base; the output staging comes first
@@ -188,6 +189,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
         // what other kernels write is read and written: the kernel before this one in the stream (which may have
         // produced x or the packed weights, or may still be reading what this one overwrites) has to be complete.
         grid_dependency_wait();
+        // The block's first input box is asked for right here, by the thread that initialised its barrier (the loader's
+        // lane, which skips this box later): it is what the first products wait for longest.
+        if (tid == 32 && (int)blockIdx.x < P.nitems) {
+            const int item = (int)blockIdx.x;
+            int tile = tc_fdiv(item, P.dv_parts);
+            const int bn = tc_fdiv(tile, P.dv_thw);
+            tile -= bn * (P.tiles_h * P.tiles_w);
+            const int bh = tc_fdiv(tile, P.dv_tw), bw = tile - bh * P.tiles_w;
+            mbar_expect_tx(bar_dwready, (uint32_t)P.xbox_bytes);
+#pragma unroll 1
+            for (int l = 0; l < P.nloads; ++l)
+                tma_load_4d(x_s + P.load_off[l], &P.tmap_xp[P.load_map[l]], P.first_cbase, bw * P.PW + P.load_dw[l], bh * P.PH + P.load_dh[l],
+                            bn * P.TN, bar_dwready);
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -347,11 +362,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) fused_tc_kernel(const __grid_co
                     if (!(flags & 1)) { mbar_arrive(bar); continue; }
                     if (box >= P.nx)
                         tc_wait(bar_xfree + 8 * xslot, (xuse - 1u) & 1u, &abort_flag, P.status, kStatusWaitStage);
-                    mbar_expect_tx(bar, (uint32_t)P.xbox_bytes);
-                    const uint32_t dst = x_s + xslot * P.xslot_bytes;
+                    if (u > 0) {       // the block's first box was asked for in the prologue
+                        mbar_expect_tx(bar, (uint32_t)P.xbox_bytes);
+                        const uint32_t dst = x_s + xslot * P.xslot_bytes;
 #pragma unroll 1
-                    for (int l = 0; l < P.nloads; ++l)
-                        tma_load_4d(dst + P.load_off[l], &P.tmap_xp[P.load_map[l]], cbase, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, bar);
+                        for (int l = 0; l < P.nloads; ++l)
+                            tma_load_4d(dst + P.load_off[l], &P.tmap_xp[P.load_map[l]], cbase, wi0 + P.load_dw[l], hi0 + P.load_dh[l], n0, bar);
+                    }
                     ++box;
                     if (++xslot == (uint32_t)P.nx) { xslot = 0; ++xuse; }
                 }
@@ -983,6 +1000,7 @@ gdws_status_t bf16_fused_tc(gdws_plan_s *p, const gdws_tensor_t *x, gdws_tensor_
     P.rec_hw = p->tc_rec_hw; P.nslabs_total = p->tc_nslabs;
     P.bias_len = p->Dpad;
     P.nbw = std::min(kTcBuildWarps, (m * 16 + 31) / 32);
+    P.first_cbase = p->tc_chunks[P.order[0]].cbase;
     auto magic = [](int d, uint32_t (&md)[2]) {
         int sh = 0;
         while ((1 << sh) < d) ++sh;
