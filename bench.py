@@ -68,9 +68,9 @@ def layer_numbers(spec: gi.LayerSpec, G: int):
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (key: config, layer, path, GDW stage).  An entry is removed when its kernel changes.
 TRAFFIC_BYTES_PER_LAUNCH = {
-    (1, 0, "fused", 2): 9180160,      # x + weights; y (8.39 MB) stays in L2 within the captured launch
-    (2, 0, "fused", 1): 25803264,     # x + weights; y (25.7 MB) stays in L2
-    (3, 0, "fused", 2): 92920064,     # x (67.1 MB) + the part of y that left L2
+    (1, 0, "fused", 2): 9180928,      # x + weights; y (8.39 MB) stays in L2 within the captured launch
+    (2, 0, "fused", 1): 25805312,     # x + weights; y (25.7 MB) stays in L2
+    (3, 0, "fused", 2): 94107136,     # x (67.1 MB) + the part of y that left L2
 }
 
 
