@@ -421,25 +421,28 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_bf16_kernel(const __gr
     int4 *meta_tab = reinterpret_cast<int4 *>(base + (w_s - a_s) + (size_t)P.nwslots * wblock);
 
     grid_launch_dependents();      // the next kernel in the stream may start its prologue as SMs become free
-    if (tid == 0) {
-        abort_flag = 0;
-        for (int i = 0; i < 4; ++i) {
-            mbar_init(bar_afree + 8 * i, ZOUT ? kEpiWarps : 1);
-            mbar_init(bar_open + 8 * i, 1);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_accfull + 8 * i, 1);
-            mbar_init(bar_accfree + 8 * i, kEpiWarps);
-        }
-        mbar_init(bar_drain, 1);
-        for (int i = 0; i < kMaxBUnits; ++i) { mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1); }
-        for (int i = 0; i < kMaxSlots; ++i) {
+    if (tid == 0) abort_flag = 0;
+    {
+        // Eight threads of warp 1 initialise the barriers, one ring slot each (warp 0 allocates tensor memory meanwhile).
+        static_assert(kMaxBUnits == 8 && kMaxSlots == 8, "one ring slot per initialising thread");
+        const int i = tid - 32;
+        if (i >= 0 && i < 8) {
+            if (i < 4) {
+                mbar_init(bar_afree + 8 * i, ZOUT ? kEpiWarps : 1);
+                mbar_init(bar_open + 8 * i, 1);
+            }
+            if (i < 2) {
+                mbar_init(bar_accfull + 8 * i, 1);
+                mbar_init(bar_accfree + 8 * i, kEpiWarps);
+            }
+            if (i == 0) mbar_init(bar_drain, 1);
+            mbar_init(bar_bfull + 8 * i, 1); mbar_init(bar_bfree + 8 * i, 1);
             mbar_init(bar_xfull + 8 * i, 1);
             mbar_init(bar_xfree + 8 * i, 2 * kDwGroupWarps);   // the last two chunks that use a box release it, warp by warp
             mbar_init(bar_wfull + 8 * i, 1);
             mbar_init(bar_wfree + 8 * i, kDwGroupWarps);
+            fence_mbar_init();
         }
-        fence_mbar_init();
     }
     if (!ZOUT && warp == kCtrlWarp) tmem_alloc(smem_u32(&tmem_slot), (uint32_t)(P.nacc * P.acc_cols));
     // up to here only this block's shared and tensor memory were touched; the kernel before this one in the stream has
