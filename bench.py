@@ -69,8 +69,8 @@ def layer_numbers(spec: gi.LayerSpec, G: int):
 # summarised under profiles/ (key: config, layer, path, GDW stage).  An entry is removed when its kernel changes.
 TRAFFIC_BYTES_PER_LAUNCH = {
     (1, 0, "fused", 2): 9180928,      # x + weights; y (8.39 MB) stays in L2 within the captured launch
-    (2, 0, "fused", 1): 25805312,     # x + weights; y (25.7 MB) stays in L2
-    (3, 0, "fused", 2): 94107136,     # x (67.1 MB) + the part of y that left L2
+    (2, 0, "fused", 1): 25794304,     # x + weights; y (25.7 MB) stays in L2
+    (3, 0, "fused", 2): 93909504,     # x (67.1 MB) + the part of y that left L2
 }
 
 
